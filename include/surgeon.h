@@ -43,7 +43,9 @@ typedef enum {
   SURGEON_ERR_DEGENERATE = 3,       /* Eq. 7 is 0/0 for this input; output filled with zeros          */
   SURGEON_ERR_UNSUPPORTED = 4,      /* layer geometry / dtype / size the library does not implement   */
   SURGEON_ERR_CUDA = 5,             /* a CUDA runtime call failed                                     */
-  SURGEON_ERR_TIMEOUT = 6           /* device-side bounded wait expired (only in surgeon_header)      */
+  SURGEON_ERR_TIMEOUT = 6,          /* device-side bounded wait expired (only in surgeon_header)      */
+  SURGEON_ERR_INTERNAL = 7          /* device-side self-check failed, e.g. the kept count does not
+                                       add up (only in surgeon_header)                                */
 } surgeon_status;
 
 typedef enum { SURGEON_F32 = 0, SURGEON_BF16 = 1 } surgeon_dtype;

@@ -1,0 +1,190 @@
+// extern "C" entry points of libsurgeon: argument checks and host-side arithmetic; every step
+// that touches tensor data is a kernel launched from the other translation units.
+#include <math.h>
+
+#include "surgeon_internal.cuh"
+
+namespace surgeon {
+
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Algorithm 1 line 6: kept count for `ratio`; one double multiply, one floor.
+inline int64_t kept_count(int64_t n, double ratio) {
+  double pruned = floor(ratio * static_cast<double>(n));
+  if (pruned < 0.0) pruned = 0.0;
+  int64_t np = static_cast<int64_t>(pruned);
+  if (np > n) np = n;
+  return n - np;
+}
+
+bool desc_ok(const surgeon_layer_desc* d, surgeon_status* why) {
+  *why = SURGEON_ERR_INVALID_ARG;
+  if (!d) return false;
+  if (d->kind != 0 && d->kind != 1) return false;
+  if (d->path != 0 && d->path != 1) return false;
+  if (d->batch <= 0 || d->c_in <= 0 || d->c_out <= 0 || d->h <= 0 || d->w <= 0) return false;
+  if (d->kh <= 0 || d->kw <= 0 || d->stride <= 0 || d->pad < 0) return false;
+  if (d->kind == 0 && (d->h != 1 || d->w != 1 || d->kh != 1 || d->kw != 1 || d->stride != 1 ||
+                       d->pad != 0))
+    return false;
+  if (d->h + 2 * d->pad < d->kh || d->w + 2 * d->pad < d->kw) return false;
+  *why = SURGEON_ERR_UNSUPPORTED;
+  const long long oh = (d->h + 2 * d->pad - d->kh) / d->stride + 1;
+  const long long ow = (d->w + 2 * d->pad - d->kw) / d->stride + 1;
+  const long long lim = 2147483647LL;
+  if (static_cast<long long>(d->batch) * d->c_in * d->h * d->w > lim) return false;
+  if (static_cast<long long>(d->batch) * d->c_out * oh * ow > lim) return false;
+  if (static_cast<long long>(d->c_out) * d->c_in * d->kh * d->kw > lim) return false;
+  if (d->pad >= d->kh || d->pad >= d->kw) return false;  // windows entirely in the padding
+  *why = SURGEON_OK;
+  return true;
+}
+
+}  // namespace
+}  // namespace surgeon
+
+using namespace surgeon;
+
+extern "C" {
+
+surgeon_status surgeon_layer_ratios(const double* gi, const double* lam, int32_t n_layers,
+                                    double* ratios_out) {
+  if (!gi || !lam || !ratios_out || n_layers <= 0) return SURGEON_ERR_INVALID_ARG;
+  double total = 0.0, g_max = 0.0;
+  for (int i = 0; i < n_layers; ++i) {
+    if (!isfinite(gi[i]) || gi[i] < 0.0 || !isfinite(lam[i]) || !(lam[i] > 0.0))
+      return SURGEON_ERR_INVALID_ARG;
+    total += lam[i];
+    if (gi[i] > g_max) g_max = gi[i];
+  }
+  // Eq. 5: M_i = -log(m_i / sum m); kept in ratios_out until Eq. 6 overwrites it.
+  double m_max = 0.0;
+  for (int i = 0; i < n_layers; ++i) {
+    const double mi = -log(lam[i] / total);
+    ratios_out[i] = mi;
+    if (mi > m_max) m_max = mi;
+  }
+  // Eq. 6: I_i = (M_i / max M) * (G_i / max G).
+  double i_max = 0.0;
+  for (int i = 0; i < n_layers; ++i) {
+    const double imp = (m_max > 0.0 && g_max > 0.0) ? (ratios_out[i] / m_max) * (gi[i] / g_max) : 0.0;
+    ratios_out[i] = imp;
+    if (imp > i_max) i_max = imp;
+  }
+  if (!(i_max > 0.0)) {
+    for (int i = 0; i < n_layers; ++i) ratios_out[i] = 0.0;
+    return SURGEON_ERR_DEGENERATE;
+  }
+  // Eq. 7: p_i = 1 - I_i / max I.
+  for (int i = 0; i < n_layers; ++i) ratios_out[i] = 1.0 - ratios_out[i] / i_max;
+  return SURGEON_OK;
+}
+
+surgeon_status surgeon_compact_sizes(int64_t n, surgeon_dtype dt, double ratio, int64_t* n_keep,
+                                     size_t* bitmap_bytes, size_t* values_bytes,
+                                     size_t* offsets_bytes, size_t* workspace_bytes) {
+  if (n < 0 || !(ratio >= 0.0 && ratio <= 1.0) || (dt != SURGEON_F32 && dt != SURGEON_BF16))
+    return SURGEON_ERR_INVALID_ARG;
+  if (n > SURGEON_MAX_N) return SURGEON_ERR_UNSUPPORTED;
+  const int64_t k = kept_count(n, ratio);
+  if (n_keep) *n_keep = k;
+  if (bitmap_bytes) *bitmap_bytes = static_cast<size_t>((n + 31) / 32) * 4;
+  if (values_bytes) *values_bytes = static_cast<size_t>(k) * (dt == SURGEON_F32 ? 4 : 2);
+  if (offsets_bytes)
+    *offsets_bytes = static_cast<size_t>((n + SURGEON_BLOCK - 1) / SURGEON_BLOCK + 1) * 8;
+  if (workspace_bytes) *workspace_bytes = prune_workspace_bytes(n);
+  return SURGEON_OK;
+}
+
+surgeon_status surgeon_prune_compact(const void* x, int64_t n, surgeon_dtype dt, double ratio,
+                                     surgeon_compressed* out, void* workspace,
+                                     size_t workspace_bytes, void* cuda_stream) {
+  if (!out || n < 0 || !(ratio >= 0.0 && ratio <= 1.0) ||
+      (dt != SURGEON_F32 && dt != SURGEON_BF16))
+    return SURGEON_ERR_INVALID_ARG;
+  if (n > SURGEON_MAX_N) return SURGEON_ERR_UNSUPPORTED;
+  const int64_t k = kept_count(n, ratio);
+  if (!out->header || !out->block_offsets || !workspace) return SURGEON_ERR_INVALID_ARG;
+  if (n > 0 && (!x || !out->bitmap)) return SURGEON_ERR_INVALID_ARG;
+  if (k > 0 && !out->values) return SURGEON_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(out->bitmap) || !aligned16(out->values) ||
+      !aligned16(out->block_offsets) || !aligned16(out->header) || !aligned16(workspace))
+    return SURGEON_ERR_INVALID_ARG;
+  if (workspace_bytes < prune_workspace_bytes(n)) return SURGEON_ERR_BUFFER_TOO_SMALL;
+  out->n = n;
+  out->dt = static_cast<int32_t>(dt);
+  out->reserved = 0;
+  const cudaError_t e = launch_prune_compact(x, n, static_cast<int>(dt), k, *out, workspace,
+                                             static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? SURGEON_OK : SURGEON_ERR_CUDA;
+}
+
+size_t surgeon_weight_grad_workspace(const surgeon_layer_desc* d) {
+  surgeon_status why;
+  if (!desc_ok(d, &why)) return 0;
+  const size_t b = d->path == 1 ? weight_grad_fp32_workspace(*d) : weight_grad_tc_workspace(*d);
+  return (b + 255) & ~static_cast<size_t>(255);
+}
+
+surgeon_status surgeon_weight_grad(const surgeon_compressed* act, const surgeon_layer_desc* d,
+                                   const float* grad_out, float* dw, int32_t accumulate,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  surgeon_status why;
+  if (!desc_ok(d, &why)) return why;
+  if (!act || !grad_out || !dw || !act->bitmap || !act->block_offsets) return SURGEON_ERR_INVALID_ARG;
+  if (act->dt != SURGEON_F32 && act->dt != SURGEON_BF16) return SURGEON_ERR_INVALID_ARG;
+  if (act->n != static_cast<int64_t>(d->batch) * d->c_in * d->h * d->w) return SURGEON_ERR_INVALID_ARG;
+  if (!aligned16(act->bitmap) || !aligned16(act->values) || !aligned16(act->block_offsets) ||
+      !aligned16(grad_out) || !aligned16(dw) || !aligned16(workspace))
+    return SURGEON_ERR_INVALID_ARG;
+  const size_t need = surgeon_weight_grad_workspace(d);
+  if (need > 0 && (!workspace || workspace_bytes < need)) return SURGEON_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const cudaError_t e =
+      d->path == 1 ? launch_weight_grad_fp32(*act, *d, grad_out, dw, accumulate ? 1 : 0, workspace, s)
+                   : launch_weight_grad_tc(*act, *d, grad_out, dw, accumulate ? 1 : 0, workspace, s);
+  if (e == cudaErrorNotSupported) return SURGEON_ERR_UNSUPPORTED;
+  return e == cudaSuccess ? SURGEON_OK : SURGEON_ERR_CUDA;
+}
+
+surgeon_status surgeon_decompress(const surgeon_compressed* act, void* x_out, void* cuda_stream) {
+  if (!act || act->n < 0 || (act->dt != SURGEON_F32 && act->dt != SURGEON_BF16))
+    return SURGEON_ERR_INVALID_ARG;
+  if (act->n > 0 && (!x_out || !act->bitmap || !act->block_offsets)) return SURGEON_ERR_INVALID_ARG;
+  if (!aligned16(x_out) || !aligned16(act->bitmap) || !aligned16(act->values) ||
+      !aligned16(act->block_offsets))
+    return SURGEON_ERR_INVALID_ARG;
+  const cudaError_t e = launch_decompress(*act, x_out, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? SURGEON_OK : SURGEON_ERR_CUDA;
+}
+
+const char* surgeon_status_string(surgeon_status s) {
+  switch (s) {
+    case SURGEON_OK: return "ok";
+    case SURGEON_ERR_INVALID_ARG: return "invalid argument";
+    case SURGEON_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+    case SURGEON_ERR_DEGENERATE: return "degenerate input (ratio rule is 0/0)";
+    case SURGEON_ERR_UNSUPPORTED: return "unsupported geometry, dtype or size";
+    case SURGEON_ERR_CUDA: return "CUDA runtime error";
+    case SURGEON_ERR_TIMEOUT: return "device-side bounded wait expired";
+    case SURGEON_ERR_INTERNAL: return "device-side self-check failed";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

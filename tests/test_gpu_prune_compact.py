@@ -1,0 +1,126 @@
+"""GPU parity: surgeon_prune_compact / surgeon_decompress through the C ABI vs the CPU oracle,
+bit for bit (threshold key, kept count, tie quota, bitmap, packed values, block offsets)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2503_20354_b200 import binding as B
+from paper_2503_20354_b200 import workloads as W
+from gpu_util import assert_store_equals_oracle
+
+pytestmark = pytest.mark.gpu
+
+RATIOS_CFG1 = (0.0, 0.3, 0.6, 0.9, 1.0)
+
+
+def _as(x32: torch.Tensor, bf16: bool) -> torch.Tensor:
+    return x32.to(torch.bfloat16) if bf16 else x32
+
+
+@pytest.mark.parametrize("ratio", RATIOS_CFG1)
+def test_config1_tiny_conv_activation(ratio):
+    layer = W.tiny_conv()[0]
+    x = W.activation(layer, seed=0)
+    comp, ref = assert_store_equals_oracle(x, ratio)
+    # decompress on the device gives the oracle's dense pruned tensor bitwise
+    dense = B.surgeon_decompress(comp).cpu().numpy()
+    exp = oracle.decompress(ref["bitmap"], ref["values"], x.numel())
+    assert np.array_equal(dense.view(np.uint8), exp.view(np.uint8))
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 1023, 1024, 1025, 8191, 8192, 8193, 65536 + 7,
+                               3 * 8192 + 1000])
+def test_edge_sizes(n, bf16):
+    x = _as(W.draw("relu_normal", n, seed=1, tag=n), bf16)
+    for ratio in (0.0, 0.5, 0.77, 1.0):
+        assert_store_equals_oracle(x, ratio, method=0 if n < 5000 else 1)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_empty_tensor(bf16):
+    x = torch.empty(0, dtype=torch.bfloat16 if bf16 else torch.float32, device="cuda")
+    comp = B.surgeon_prune_compact(x, 0.5)
+    torch.cuda.synchronize()
+    _, _, offs, hdr = comp.to_numpy()
+    assert hdr.n_keep == 0 and hdr.status == 0 and offs.tolist() == [0]
+    assert hdr.threshold_key == (0xFFFF if bf16 else 0xFFFFFFFF)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("dist", ["relu_normal", "normal", "student_t2", "ties16", "gelu_normal"])
+def test_distributions_and_ratios(dist, bf16):
+    n = (1 << 20) + 4321   # many tiles and a ragged tail
+    x = _as(W.draw(dist, n, seed=2), bf16)
+    for ratio in (0.1, 0.5, 0.9, 0.99):
+        assert_store_equals_oracle(x, ratio)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_special_values(bf16):
+    x = W.draw("normal", 5000, seed=3)
+    x[7] = float("nan"); x[100] = float("inf"); x[101] = -float("inf"); x[9] = -0.0; x[10] = 0.0
+    x[4000:4100] = 0.0
+    x = _as(x, bf16)
+    for ratio in (0.0, 0.2, 0.999, 0.9998, 1.0):
+        assert_store_equals_oracle(x, ratio, method=0)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_all_equal_and_two_level(bf16):
+    # every key equal: the kept set is the first n_keep indices
+    x = _as(torch.full((20000,), 1.5), bf16)
+    for ratio in (0.25, 0.5, 0.9999):
+        comp, ref = assert_store_equals_oracle(x, ratio)
+        assert ref["c_gt"] == 0 and ref["q"] == ref["k"]
+    x = torch.zeros(30000)
+    x[::3] = -2.0
+    for ratio in (0.1, 0.6667, 0.9):
+        assert_store_equals_oracle(_as(x, bf16), ratio)
+
+
+def test_repeat_calls_are_bitwise_identical_and_reuse_buffers():
+    x = W.draw("ties16", 300000, seed=5).cuda()
+    comp = B.surgeon_prune_compact(x, 0.7)
+    a = [t.copy() if isinstance(t, np.ndarray) else t for t in comp.to_numpy()[:3]]
+    ws = torch.empty(comp.sizes.workspace_bytes, dtype=torch.uint8, device="cuda")
+    for _ in range(3):
+        B.surgeon_prune_compact(x, 0.7, out=comp, workspace=ws)
+        b = comp.to_numpy()[:3]
+        assert all(np.array_equal(u, v) for u, v in zip(a, b))
+
+
+def test_non_default_stream_and_canaries():
+    # outputs sit inside larger buffers; the words after each output must stay untouched
+    n = 50000 + 13
+    x = W.draw("normal", n, seed=6).cuda()
+    sizes = B.surgeon_compact_sizes(n, B.SURGEON_F32, 0.4)
+    comp = B.CompressedActivation(n, B.SURGEON_F32, 0.4, x.device, sizes)
+    pad = 64
+    big_bitmap = torch.full((sizes.bitmap_bytes // 4 + pad,), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+    big_vals = torch.full((sizes.n_keep + pad,), 12345.0, dtype=torch.float32, device="cuda")
+    big_offs = torch.full((sizes.offsets_bytes // 8 + pad,), 0x1234567, dtype=torch.int64, device="cuda")
+    comp.bitmap, comp.values, comp.block_offsets = big_bitmap, big_vals, big_offs
+    comp.c.bitmap, comp.c.values, comp.c.block_offsets = (big_bitmap.data_ptr(), big_vals.data_ptr(),
+                                                          big_offs.data_ptr())
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        B.surgeon_prune_compact(x, 0.4, out=comp, stream=s)
+    s.synchronize()
+    assert_store_equals_oracle(x.cpu(), 0.4, comp=comp)
+    assert torch.all(big_bitmap[sizes.bitmap_bytes // 4:] == 0x5A5A5A5A)
+    assert torch.all(big_vals[sizes.n_keep:] == 12345.0)
+    assert torch.all(big_offs[sizes.offsets_bytes // 8:] == 0x1234567)
+
+
+def test_argument_errors_on_device():
+    x = torch.zeros(1024, device="cuda")
+    comp = B.CompressedActivation(1024, 0, 0.5, x.device)
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.SurgeonError) as e:
+        B.surgeon_prune_compact(x, 0.5, out=comp, workspace=small)
+    assert e.value.status == B.SURGEON_ERR_BUFFER_TOO_SMALL
+    with pytest.raises(B.SurgeonError) as e:
+        B.surgeon_prune_compact(x[1:], 0.5)      # 4-byte aligned only
+    assert e.value.status == B.SURGEON_ERR_INVALID_ARG

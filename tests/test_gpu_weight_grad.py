@@ -1,0 +1,113 @@
+"""GPU parity: surgeon_weight_grad through the C ABI vs the fp64 oracle.
+
+Tolerance (relative Frobenius error against the fp64 oracle): 1e-5 for the fp32 CUDA-core path,
+5e-3 for the tensor-core path (bf16 operands, fp32 accumulation)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2503_20354_b200 import binding as B
+from paper_2503_20354_b200 import workloads as W
+from gpu_util import oracle_dw, rel_frobenius
+
+pytestmark = pytest.mark.gpu
+
+TOL = {B.PATH_FP32: 1e-5, B.PATH_TENSOR_CORE: 5e-3}
+PATHS = [B.PATH_FP32, B.PATH_TENSOR_CORE]
+
+
+def run_layer(layer, ratio, path, seed=0, sigma=0.01):
+    a = W.activation(layer, seed)
+    g = W.grad_out(layer, seed, sigma=sigma)
+    comp = B.surgeon_prune_compact(a.cuda(), ratio)
+    dw = B.surgeon_weight_grad(comp, B.layer_desc(layer, path), g.cuda())
+    torch.cuda.synchronize()
+    a_bits = W.as_numpy_bits(a).reshape(-1)
+    r = oracle.prune_compact(a_bits, ratio)
+    pruned = oracle.decompress(r["bitmap"], r["values"], a_bits.size)
+    ref = oracle_dw(layer, pruned, g.numpy())
+    return dw.cpu().numpy(), ref, a_bits, g.numpy()
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("ratio", [0.0, 0.3, 0.6, 0.9, 1.0])
+def test_config1_tiny_conv(ratio, path):
+    layer = W.tiny_conv()[0]
+    dw, ref, a_bits, g = run_layer(layer, ratio, path)
+    assert dw.shape == (64, 64, 3, 3)
+    if ratio == 1.0:
+        assert not dw.any()                     # empty store: exactly zero
+    else:
+        assert rel_frobenius(dw, ref) <= TOL[path]
+    if ratio == 0.0:                            # dense gradient computed from x itself
+        dense = oracle_dw(layer, a_bits, g)
+        assert rel_frobenius(dw, dense) <= TOL[path]
+
+
+SHAPES = [
+    # ragged tiles, strides, 1x1, 7x7 stem, FC-like and token-major linears
+    W.conv("c3x3_s2", 3, 20, 18, 24, 3, 2),
+    W.conv("c3x3_odd", 2, 17, 13, 70, 3, 1),
+    W.conv("c1x1", 4, 40, 14, 96, 1, 1, 0),
+    W.conv("c1x1_s2", 4, 64, 14, 130, 1, 2, 0),
+    W.conv("stem7x7", 2, 3, 64, 64, 7, 2, 3, dist="normal"),
+    W.conv("c3x3_7x7map", 5, 32, 7, 48, 3, 1),
+    W.conv("c3x3_nopad", 2, 8, 10, 8, 3, 1, 0),
+    W.linear("fc", 64, 2048, 1000, dist="abs_normal", dt=W.F32),
+    W.linear("tokens", 2 * 197, 768, 256, dist="normal", dt=W.F32),
+    W.linear("tiny", 5, 7, 3, dist="normal", dt=W.F32),
+]
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("layer", SHAPES, ids=lambda l: l.name)
+def test_layer_shapes(layer, bf16, path):
+    from dataclasses import replace
+    layer = replace(layer, dt=W.BF16 if bf16 else W.F32)
+    for ratio in (0.0, 0.7):
+        dw, ref, _, _ = run_layer(layer, ratio, path, seed=3)
+        assert rel_frobenius(dw, ref) <= TOL[path], (layer.name, ratio)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_accumulate_and_reproducible(path):
+    layer = W.conv("acc", 2, 16, 16, 32, 3)
+    a = W.activation(layer, 9).cuda()
+    g = W.grad_out(layer, 9).cuda()
+    comp = B.surgeon_prune_compact(a, 0.5)
+    d = B.layer_desc(layer, path)
+    dw1 = B.surgeon_weight_grad(comp, d, g)
+    dw2 = B.surgeon_weight_grad(comp, d, g)
+    assert torch.equal(dw1, dw2)                       # fixed summation order
+    acc = dw1.clone()
+    B.surgeon_weight_grad(comp, d, g, dw=acc, accumulate=True)
+    torch.testing.assert_close(acc, 2 * dw1, rtol=1e-6, atol=0)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_one_hot_gradient_gives_shifted_copy(path):
+    layer = W.conv("onehot", 2, 3, 6, 2, 3, 2, 1, dist="normal")
+    a = torch.arange(layer.n_act, dtype=torch.float32).reshape(layer.act_shape) + 1.0
+    g = torch.zeros(layer.grad_shape)
+    g[1, 1, 0, 2] = 1.0
+    comp = B.surgeon_prune_compact(a.cuda(), 0.0)
+    dw = B.surgeon_weight_grad(comp, B.layer_desc(layer, path), g.cuda()).cpu().numpy()
+    ref = oracle.dw_conv2d(a.numpy(), g.numpy(), 3, 3, 2, 1)
+    assert rel_frobenius(dw, ref) <= TOL[path] and not dw[0].any()
+
+
+def test_weight_grad_argument_errors():
+    layer = W.conv("err", 2, 4, 8, 4, 3)
+    a = W.activation(layer, 1).cuda()
+    g = W.grad_out(layer, 1).cuda()
+    comp = B.surgeon_prune_compact(a, 0.5)
+    d = B.layer_desc(layer, B.PATH_FP32)
+    with pytest.raises(B.SurgeonError) as e:
+        B.surgeon_weight_grad(comp, d, g, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == B.SURGEON_ERR_BUFFER_TOO_SMALL
+    wrong = B.layer_desc(W.conv("err2", 3, 4, 8, 4, 3), B.PATH_FP32)   # activation size mismatch
+    with pytest.raises(B.SurgeonError) as e:
+        B.surgeon_weight_grad(comp, wrong, g)
+    assert e.value.status == B.SURGEON_ERR_INVALID_ARG
