@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the dynamic-activation-sparsity hot path on B200.
+
+One step = one pass of the whole path over one batch of the WideResNet-28-10-shaped stack
+(batch 200, 28 conv layers, fp32 activations): per-layer ratios (Eq. 5-7), prune+compact of every
+saved activation (Algorithm 1 lines 6-7), and the weight gradient of every layer from its
+compressed store (lines 11-12).  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload wrn28|tiny|resnet50|vit] [--batch B] [--path tc|fp32]
+
+N > 1 (launched with torch.distributed.run): every rank runs an independent replica of the
+step on its own GPU (the path has no exchange step); time is the max over ranks.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "prune+compact GB/s and sparse-act dW TFLOP/s, as % of B200 HBM/tensor peak"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# fp32 CUDA-core peak for the fp32 path: 148 SMs x 128 FMA lanes x 2 flop x 1.965 GHz
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def get_layers(workload: str, batch):
+    from paper_2503_20354_b200 import workloads as W
+    if workload == "wrn28":
+        return W.wrn28_10(batch or 200), "WideResNet-28-10-shaped stack, 32x32, batch %d, fp32 activations" % (batch or 200)
+    if workload == "tiny":
+        return W.tiny_conv(batch or 16), "tiny conv 3x3 64->64 on [%d,64,32,32] fp32" % (batch or 16)
+    if workload == "resnet50":
+        return W.resnet50(batch or 64), "ResNet-50-shaped stack, 224x224, batch %d, bf16 activations" % (batch or 64)
+    if workload == "vit":
+        return W.vit_b16(batch or 64), "ViT-B/16-shaped stack, batch %d, bf16 activations" % (batch or 64)
+    raise SystemExit("unknown workload %r" % workload)
+
+
+def prune_alg_bytes(layer, n_keep: int) -> int:
+    """Algorithmic bytes of prune+compact: two reads of the tensor (one to find the threshold,
+    one to emit), the bitmap, the packed values and the block offsets."""
+    es = 4 if layer.dt == 0 else 2
+    n = layer.n_act
+    return 2 * n * es + (n + 7) // 8 + n_keep * es + 8 * ((n + 1023) // 1024 + 1)
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.lines, self.proc, self.idx = [], None, device_index
+
+    def start(self):
+        try:
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = vis.split(",")[self.idx] if vis else str(self.idx)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", idx, "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in self.lines:
+            f = [v.strip() for v in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus: int):
+    """(rank, world, device).  One process per GPU; rendezvous from the torchrun environment."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        if torch.cuda.is_available():
+            torch.cuda.set_device(local)
+        dist.init_process_group(backend=backend)
+    elif torch.cuda.is_available():
+        torch.cuda.set_device(0)
+    return rank, world, local
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    """Max of a per-rank scalar (the job's time is its slowest rank's)."""
+    if world == 1:
+        return float(value)
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+# ------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------
+
+class Stack:
+    """Device-resident inputs, stores, outputs and scratch of one replica of the workload."""
+
+    def __init__(self, layers, path: int, seed: int, device, worst_case_store=True):
+        from paper_2503_20354_b200 import binding as B
+        from paper_2503_20354_b200 import workloads as W
+        self.B, self.layers, self.path, self.device = B, layers, path, device
+        self.gi = W.gradient_importance(len(layers), seed)
+        self.lam = np.array([l.act_bytes for l in layers], dtype=np.float64)
+        self.x = [W.activation(l, seed, i, device=device) for i, l in enumerate(layers)]
+        self.g = [W.grad_out(l, seed, i, device=device) for i, l in enumerate(layers)]
+        self.desc = [B.layer_desc(l, path) for l in layers]
+        self.dw = [torch.empty(l.dw_shape, dtype=torch.float32, device=device) for l in layers]
+        # stores sized for ratio 0: ratios change every batch, the buffers do not
+        self.store = [B.CompressedActivation(l.n_act, l.dt, 0.0, device) for l in layers]
+        ws1 = max(s.sizes.workspace_bytes for s in self.store)
+        ws2 = max(B.surgeon_weight_grad_workspace(d) for d in self.desc)
+        self.ws = torch.empty(max(ws1, ws2, 256), dtype=torch.uint8, device=device)
+        self.ratios = None
+
+    def step(self, ev=None):
+        B = self.B
+        if ev: ev[0].record()
+        self.ratios = B.surgeon_layer_ratios(self.gi, self.lam, allow_degenerate=True)   # Eq. 5-7
+        for i in range(len(self.layers)):                                                # forward
+            B.surgeon_prune_compact(self.x[i], float(self.ratios[i]), out=self.store[i], workspace=self.ws)
+        if ev: ev[1].record()
+        for i in reversed(range(len(self.layers))):                                      # backward
+            B.surgeon_weight_grad(self.store[i], self.desc[i], self.g[i], dw=self.dw[i], workspace=self.ws)
+        if ev: ev[2].record()
+
+
+def run_ours(args, rank, world, local):
+    from paper_2503_20354_b200 import binding as B
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    B.lib()
+    device = torch.device("cuda", local if world > 1 else 0)
+    layers, desc_text = get_layers(args.workload, args.batch)
+    path = B.PATH_FP32 if args.path == "fp32" else B.PATH_TENSOR_CORE
+    stack = Stack(layers, path, args.seed + rank, device)
+    torch.cuda.synchronize()
+    peaks = load_peaks()
+
+    for _ in range(args.warmup):
+        stack.step()
+    torch.cuda.synchronize()
+    barrier(world)
+
+    sampler = ClockSampler(local if world > 1 else 0)
+    sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    launches0 = B.surgeon_launch_count()
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t_begin.record()
+    for s in range(args.steps):
+        stack.step(evs[s])
+    t_end.record()
+    torch.cuda.synchronize()
+    barrier(world)
+    launches = B.surgeon_launch_count() - launches0
+    clocks = sampler.stop()
+    total_ms = max_over_ranks(t_begin.elapsed_time(t_end), world, device)
+    prune_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
+    dw_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
+    ms_per_step = total_ms / args.steps
+
+    # device-side status of every store (one small read per layer, outside the timed region)
+    for s in stack.store:
+        h = s.read_header()
+        if h.status != 0:
+            raise SystemExit("device status %d in a compressed store" % h.status)
+
+    flops = sum(l.flops for l in layers)
+    pbytes = sum(prune_alg_bytes(l, s.sizes.n_keep) for l, s in zip(layers, stack.store))
+    stored = sum(s.stored_bytes for s in stack.store)
+    dense = sum(l.act_bytes for l in layers)
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    prune_gbs = pbytes / (prune_ms * 1e-3) / 1e9
+    dw_tflops = flops / (dw_ms * 1e-3) / 1e12
+    if path == B.PATH_TENSOR_CORE:
+        peak, bound, unit = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])), "tensor", "TFLOP/s"
+        peak_note = "%s bf16 cuBLAS, sustained" % peaks["_source"]
+    else:
+        peak, bound, unit = FP32_ALU_TFLOPS, "alu", "TFLOP/s"
+        peak_note = "derived: 148 SMs x 128 fp32 FMA lanes x 2 x 1.965 GHz"
+    roofline = {"kernel": "weight gradient (all layers of one step)", "bound": bound,
+                "achieved": round(dw_tflops, 3), "peak": round(peak, 1), "unit": unit,
+                "frac": round(dw_tflops / peak, 4), "traffic": None, "peak_source": peak_note}
+
+    # ---- end to end through the C ABI with host buffers --------------------------------------
+    e2e = run_e2e(stack, layers, args, world, device, flops)
+
+    out = {
+        "metric": METRIC, "value": round(value, 3), "unit": "TFLOP/s (dense-equivalent dW flops / whole-step time)",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if path == B.PATH_TENSOR_CORE else "f32", "data": "synthetic",
+        "config": {"workload": desc_text, "layers": len(layers), "ratios": "GI/LAM rule, GI~LogNormal(0,1)",
+                   "path": args.path, "l2": "inputs larger than L2 (%.2f GB read per step)" % ((dense + sum(g.numel() * 4 for g in stack.g)) / 1e9),
+                   "replicas": world},
+        "parts": {
+            "prune_compact": {"ms": round(prune_ms, 4), "GB/s": round(prune_gbs, 1),
+                              "frac_hbm": round(prune_gbs / float(peaks["hbm_gbs"]), 4),
+                              "peak_GB/s": peaks["hbm_gbs"], "peak_source": peaks["_source"] + " copy bandwidth",
+                              "algorithmic_bytes": pbytes},
+            "weight_grad": {"ms": round(dw_ms, 4), "TFLOP/s": round(dw_tflops, 3), "flops": flops},
+            "store_bytes": stored, "dense_bytes": dense, "mean_ratio": float(np.mean(stack.ratios)),
+        },
+        "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+    }
+    if rank == 0:
+        if args.cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline(args, budget_s=20.0)
+        print(json.dumps(out))
+
+
+def run_e2e(stack, layers, args, world, device, flops):
+    """Same step with HOST inputs: per step, pinned host activations and gradients are copied in,
+    the path runs, and every dW is copied back to pinned host memory."""
+    steps = max(1, min(args.steps, args.e2e_steps))
+    hx = [torch.empty(x.shape, dtype=x.dtype).pin_memory() for x in stack.x]
+    hg = [torch.empty(g.shape, dtype=g.dtype).pin_memory() for g in stack.g]
+    hdw = [torch.empty(d.shape, dtype=d.dtype).pin_memory() for d in stack.dw]
+    for h, d in zip(hx + hg, stack.x + stack.g):
+        h.copy_(d)
+    torch.cuda.synchronize()
+    h2d = sum(t.numel() * t.element_size() for t in hx + hg)
+    d2h = sum(t.numel() * t.element_size() for t in hdw)
+
+    def one():
+        for d, h in zip(stack.x + stack.g, hx + hg):
+            d.copy_(h, non_blocking=True)
+        stack.step()
+        for h, d in zip(hdw, stack.dw):
+            h.copy_(d, non_blocking=True)
+
+    one()
+    torch.cuda.synchronize()
+    barrier(world)
+    b, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    b.record()
+    for _ in range(steps):
+        one()
+    e.record()
+    torch.cuda.synchronize()
+    barrier(world)
+    ms = max_over_ranks(b.elapsed_time(e), world, device) / steps
+    return {"value": round(world * flops / (ms * 1e-3) / 1e12, 4), "unit": "TFLOP/s", "ms_per_step": round(ms, 3),
+            "steps": steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------
+
+def oracle_step(layers, inputs, ratios):
+    """The oracle's pass over `layers`: ratios, prune+compact, decompress, dW (fp64)."""
+    import oracle
+    for l, (a, g), p in zip(layers, inputs, ratios):
+        r = oracle.prune_compact(a.reshape(-1), float(p))
+        pruned = oracle.decompress(r["bitmap"], r["values"], a.size).reshape(l.act_shape)
+        if l.kind == 1:
+            oracle.dw_conv2d(pruned, g, l.kh, l.kw, l.stride, l.pad)
+        else:
+            oracle.dw_linear(pruned, g)
+
+
+def oracle_sample(args, budget_s: float, grow: bool = False):
+    """A bounded sample of the workload for the CPU: the same stack at batch 1, thinned to every
+    `stride`-th layer until one pass fits the budget; with `grow`, the batch is then raised (up to
+    16) so that one pass takes a sizeable part of the budget."""
+    import oracle
+    from paper_2503_20354_b200 import workloads as W
+    full, _ = get_layers(args.workload, args.batch)
+    batch = 1
+    small = W.shrink(full, batch)
+    gi = W.gradient_importance(len(small), args.seed)
+    lam = np.array([l.act_bytes for l in full], dtype=np.float64)
+    _, ratios = oracle.layer_ratios(gi, lam)
+    stride = 1
+    while True:
+        idx = list(range(0, len(small), stride))
+        layers = [small[i] for i in idx]
+        inputs = [(W.as_numpy_bits(W.activation(small[i], args.seed, i)), W.grad_out(small[i], args.seed, i).numpy())
+                  for i in idx]
+        t0 = time.perf_counter()
+        oracle_step(layers, inputs, ratios[idx])
+        dt = time.perf_counter() - t0
+        if grow and batch == 1 and dt < budget_s / 4:
+            batch = max(2, min(16, int(0.6 * budget_s / dt)))
+            small = W.shrink(full, batch)
+            continue
+        if dt <= budget_s or len(layers) == 1 or batch > 1:
+            break
+        stride *= 2
+    text = "%s at batch %d, %d of %d layers (every %d-th)" % (args.workload, batch, len(layers), len(small), stride)
+    return layers, inputs, ratios[idx], dt, text
+
+
+def cpu_baseline(args, budget_s: float):
+    import oracle
+    layers, inputs, ratios, dt, text = oracle_sample(args, budget_s, grow=True)
+    flops = sum(l.flops for l in layers)
+    return {"value": round(flops / dt / 1e12, 6), "unit": "TFLOP/s", "cores": oracle.num_threads(),
+            "kind": "oracle", "sample": text, "seconds": round(dt, 3)}
+
+
+def run_reference(args, rank, world):
+    """The CPU oracle as the reference arm (rank 0 only)."""
+    if rank != 0:
+        return
+    import oracle
+    total = max(1, args.steps + args.warmup)
+    layers, inputs, ratios, dt, text = oracle_sample(args, budget_s=max(0.5, 120.0 / total))
+    for _ in range(args.warmup):
+        oracle_step(layers, inputs, ratios)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(layers, inputs, ratios)
+    ms = (time.perf_counter() - t0) * 1e3 / max(1, args.steps)
+    flops = sum(l.flops for l in layers)
+    v = round(flops / (ms * 1e-3) / 1e12, 6)
+    _, desc_text = get_layers(args.workload, args.batch)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": "TFLOP/s (dense-equivalent dW flops / whole-step time)",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": desc_text, "sample": text},
+        "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": text},
+        "e2e": {"value": v, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="wrn28", choices=["wrn28", "tiny", "resnet50", "vit"])
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--path", default="tc", choices=["tc", "fp32"])
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        rank = int(os.environ.get("RANK", "0"))
+        run_reference(args, rank, int(os.environ.get("WORLD_SIZE", "1")))
+        return
+    rank, world, local = dist_setup(args.gpus)
+    try:
+        run_ours(args, rank, world, local)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -169,6 +169,11 @@ surgeon_status surgeon_decompress(const surgeon_compressed* act, void* x_out, vo
 /* Static text for a status code. */
 const char* surgeon_status_string(surgeon_status s);
 
+/* Diagnostic without a counterpart in the paper: how many kernels this library has launched in
+ * this process so far (all streams, all devices).  Benchmarks report the difference around a
+ * timed region. */
+uint64_t surgeon_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -79,6 +79,8 @@ def lib():
                                           C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]
         l.surgeon_decompress.restype = C.c_int
         l.surgeon_decompress.argtypes = [C.POINTER(Compressed), C.c_void_p, C.c_void_p]
+        l.surgeon_launch_count.restype = C.c_uint64
+        l.surgeon_launch_count.argtypes = []
         l.surgeon_status_string.restype = C.c_char_p
         l.surgeon_status_string.argtypes = [C.c_int]
         _lib = l
@@ -87,6 +89,11 @@ def lib():
 
 def status_string(status: int) -> str:
     return lib().surgeon_status_string(int(status)).decode()
+
+
+def surgeon_launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return int(lib().surgeon_launch_count())
 
 
 def _check(status: int, where: str, allow=()):

@@ -2,9 +2,15 @@
 // that touches tensor data is a kernel launched from the other translation units.
 #include <math.h>
 
+#include <atomic>
+
 #include "surgeon_internal.cuh"
 
 namespace surgeon {
+
+static std::atomic<unsigned long long> g_launches{0};
+void note_launches(int n) { g_launches.fetch_add(static_cast<unsigned long long>(n), std::memory_order_relaxed); }
+unsigned long long launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
 
 int sm_count() {
   static int cached[64] = {0};
@@ -172,6 +178,8 @@ surgeon_status surgeon_decompress(const surgeon_compressed* act, void* x_out, vo
   const cudaError_t e = launch_decompress(*act, x_out, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SURGEON_OK : SURGEON_ERR_CUDA;
 }
+
+uint64_t surgeon_launch_count(void) { return launches_so_far(); }
 
 const char* surgeon_status_string(surgeon_status s) {
   switch (s) {

@@ -321,6 +321,7 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
 
   if (k == 0) {
     header_empty_kernel<<<1, 1, 0, stream>>>(out.header, Elem<DT>::kSentinel);
+    note_launches(1);
   } else {
     constexpr int VEC = 16 / static_cast<int>(sizeof(typename Elem<DT>::type));
     const long long nvec = n / VEC;
@@ -333,16 +334,19 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
           x, n, k, 1, st, ghist + kMaxBins, out.header);
       radix_hist_kernel<0, 0, 9, true><<<grid, kHistThreads, 0, stream>>>(
           x, n, k, 2, st, ghist + 2 * kMaxBins, out.header);
+      note_launches(3);
     } else {
       radix_hist_kernel<1, 4, 11, false><<<grid, kHistThreads, 0, stream>>>(
           x, n, k, 0, st, ghist, out.header);
       radix_hist_kernel<1, 0, 4, true><<<grid, kHistThreads, 0, stream>>>(
           x, n, k, 1, st, ghist + kMaxBins, out.header);
+      note_launches(2);
     }
   }
   if (n == 0) {
     offsets_empty_kernel<<<1, 1, 0, stream>>>(
         reinterpret_cast<unsigned long long*>(out.block_offsets));
+    note_launches(1);
   } else {
     const long long tiles = (n + kTileElems - 1) / kTileElems;
     const long long cap = 8LL * sm_count();
@@ -351,6 +355,7 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
         x, n, out.header, out.bitmap, out.values,
         reinterpret_cast<unsigned long long*>(out.block_offsets), &st->compact_ticket, tile_state,
         static_cast<int>(tiles));
+    note_launches(1);
   }
   return cudaGetLastError();
 }
@@ -375,6 +380,7 @@ cudaError_t launch_decompress(const surgeon_compressed& act, void* x_out, cudaSt
     decompress_kernel<0><<<grid, 256, 0, stream>>>(act.bitmap, act.values, offs, act.n, x_out);
   else
     decompress_kernel<1><<<grid, 256, 0, stream>>>(act.bitmap, act.values, offs, act.n, x_out);
+  note_launches(1);
   return cudaGetLastError();
 }
 

@@ -65,6 +65,8 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
 
 // Number of SMs of the current device (cached per device id).
 int sm_count();
+// Adds to the process-wide kernel-launch counter behind surgeon_launch_count().
+void note_launches(int n);
 
 __device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31; }
 __device__ __forceinline__ uint32_t lanemask_lt() {

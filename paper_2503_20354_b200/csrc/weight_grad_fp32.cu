@@ -180,10 +180,12 @@ cudaError_t launch_weight_grad_fp32(const surgeon_compressed& act, const surgeon
       dw_fp32_kernel<0><<<grid, 256, 0, stream>>>(act.bitmap, act.values, offs, grad_out, partial, g);
     else
       dw_fp32_kernel<1><<<grid, 256, 0, stream>>>(act.bitmap, act.values, offs, grad_out, partial, g);
+    note_launches(1);
   }
   const long long mn = g.M * g.N;
   reduce_chunks_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
       partial, mn, static_cast<int>(chunks), dw, accumulate);
+  note_launches(1);
   return cudaGetLastError();
 }
 
