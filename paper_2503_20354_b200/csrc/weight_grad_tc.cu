@@ -1,11 +1,590 @@
-// Tensor-core path of surgeon_weight_grad (tcgen05 / TMEM).  Not built yet: the entry point
-// reports SURGEON_ERR_UNSUPPORTED for path 0 until the kernel lands.
+// Tensor-core path of surgeon_weight_grad (Algorithm 1 lines 11-12, Eq. 2) for sm_100a.
+//
+// Implicit GEMM on tcgen05:  D[nn, o] = sum_k Acol[nn, k] * G[o, k]
+//   nn = (c, r, s)  im2col column of the activation  -> MMA M (128 rows per CTA tile, TMEM lanes)
+//   o  = output channel                              -> MMA N (tile of <= 256, TMEM columns)
+//   k  = (b, y, x) output position / row t           -> MMA K, 64 per pipeline stage
+// Both operands are bf16, K-major, in the 128-byte-swizzled shared-memory layout that the UMMA
+// descriptors name; accumulation is fp32 in tensor memory.
+//
+// Nothing dense comes from HBM: producer warps read the bitmap, the block offsets and the packed
+// values, rebuild the rows of the pruned activation a K-tile needs in a shared-memory patch
+// (Algorithm 1 line 11, "Reshape"), and write the im2col view of that patch into the operand
+// tile.  The same warps convert the fp32 output gradient to bf16 on the way into its tile.  One
+// elected thread issues the MMAs; tcgen05.commit hands stages back to the producers.
+// The reduction is split over CTAs in contiguous K ranges; partial tiles go to scratch and are
+// summed in a fixed order, so results are bitwise reproducible.
+//
+// Every wait on an mbarrier is bounded; when one gives up the CTA records SURGEON_ERR_TIMEOUT in
+// the scratch status word, frees its tensor memory and returns.
 #include "surgeon_internal.cuh"
 
 namespace surgeon {
-size_t weight_grad_tc_workspace(const surgeon_layer_desc&) { return 0; }
-cudaError_t launch_weight_grad_tc(const surgeon_compressed&, const surgeon_layer_desc&,
-                                  const float*, float*, int, void*, cudaStream_t) {
-  return cudaErrorNotSupported;
+
+namespace {
+
+constexpr int kTileM = 128;          // im2col columns (nn) per CTA tile = TMEM lanes
+constexpr int kTileK = 64;           // bf16 elements per stage row = one 128-byte swizzle row
+constexpr int kProducerWarps = 8;
+constexpr int kProducerThreads = kProducerWarps * 32;
+constexpr int kThreads = 32 + kProducerThreads;  // warp 0 issues MMAs
+constexpr int kPatchBytes = 32 * 1024;
+constexpr int kPatchElems = kPatchBytes / 2;
+constexpr int kMaxStages = 4;
+constexpr uint32_t kWaitCap = 1u << 22;
+constexpr size_t kStatusBytes = 256;  // scratch header in front of the partial tiles
+
+struct TcParams {
+  // layer
+  int kind, B, C, H, W, O, KH, KW, stride, pad, OH, OW;
+  int P;            // output positions per image (conv) or rows T (linear)
+  int n_gemm;       // C*KH*KW
+  int RS;           // KH*KW
+  // tiling
+  int tile_n;       // output channels per CTA tile (multiple of 16, <= 256)
+  int m_tiles, n_tiles, splits;
+  int tiles_per_img, total_ktiles, ktiles_per_split;
+  int stages, tmem_cols;
+  int group_ch;     // channels (conv) decompressed per patch pass
+  int max_rows;     // input rows one K-tile can touch (conv)
+  int dt;           // activation dtype
+  int g_vec_ok;     // gradient rows can be read with 16-byte loads
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; false when it gave up.  `sleep_ns` > 0 backs off between polls (long waits).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t sleep_ns = 0) {
+  for (uint32_t i = 0; i < kWaitCap; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (sleep_ns) __nanosleep(sleep_ns);
+  }
+  return false;
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst),
+               "r"(cols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
+               : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the mbarrier once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void producer_sync() {
+  asm volatile("bar.sync 1, %0;" ::"n"(kProducerThreads) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups
+// of 8 rows 1024 bytes apart (tile base 1024-byte aligned).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);  // start address, 16-byte units
+  d |= static_cast<uint64_t>(1) << 16;                  // leading byte offset (unused with swizzle)
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;          // stride byte offset between 8-row groups
+  d |= static_cast<uint64_t>(1) << 46;                  // descriptor version of this architecture
+  d |= static_cast<uint64_t>(2) << 61;                  // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
+__host__ __device__ inline uint32_t make_idesc(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+// Byte offset of 16-byte chunk `chunk` (0..7) of row `row` inside a swizzled K-major tile.
+__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
+  return static_cast<uint32_t>(row) * 128u + (static_cast<uint32_t>(chunk ^ (row & 7)) << 4);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ unsigned short to_bf16_bits(float v) {
+  return static_cast<unsigned short>(pack_bf16x2(v, 0.0f) & 0xFFFFu);
+}
+
+// ---- decompression of one contiguous flat range into shared memory (one warp) ---------------
+// dst[i] = bf16 of the pruned activation at flat index start + i, i < len  (Algorithm 1 line 11).
+template <int DT>
+__device__ __forceinline__ void decompress_range(const uint32_t* __restrict__ bitmap,
+                                                 const void* __restrict__ values,
+                                                 const unsigned long long* __restrict__ offsets,
+                                                 long long start, int len,
+                                                 unsigned short* __restrict__ dst) {
+  const uint32_t lane = lane_id();
+  const uint32_t lt = lanemask_lt();
+  const long long first_word = start >> 5;
+  const long long last_word = (start + len - 1) >> 5;
+  const long long blk = start >> 10;
+  const long long blk_word0 = blk << 5;
+  uint32_t w = 0;
+  if (blk_word0 + lane < first_word) w = __ldg(bitmap + blk_word0 + lane);
+  long long rank = static_cast<long long>(__ldg(offsets + blk)) + warp_sum(__popc(w));
+  for (long long wi = first_word; wi <= last_word; ++wi) {
+    const uint32_t word = __ldg(bitmap + wi);
+    const long long j = (wi << 5) + lane;
+    const bool in_range = (j >= start) && (j < start + len);
+    unsigned short v = 0;
+    if (in_range && ((word >> lane) & 1u)) {
+      const long long r = rank + __popc(word & lt);
+      if (DT == 0) v = to_bf16_bits(__ldg(reinterpret_cast<const float*>(values) + r));
+      else v = __ldg(reinterpret_cast<const unsigned short*>(values) + r);
+    }
+    if (in_range) dst[j - start] = v;
+    rank += __popc(word);
+  }
+}
+
+struct RowInfo {   // one im2col row (nn) of the CTA's M tile
+  short c;         // input channel, -1 when nn is past the end
+  signed char r, s;
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 1)
+dw_tc_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ values,
+             const unsigned long long* __restrict__ offsets, const float* __restrict__ grad,
+             float* __restrict__ partial, uint32_t* __restrict__ status, TcParams p) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  // carve: [stages][A 16 KB | B tile_n*128] | patch | barriers | row table
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  const int b_bytes = p.tile_n * 128;
+  const int stage_bytes = kTileM * 128 + b_bytes;
+  unsigned short* patch = reinterpret_cast<unsigned short*>(smem + p.stages * stage_bytes);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(
+      smem + p.stages * stage_bytes + kPatchBytes);
+  RowInfo* rows = reinterpret_cast<RowInfo*>(bars + 2 * kMaxStages + 2);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(rows + kTileM);
+  volatile uint32_t* fail = tmem_slot + 1;
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  const uint32_t lane = lane_id();
+  const int m_tile = blockIdx.x, n_tile = blockIdx.y, split = blockIdx.z;
+  const int nn0 = m_tile * kTileM;
+  const int o0 = n_tile * p.tile_n;
+  const int kt_begin = split * p.ktiles_per_split;
+  const int kt_end = min(kt_begin + p.ktiles_per_split, p.total_ktiles);
+  const int n_kt = kt_end - kt_begin;
+
+  const uint32_t full_bar = smem_u32(bars);
+  const uint32_t empty_bar = smem_u32(bars + kMaxStages);
+  const uint32_t acc_bar = smem_u32(bars + 2 * kMaxStages);
+
+  if (tid == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(full_bar + 8 * s, kProducerWarps);
+      mbar_init(empty_bar + 8 * s, 1);
+    }
+    mbar_init(acc_bar, 1);
+    *fail = 0;
+    fence_barrier_init();
+  }
+  for (int i = tid; i < kTileM; i += kThreads) {
+    const int nn = nn0 + i;
+    RowInfo ri;
+    if (nn < p.n_gemm) {
+      const int c = nn / p.RS;
+      const int rs = nn - c * p.RS;
+      ri.c = static_cast<short>(c);
+      ri.r = static_cast<signed char>(rs / p.KW);
+      ri.s = static_cast<signed char>(rs - (rs / p.KW) * p.KW);
+    } else {
+      ri.c = -1; ri.r = 0; ri.s = 0;
+    }
+    rows[i] = ri;
+  }
+  if (warp == 0) tmem_alloc(smem_u32(tmem_slot), p.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ================= MMA issuer =================
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(kTileM, p.tile_n);
+      bool ok = true;
+      for (int it = 0; it < n_kt && ok; ++it) {
+        const int s = it % p.stages;
+        const uint32_t parity = (it / p.stages) & 1;
+        ok = mbar_wait(full_bar + 8 * s, parity);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
+        const uint32_t b_addr = a_addr + kTileM * 128;
+#pragma unroll
+        for (int kk = 0; kk < kTileK / 16; ++kk) {
+          umma_bf16(tmem_base, make_desc(a_addr + kk * 32), make_desc(b_addr + kk * 32), idesc,
+                    (it > 0 || kk > 0) ? 1u : 0u);
+        }
+        umma_commit(empty_bar + 8 * s);   // stage is free once these MMAs have read it
+      }
+      if (!ok) { *fail = 1; atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); }
+      umma_commit(acc_bar);               // accumulator complete (or abandoned)
+    }
+    __syncwarp();
+  } else {
+    // ================= producers =================
+    const int ptid = tid - 32;
+    const int pwarp = warp - 1;
+    const int first_c = rows[0].c;       // M tiles never start past the end
+    int last_c = first_c;
+    for (int i = kTileM - 1; i >= 0; --i) {
+      if (rows[i].c >= 0) { last_c = rows[i].c; break; }
+    }
+    bool ok = true;
+    for (int it = 0; it < n_kt; ++it) {
+      const int s = it % p.stages;
+      if (it >= p.stages) {
+        const uint32_t parity = ((it / p.stages) - 1) & 1;
+        if (!mbar_wait(empty_bar + 8 * s, parity)) {
+          *fail = 1;
+          atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+        }
+      }
+      producer_sync();            // after it, every producer reads the same value of *fail
+      if (*fail) { ok = false; break; }
+      unsigned char* a_tile = smem + s * stage_bytes;
+      unsigned char* b_tile = a_tile + kTileM * 128;
+      const int kt = kt_begin + it;
+      const int img = kt / p.tiles_per_img;
+      const int p0 = (kt - img * p.tiles_per_img) * kTileK;
+
+      // ---- gradient tile: fp32 -> bf16, rows = output channels, K contiguous ----
+      if (p.kind == 1) {
+        const int tasks = p.tile_n * 8;
+        for (int t = ptid; t < tasks; t += kProducerThreads) {
+          const int row = t >> 3, chunk = t & 7;
+          const int o = o0 + row;
+          const int pp = p0 + chunk * 8;
+          uint4 out = make_uint4(0, 0, 0, 0);
+          if (o < p.O && pp < p.P) {
+            const float* src = grad + (static_cast<long long>(img) * p.O + o) * p.P + pp;
+            if (p.g_vec_ok && pp + 8 <= p.P) {
+              const float4 a = __ldg(reinterpret_cast<const float4*>(src));
+              const float4 b = __ldg(reinterpret_cast<const float4*>(src) + 1);
+              out.x = pack_bf16x2(a.x, a.y); out.y = pack_bf16x2(a.z, a.w);
+              out.z = pack_bf16x2(b.x, b.y); out.w = pack_bf16x2(b.z, b.w);
+            } else {
+              float v[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) v[e] = (pp + e < p.P) ? __ldg(src + e) : 0.0f;
+              out.x = pack_bf16x2(v[0], v[1]); out.y = pack_bf16x2(v[2], v[3]);
+              out.z = pack_bf16x2(v[4], v[5]); out.w = pack_bf16x2(v[6], v[7]);
+            }
+          }
+          *reinterpret_cast<uint4*>(b_tile + tile_off(row, chunk)) = out;
+        }
+      } else {
+        // linear: grad is [T, O]; lanes take consecutive output channels
+        const int tasks = p.tile_n * 8;
+        for (int t = ptid; t < tasks; t += kProducerThreads) {
+          const int chunk = t / p.tile_n, row = t - chunk * p.tile_n;
+          const int o = o0 + row;
+          const int pp = p0 + chunk * 8;
+          float v[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            v[e] = (o < p.O && pp + e < p.P)
+                       ? __ldg(grad + static_cast<long long>(pp + e) * p.O + o) : 0.0f;
+          uint4 out;
+          out.x = pack_bf16x2(v[0], v[1]); out.y = pack_bf16x2(v[2], v[3]);
+          out.z = pack_bf16x2(v[4], v[5]); out.w = pack_bf16x2(v[6], v[7]);
+          *reinterpret_cast<uint4*>(b_tile + tile_off(row, chunk)) = out;
+        }
+      }
+
+      // ---- activation tile: decompress a patch, then write its im2col view ----
+      if (p.kind == 1) {
+        const int k_valid = min(kTileK, p.P - p0);
+        const int y_first = p0 / p.OW;
+        const int y_last = (p0 + k_valid - 1) / p.OW;
+        int iy_lo = y_first * p.stride - p.pad;
+        int iy_hi = y_last * p.stride + p.KH - 1 - p.pad;
+        if (iy_lo < 0) iy_lo = 0;
+        if (iy_hi > p.H - 1) iy_hi = p.H - 1;
+        const int range_len = (iy_hi - iy_lo + 1) * p.W;
+        for (int cg = first_c; cg <= last_c; cg += p.group_ch) {
+          const int cg_end = min(cg + p.group_ch, last_c + 1);
+          for (int c = cg + pwarp; c < cg_end; c += kProducerWarps) {
+            const long long start =
+                ((static_cast<long long>(img) * p.C + c) * p.H + iy_lo) * p.W;
+            decompress_range<DT>(bitmap, values, offsets, start, range_len,
+                                 patch + (c - cg) * range_len);
+          }
+          producer_sync();
+          // rows of this channel group: nn in [cg*RS, cg_end*RS)
+          int row_lo = cg * p.RS - nn0;
+          int row_hi = cg_end * p.RS - nn0;
+          if (row_lo < 0) row_lo = 0;
+          if (row_hi > kTileM || cg_end > last_c) row_hi = kTileM;   // last group also zeroes pad rows
+          const int tasks = (row_hi - row_lo) * 8;
+          for (int t = ptid; t < tasks; t += kProducerThreads) {
+            const int row = row_lo + (t >> 3), chunk = t & 7;
+            const RowInfo ri = rows[row];
+            uint32_t h[8];
+            if (ri.c < 0) {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) h[e] = 0;
+            } else {
+              const unsigned short* src = patch + (ri.c - cg) * range_len;
+              int pp = p0 + chunk * 8;
+              int y = pp / p.OW;
+              int x = pp - y * p.OW;
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const int iy = y * p.stride + ri.r - p.pad;
+                const int ix = x * p.stride + ri.s - p.pad;
+                uint32_t v = 0;
+                if (pp < p.P && iy >= iy_lo && iy <= iy_hi && ix >= 0 && ix < p.W)
+                  v = src[(iy - iy_lo) * p.W + ix];
+                h[e] = v;
+                ++pp; ++x;
+                if (x == p.OW) { x = 0; ++y; }
+              }
+            }
+            uint4 out;
+            out.x = h[0] | (h[1] << 16); out.y = h[2] | (h[3] << 16);
+            out.z = h[4] | (h[5] << 16); out.w = h[6] | (h[7] << 16);
+            *reinterpret_cast<uint4*>(a_tile + tile_off(row, chunk)) = out;
+          }
+          producer_sync();   // the patch is overwritten by the next group / stage
+        }
+      } else {
+        // linear: activation [T, C]; patch[k][i] = A[p0 + k, nn0 + i]
+        const int k_valid = min(kTileK, p.P - p0);
+        const int c_valid = min(kTileM, p.n_gemm - nn0);
+        for (int k = pwarp; k < k_valid; k += kProducerWarps) {
+          decompress_range<DT>(bitmap, values, offsets,
+                               static_cast<long long>(p0 + k) * p.C + nn0, c_valid,
+                               patch + k * kTileM);
+        }
+        producer_sync();
+        for (int t = ptid; t < kTileM * 8; t += kProducerThreads) {
+          const int chunk = t >> 7, row = t & (kTileM - 1);
+          uint32_t h[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const int k = chunk * 8 + e;
+            h[e] = (row < c_valid && k < k_valid) ? patch[k * kTileM + row] : 0u;
+          }
+          uint4 out;
+          out.x = h[0] | (h[1] << 16); out.y = h[2] | (h[3] << 16);
+          out.z = h[4] | (h[5] << 16); out.w = h[6] | (h[7] << 16);
+          *reinterpret_cast<uint4*>(a_tile + tile_off(row, chunk)) = out;
+        }
+        producer_sync();
+      }
+      fence_proxy_async();   // generic-proxy writes -> visible to the tensor core's reads
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full_bar + 8 * s);
+    }
+    (void)ok;
+  }
+
+  // ================= epilogue: TMEM -> scratch partial tile =================
+  if (warp >= 1 && warp <= 4) {
+    const bool done = mbar_wait(acc_bar, 0, 256);
+    tc_fence_after();
+    if (done && !*fail) {
+      const int lane_grp = warp & 3;              // TMEM lanes this warp may read
+      const int row = lane_grp * 32 + static_cast<int>(lane);
+      const int nn = nn0 + row;
+      float* out = partial + static_cast<long long>(split) * p.O * p.n_gemm;
+      for (int col = 0; col < p.tile_n; col += 16) {
+        uint32_t r[16];
+        tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_grp * 32) << 16) + col, r);
+        if (nn < p.n_gemm) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int o = o0 + col + e;
+            if (o < p.O) out[static_cast<long long>(o) * p.n_gemm + nn] = __uint_as_float(r[e]);
+          }
+        }
+      }
+    } else if (!done && lane == 0) {
+      atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+}
+
+// Sums the split partials in order and writes (or adds to) dw; copies the device status into
+// the activation's header when a wait timed out.
+__global__ void __launch_bounds__(256)
+reduce_splits_kernel(const float* __restrict__ partial, long long mn, int splits,
+                     float* __restrict__ dw, int accumulate, const uint32_t* __restrict__ status,
+                     surgeon_header* __restrict__ hdr) {
+  const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i == 0 && *status != 0 && hdr) atomicMax(&hdr->status, *status);
+  if (i >= mn) return;
+  float s = partial[i];
+  for (int z = 1; z < splits; ++z) s += partial[z * mn + i];
+  dw[i] = accumulate ? dw[i] + s : s;
+}
+
+bool plan(const surgeon_layer_desc& d, int dt, TcParams* out) {
+  TcParams p{};
+  p.kind = d.kind; p.B = d.batch; p.C = d.c_in; p.H = d.h; p.W = d.w; p.O = d.c_out;
+  p.KH = d.kh; p.KW = d.kw; p.stride = d.stride; p.pad = d.pad;
+  p.OH = (d.h + 2 * d.pad - d.kh) / d.stride + 1;
+  p.OW = (d.w + 2 * d.pad - d.kw) / d.stride + 1;
+  p.RS = d.kh * d.kw;
+  p.n_gemm = d.c_in * p.RS;
+  p.dt = dt;
+  int imgs;
+  if (d.kind == 1) { p.P = p.OH * p.OW; imgs = d.batch; }
+  else { p.P = d.batch; imgs = 1; }
+  if (d.kh > 127 || d.kw > 127 || d.c_in > 32767) return false;
+  const int nt = (p.O + 255) / 256;
+  p.n_tiles = nt;
+  p.tile_n = ((p.O + nt - 1) / nt + 15) / 16 * 16;
+  p.m_tiles = (p.n_gemm + kTileM - 1) / kTileM;
+  p.tiles_per_img = (p.P + kTileK - 1) / kTileK;
+  const long long total = static_cast<long long>(imgs) * p.tiles_per_img;
+  if (total > 2147483647LL) return false;
+  p.total_ktiles = static_cast<int>(total);
+  const int sms = sm_count();
+  const long long tiles_mn = static_cast<long long>(p.m_tiles) * p.n_tiles;
+  int splits = static_cast<int>(tiles_mn >= sms ? 1 : sms / tiles_mn);
+  const int max_by_work = (p.total_ktiles + 3) / 4;   // at least 4 K-tiles per split
+  if (splits > max_by_work) splits = max_by_work;
+  if (splits < 1) splits = 1;
+  if (splits > 65535) splits = 65535;
+  p.ktiles_per_split = (p.total_ktiles + splits - 1) / splits;
+  p.splits = (p.total_ktiles + p.ktiles_per_split - 1) / p.ktiles_per_split;
+  // patch: rows one K-tile can touch
+  if (d.kind == 1) {
+    const int out_rows = (kTileK + p.OW - 2) / p.OW + 1;           // rows spanned by 64 positions
+    int in_rows = (out_rows - 1) * p.stride + p.KH;
+    if (in_rows > p.H) in_rows = p.H;
+    p.max_rows = in_rows;
+    const long long per_ch = static_cast<long long>(in_rows) * p.W;
+    if (per_ch > kPatchElems) return false;
+    p.group_ch = static_cast<int>(kPatchElems / per_ch);
+  } else {
+    p.max_rows = 1;
+    p.group_ch = 1;
+  }
+  p.g_vec_ok = (d.kind == 1 && (p.P % 4) == 0) ? 1 : 0;
+  p.tmem_cols = 32;
+  while (p.tmem_cols < p.tile_n) p.tmem_cols *= 2;
+  const int stage_bytes = kTileM * 128 + p.tile_n * 128;
+  const int fixed = kPatchBytes + 1024 /*align*/ + 1024 /*barriers, row table*/;
+  int stages = (227 * 1024 - fixed) / stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) return false;
+  p.stages = stages;
+  *out = p;
+  return true;
+}
+
+size_t smem_bytes(const TcParams& p) {
+  return static_cast<size_t>(p.stages) * (kTileM * 128 + p.tile_n * 128) + kPatchBytes + 2048;
+}
+
+}  // namespace
+
+size_t weight_grad_tc_workspace(const surgeon_layer_desc& d) {
+  TcParams p;
+  if (!plan(d, 0, &p)) return 0;
+  return kStatusBytes + static_cast<size_t>(p.splits) * p.O * p.n_gemm * sizeof(float);
+}
+
+cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_layer_desc& d,
+                                  const float* grad_out, float* dw, int accumulate,
+                                  void* workspace, cudaStream_t stream) {
+  TcParams p;
+  if (!plan(d, act.dt, &p)) return cudaErrorNotSupported;
+  uint32_t* status = static_cast<uint32_t*>(workspace);
+  float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes);
+  cudaError_t e = cudaMemsetAsync(status, 0, kStatusBytes, stream);
+  if (e != cudaSuccess) return e;
+  const size_t smem = smem_bytes(p);
+  const unsigned long long* offs = reinterpret_cast<const unsigned long long*>(act.block_offsets);
+  dim3 grid(p.m_tiles, p.n_tiles, p.splits);
+  if (act.dt == 0) {
+    e = cudaFuncSetAttribute(dw_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    dw_tc_kernel<0><<<grid, kThreads, smem, stream>>>(act.bitmap, act.values, offs, grad_out,
+                                                      partial, status, p);
+  } else {
+    e = cudaFuncSetAttribute(dw_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    dw_tc_kernel<1><<<grid, kThreads, smem, stream>>>(act.bitmap, act.values, offs, grad_out,
+                                                      partial, status, p);
+  }
+  const long long mn = static_cast<long long>(p.O) * p.n_gemm;
+  reduce_splits_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
+      partial, mn, p.splits, dw, accumulate, status, act.header);
+  note_launches(2);
+  return cudaGetLastError();
+}
+
 }  // namespace surgeon
