@@ -249,7 +249,7 @@ def run_ours(args, rank, world, local):
                 "frac": round(dw_tflops / peak, 4), "traffic": None, "peak_source": peak_note}
 
     # ---- end to end through the C ABI with host buffers --------------------------------------
-    e2e = run_e2e(stack, layers, args, world, device, flops)
+    e2e = run_e2e(stack, layers, args, world, device, flops) if args.e2e else None
 
     out = {
         "metric": METRIC, "value": round(value, 3), "unit": "TFLOP/s (dense-equivalent dW flops / whole-step time)",
@@ -405,6 +405,7 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--no-e2e", dest="e2e", action="store_false", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

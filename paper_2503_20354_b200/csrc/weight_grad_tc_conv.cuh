@@ -1,0 +1,27 @@
+// Plan and launcher of the fast stride-1 convolution kernel (weight_grad_tc_conv.cu).
+#pragma once
+
+#include "surgeon_internal.cuh"
+
+namespace surgeon {
+
+struct FastParams {
+  int mode;                 // 0 = 3x3 pad 1 through a shared-memory patch, 1 = 1x1 direct
+  int B, C, H, W, O;
+  int P;                    // output positions per image (= H*W)
+  int n_gemm;               // C*KH*KW
+  int acc_n, n_acc;         // columns per accumulator, accumulators per CTA (1 or 2)
+  int n_tiles, m_tiles;
+  int tiles_per_img, total_ktiles, ktiles_per_split, splits;
+  int tmem_cols, stages, smem_bytes;
+};
+
+// False when the layer is not one the fast kernel handles.
+bool plan_conv_fast(const surgeon_layer_desc& d, FastParams* out);
+
+// Enqueues the kernel; partial = [splits][O][n_gemm] fp32, status = one zeroed word.
+cudaError_t launch_conv_fast(const surgeon_compressed& act, const FastParams& p,
+                             const float* grad_out, float* partial, uint32_t* status,
+                             cudaStream_t stream);
+
+}  // namespace surgeon

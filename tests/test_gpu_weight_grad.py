@@ -54,6 +54,17 @@ SHAPES = [
     W.conv("stem7x7", 2, 3, 64, 64, 7, 2, 3, dist="normal"),
     W.conv("c3x3_7x7map", 5, 32, 7, 48, 3, 1),
     W.conv("c3x3_nopad", 2, 8, 10, 8, 3, 1, 0),
+    # stride-1 3x3 / 1x1 convs with rows a multiple of 8 wide (the two-group fast kernel)
+    W.conv("f3x3_w16_partial_ch", 3, 20, 16, 24, 3),
+    W.conv("f3x3_w8_two_acc", 4, 32, 8, 320, 3),
+    W.conv("f3x3_w56", 2, 8, 56, 16, 3),
+    W.conv("f3x3_w32_cout640", 2, 16, 32, 640, 3),
+    W.conv("f3x3_w32_cout272_padded", 2, 16, 32, 272, 3),
+    W.Layer("f3x3_h12w8_tail_ktile", 1, 3, 8, 12, 8, 32, 3, 3, 1, 1),
+    W.Layer("f3x3_h5w16_tail_ktile", 1, 2, 8, 5, 16, 16, 3, 3, 1, 1),
+    W.conv("f1x1_w8", 5, 200, 8, 48, 1, 1, 0),
+    W.conv("f1x1_w56", 2, 64, 56, 256, 1, 1, 0),
+    W.Layer("f1x1_h12w8_tail_ktile", 1, 3, 40, 12, 8, 32, 1, 1, 1, 0),
     W.linear("fc", 64, 2048, 1000, dist="abs_normal", dt=W.F32),
     W.linear("tokens", 2 * 197, 768, 256, dist="normal", dt=W.F32),
     W.linear("tiny", 5, 7, 3, dist="normal", dt=W.F32),
