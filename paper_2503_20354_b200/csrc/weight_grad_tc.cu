@@ -444,10 +444,15 @@ size_t smem_bytes(const TcParams& p) {
 
 }  // namespace
 
+static size_t fast_partial_bytes(const FastParams& f) {
+  const size_t b = static_cast<size_t>(f.splits) * f.O * f.n_gemm * sizeof(float);
+  return (b + 255) & ~static_cast<size_t>(255);
+}
+
 size_t weight_grad_tc_workspace(const surgeon_layer_desc& d) {
   FastParams f;
   if (plan_conv_fast(d, &f))
-    return kStatusBytes + static_cast<size_t>(f.splits) * f.O * f.n_gemm * sizeof(float);
+    return kStatusBytes + fast_partial_bytes(f) + conv_fast_grad_bf16_bytes(f);
   TcParams p;
   if (!plan(d, 0, &p)) return 0;
   return kStatusBytes + static_cast<size_t>(p.splits) * p.O * p.n_gemm * sizeof(float);
@@ -462,12 +467,13 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
   if (e != cudaSuccess) return e;
   FastParams f;
   if (plan_conv_fast(d, &f)) {
-    e = launch_conv_fast(act, f, grad_out, partial, status, stream);
+    void* grad_bf16 = reinterpret_cast<char*>(partial) + fast_partial_bytes(f);
+    e = launch_conv_fast(act, f, grad_out, grad_bf16, partial, status, stream);
     if (e != cudaSuccess) return e;
     const long long fmn = static_cast<long long>(f.O) * f.n_gemm;
     reduce_splits_kernel<<<static_cast<unsigned>((fmn + 255) / 256), 256, 0, stream>>>(
         partial, fmn, f.splits, dw, accumulate, status, act.header);
-    note_launches(2);
+    note_launches(1);
     return cudaGetLastError();
   }
   TcParams p;

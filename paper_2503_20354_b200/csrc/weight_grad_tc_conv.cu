@@ -1,18 +1,22 @@
-// Fast tensor-core weight-gradient kernel for stride-1 convolutions whose rows are a multiple of
-// 8 elements wide: 3x3 / pad 1 ("patch" mode) and 1x1 / pad 0 ("direct" mode).
-// Algorithm 1 lines 11-12 with Eq. 2; same GEMM view as weight_grad_tc.cu:
-//   D[nn, o] = sum_k Acol[nn, k] * G[o, k],  nn = (c, r, s),  k = (b, y, x).
+// Fast tensor-core weight-gradient kernel for 3x3 / pad 1 ("patch" mode) and 1x1 / pad 0
+// ("direct" mode) convolutions of stride 1 or 2 whose rows are a multiple of 8 (stride 1) or
+// 16 (stride 2) elements wide.  Algorithm 1 lines 11-12 with Eq. 2; same GEMM view as
+// weight_grad_tc.cu:  D[nn, o] = sum_k Acol[nn, k] * G[o, k],  nn = (c, r, s),  k = (b, y, x).
 //
 // What differs from the general kernel:
-//   * two producer groups of 8 warps fill alternate pipeline stages, so the global-load latency
-//     of one group hides behind the other group's arithmetic and the MMAs;
-//   * per K-tile, the bitmap words of every channel range and the rank of each word's first
-//     bit are staged in shared memory one tile ahead; decompression then works on units of
-//     8 elements (one bitmap byte) with eight independent loads of packed values per thread;
-//   * patch mode copies the im2col view with one 16-byte load per (channel, filter row, chunk)
-//     and funnel shifts for the s = 0 / s = 2 columns; direct mode (1x1) decompresses straight
-//     into the swizzled operand tile;
+//   * the output gradient is converted to bf16 once by a streaming pre-pass into scratch and
+//     then arrives in the swizzled operand tile by TMA, several stages ahead of the MMAs;
+//   * two producer groups of 8 warps rebuild activation tiles for alternate pipeline stages,
+//     so the load latency of one group hides behind the other group's arithmetic;
+//   * per K-tile, the bitmap bits a group needs and the rank of their first kept element are
+//     staged in shared memory one tile ahead; decompression then works on units of 8 output
+//     elements with eight independent loads of packed values per thread;
+//   * patch mode copies the im2col view with 16-byte loads and funnel shifts for the s = 0 / 2
+//     columns (stride 2 keeps even and odd input columns in separate planes of the patch);
+//     direct mode decompresses straight into the swizzled operand tile;
 //   * one or two accumulators (<= 512 TMEM columns) share each activation tile.
+#include <cuda.h>
+
 #include "surgeon_internal.cuh"
 #include "tc_common.cuh"
 #include "weight_grad_tc_conv.cuh"
@@ -30,35 +34,28 @@ constexpr int kGroupWarps = 8;
 constexpr int kGroupThreads = kGroupWarps * 32;
 constexpr int kThreads = 32 + kGroups * kGroupThreads;
 constexpr int kPatchBytes = 16 * 1024;       // per group
-constexpr int kMetaWords = 512;              // bitmap words staged per group and K-tile
+constexpr int kMetaWords = 1024;             // staged bitmap words / chunk bits per group
 constexpr int kMaxStages = 4;
-constexpr int kGBatch = 4;                   // gradient chunks a thread keeps in flight
 
 __device__ __forceinline__ void group_sync(int g) {
   asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "n"(kGroupThreads) : "memory");
 }
 
-// Unit = 8 consecutive elements (one bitmap byte).  words/wrank: staged bitmap words of the
-// range and the rank of each word's first bit; rel = bit offset of the unit from the first
-// staged word.  Returns the 8 elements as packed bf16 (Algorithm 1 line 11).
+// Eight elements selected by `bits` (bit e*step set = element e kept); the packed vector holds
+// the kept elements of these bit positions consecutively from index r0.  Returns 8 packed bf16.
 template <int DT>
-__device__ __forceinline__ uint4 decompress_unit(const uint32_t* __restrict__ words,
-                                                 const uint32_t* __restrict__ wrank, int rel,
-                                                 const void* __restrict__ values) {
-  const int wi = rel >> 5, sh = rel & 31;
-  const uint32_t word = words[wi];
-  const uint32_t byte = (word >> sh) & 0xFFu;
-  uint32_t r = wrank[wi] + __popc(word & ((1u << sh) - 1u));
+__device__ __forceinline__ uint4 gather8(uint32_t bits, uint32_t r0, int step,
+                                         const void* __restrict__ values) {
   uint4 out = make_uint4(0, 0, 0, 0);
-  if (byte == 0) return out;
+  if (bits == 0) return out;
   if (DT == 0) {
     const float* v = reinterpret_cast<const float*>(values);
     float f[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      const bool on = (byte >> e) & 1u;
-      f[e] = on ? __ldg(v + r) : 0.0f;
-      r += on ? 1u : 0u;
+      const int b = e * step;
+      const bool on = (bits >> b) & 1u;
+      f[e] = on ? __ldg(v + r0 + __popc(bits & ((1u << b) - 1u))) : 0.0f;
     }
     out.x = pack_bf16x2(f[0], f[1]); out.y = pack_bf16x2(f[2], f[3]);
     out.z = pack_bf16x2(f[4], f[5]); out.w = pack_bf16x2(f[6], f[7]);
@@ -67,9 +64,9 @@ __device__ __forceinline__ uint4 decompress_unit(const uint32_t* __restrict__ wo
     uint32_t h[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      const bool on = (byte >> e) & 1u;
-      h[e] = on ? static_cast<uint32_t>(__ldg(v + r)) : 0u;
-      r += on ? 1u : 0u;
+      const int b = e * step;
+      const bool on = (bits >> b) & 1u;
+      h[e] = on ? static_cast<uint32_t>(__ldg(v + r0 + __popc(bits & ((1u << b) - 1u)))) : 0u;
     }
     out.x = h[0] | (h[1] << 16); out.y = h[2] | (h[3] << 16);
     out.z = h[4] | (h[5] << 16); out.w = h[6] | (h[7] << 16);
@@ -80,8 +77,9 @@ __device__ __forceinline__ uint4 decompress_unit(const uint32_t* __restrict__ wo
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 1)
 dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ values,
-                    const unsigned long long* __restrict__ offsets, const float* __restrict__ grad,
-                    float* __restrict__ partial, uint32_t* __restrict__ status, FastParams p) {
+                    const unsigned long long* __restrict__ offsets,
+                    const __grid_constant__ CUtensorMap grad_map, float* __restrict__ partial,
+                    uint32_t* __restrict__ status, FastParams p) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -110,8 +108,9 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
   const uint32_t acc_bar = smem_u32(bars + 2 * kMaxStages);
 
   if (tid == 0) {
+    tma_prefetch_desc(&grad_map);
     for (int s = 0; s < p.stages; ++s) {
-      mbar_init(full_bar + 8 * s, kGroupWarps);
+      mbar_init(full_bar + 8 * s, kGroupWarps + 1);   // 8 warps + the thread that starts the TMA
       mbar_init(empty_bar + 8 * s, 1);
     }
     mbar_init(acc_bar, 1);
@@ -171,9 +170,9 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
     const int first_c = (p.mode == 0) ? nn0 / 9 : nn0;
     const int last_c = (p.mode == 0) ? (nn0 + rows_valid - 1) / 9 : nn0 + rows_valid - 1;
     const int n_ch = last_c - first_c + 1;   // mode 0: <= 16, mode 1: <= 128
-    const int range_words = (p.mode == 0) ? 32 : 4;
+    const int HW = p.H * p.W;
+    const int half_w = p.W >> 1;
 
-    // Geometry of K-tile `it` of this CTA.
     struct Tile { int img, p0, k_valid, iy_lo, range_len; };
     auto tile_of = [&](int it) {
       Tile t;
@@ -181,28 +180,27 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
       t.img = kt / p.tiles_per_img;
       t.p0 = (kt - t.img * p.tiles_per_img) * kTileK;
       t.k_valid = min(kTileK, p.P - t.p0);
+      t.iy_lo = 0;
+      t.range_len = 0;
       if (p.mode == 0) {
-        const int y_first = t.p0 / p.W;
-        const int y_last = (t.p0 + t.k_valid - 1) / p.W;
-        t.iy_lo = max(y_first - 1, 0);
-        const int iy_hi = min(y_last + 1, p.H - 1);
+        const int y_first = t.p0 / p.OW;
+        const int y_last = (t.p0 + t.k_valid - 1) / p.OW;
+        t.iy_lo = max(y_first * p.stride - 1, 0);
+        const int iy_hi = min(y_last * p.stride + 1, p.H - 1);
         t.range_len = (iy_hi - t.iy_lo + 1) * p.W;
-      } else {
-        t.iy_lo = 0;
-        t.range_len = t.k_valid;
       }
       return t;
     };
-    // First flat index of range `ri` (channel first_c + ri) of a tile.
-    auto range_start = [&](const Tile& t, int ri) -> long long {
-      const long long plane = (static_cast<long long>(t.img) * p.C + first_c + ri) * p.P;
-      return (p.mode == 0) ? plane + static_cast<long long>(t.iy_lo) * p.W : plane + t.p0;
+    auto plane_of = [&](const Tile& t, int ri) -> long long {
+      return (static_cast<long long>(t.img) * p.C + first_c + ri) * HW;
     };
-    // Stage the bitmap words and per-word ranks of every range of a tile.
+    // Stage what the decompression of a tile needs.
+    //  patch mode : per channel range, its bitmap words and the rank of each word's first bit;
+    //  direct mode: per (channel, chunk of 8 outputs), the 8*stride bitmap bits and their rank.
     auto stage_meta = [&](const Tile& t) {
       if (p.mode == 0) {
         for (int ri = gwarp; ri < n_ch; ri += kGroupWarps) {
-          const long long start = range_start(t, ri);
+          const long long start = plane_of(t, ri) + static_cast<long long>(t.iy_lo) * p.W;
           const long long first_word = start >> 5;
           const long long blk = start >> 10;
           const long long blk_word0 = blk << 5;
@@ -217,23 +215,46 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
           m_rank[ri * 32 + lane] = base + ex;
         }
       } else {
+        const int nbits = 8 * p.stride;
+        const uint32_t bmask = (nbits == 8) ? 0xFFu : 0xFFFFu;
         for (int ri = gtid; ri < n_ch; ri += kGroupThreads) {
-          const long long start = range_start(t, ri);
-          const long long first_word = start >> 5;
-          const long long blk = start >> 10;
-          const long long blk_word0 = blk << 5;
-          uint32_t base = static_cast<uint32_t>(__ldg(offsets + blk));
-          const int before = static_cast<int>(first_word - blk_word0);
+          const long long plane = plane_of(t, ri);
+          // cursor = (flat position, kept elements before it)
+          const int y0 = t.p0 / p.OW;
+          const int x00 = t.p0 - y0 * p.OW;
+          long long pos = plane + static_cast<long long>(y0 * p.stride) * p.W + x00 * p.stride;
+          const long long blk = pos >> 10;
+          uint32_t rank = static_cast<uint32_t>(__ldg(offsets + blk));
+          {
+            const long long blk_word0 = blk << 5;
+            const int before = static_cast<int>((pos >> 5) - blk_word0);
 #pragma unroll 8
-          for (int w = 0; w < 31; ++w)
-            if (w < before) base += __popc(__ldg(bitmap + blk_word0 + w));
-          const int nwords = static_cast<int>(((start + t.range_len - 1) >> 5) - first_word) + 1;
-#pragma unroll
-          for (int w = 0; w < 4; ++w) {
-            const uint32_t word = (w < nwords) ? __ldg(bitmap + first_word + w) : 0u;
-            m_words[ri * 4 + w] = word;
-            m_rank[ri * 4 + w] = base;
-            base += __popc(word);
+            for (int w = 0; w < 31; ++w)
+              if (w < before) rank += __popc(__ldg(bitmap + blk_word0 + w));
+            const uint32_t w0 = __ldg(bitmap + (pos >> 5));
+            rank += __popc(w0 & ((1u << (pos & 31)) - 1u));
+          }
+          int y = y0, x = x00;
+          for (int chunk = 0; chunk < 8; ++chunk) {
+            uint32_t bits = 0;
+            if (chunk * 8 < t.k_valid) {
+              const long long want = plane + static_cast<long long>(y * p.stride) * p.W + x * p.stride;
+              while (pos < want) {       // skipped input (odd rows of a stride-2 layer)
+                const int lo = static_cast<int>(pos & 31);
+                const long long left = want - pos;
+                const int take = (left < 32 - lo) ? static_cast<int>(left) : 32 - lo;
+                const uint32_t m = (take == 32) ? 0xFFFFFFFFu : (((1u << take) - 1u) << lo);
+                rank += __popc(__ldg(bitmap + (pos >> 5)) & m);
+                pos += take;
+              }
+              bits = (__ldg(bitmap + (pos >> 5)) >> (pos & 31)) & bmask;
+            }
+            m_words[ri * 8 + chunk] = bits;
+            m_rank[ri * 8 + chunk] = rank;
+            rank += __popc(bits);
+            pos += nbits;
+            x += 8;
+            if (x >= p.OW) { x = 0; ++y; }
           }
         }
       }
@@ -251,59 +272,46 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
       group_sync(g);    // staged metadata visible; every thread of the group sees the same *fail
       if (*fail) break;
       unsigned char* a_tile = smem + s * stage_bytes;
-      unsigned char* b_tile = a_tile + kTileM * 128;
       const Tile t = tile_of(it);
 
-      // gradient chunks travel through registers in batches, loads issued early
-      const int g_tasks = n_cols * 8;
-      const int g_batches = (g_tasks + kGroupThreads * kGBatch - 1) / (kGroupThreads * kGBatch);
-      float4 gr[kGBatch][2];
-      auto g_issue = [&](int batch) {
-#pragma unroll
-        for (int i = 0; i < kGBatch; ++i) {
-          const int task = (batch * kGBatch + i) * kGroupThreads + gtid;
-          const int row = task >> 3, chunk = task & 7;
-          const int o = o0 + row;
-          const int pp = t.p0 + chunk * 8;
-          gr[i][0] = make_float4(0.f, 0.f, 0.f, 0.f);
-          gr[i][1] = gr[i][0];
-          if (task < g_tasks && o < p.O && pp < p.P) {
-            const float4* src = reinterpret_cast<const float4*>(
-                grad + (static_cast<long long>(t.img) * p.O + o) * p.P + pp);
-            gr[i][0] = __ldg(src);
-            gr[i][1] = __ldg(src + 1);
-          }
-        }
-      };
-      auto g_store = [&](int batch) {
-#pragma unroll
-        for (int i = 0; i < kGBatch; ++i) {
-          const int task = (batch * kGBatch + i) * kGroupThreads + gtid;
-          if (task < g_tasks) {
-            uint4 out;
-            out.x = pack_bf16x2(gr[i][0].x, gr[i][0].y); out.y = pack_bf16x2(gr[i][0].z, gr[i][0].w);
-            out.z = pack_bf16x2(gr[i][1].x, gr[i][1].y); out.w = pack_bf16x2(gr[i][1].z, gr[i][1].w);
-            *reinterpret_cast<uint4*>(b_tile + tile_off(task >> 3, task & 7)) = out;
-          }
-        }
-      };
-      g_issue(0);
+      // gradient tile(s): bf16 rows [o0, o0 + n_cols) x 64 positions of image t.img, by TMA
+      if (gtid == 0) {
+        mbar_arrive_expect_tx(full_bar + 8 * s, static_cast<uint32_t>(n_cols) * 128u);
+        const uint32_t b_addr = smem_u32(a_tile) + kTileM * 128;
+        for (int a = 0; a < p.n_acc; ++a)
+          tma_load_3d(b_addr + a * p.acc_n * 128, &grad_map, t.p0, o0 + a * p.acc_n, t.img,
+                      full_bar + 8 * s);
+      }
 
       if (p.mode == 0) {
-        // ---- decompress the channel ranges into the patch, 8 elements per thread ----
+        // ---- decompress the channel ranges into the patch, 8 input elements per thread ----
         const int units_per_range = t.range_len >> 3;
         const int units = n_ch * units_per_range;
         for (int u = gtid; u < units; u += kGroupThreads) {
           const int ri = u / units_per_range;
           const int uu = u - ri * units_per_range;
-          const int bit0 = static_cast<int>(range_start(t, ri) & 31);
-          const uint4 v = decompress_unit<DT>(m_words + ri * 32, m_rank + ri * 32, bit0 + uu * 8,
-                                              values);
-          *reinterpret_cast<uint4*>(patch + ri * t.range_len + uu * 8) = v;
+          const long long start = plane_of(t, ri) + static_cast<long long>(t.iy_lo) * p.W;
+          const int rel = static_cast<int>(start & 31) + uu * 8;
+          const uint32_t word = m_words[ri * 32 + (rel >> 5)];
+          const int sh = rel & 31;
+          const uint32_t r0 = m_rank[ri * 32 + (rel >> 5)] + __popc(word & ((1u << sh) - 1u));
+          const uint4 v = gather8<DT>((word >> sh) & 0xFFu, r0, 1, values);
+          unsigned short* dst = patch + ri * t.range_len;
+          if (p.stride == 1) {
+            *reinterpret_cast<uint4*>(dst + uu * 8) = v;
+          } else {
+            // even input columns to the first half of the row, odd ones to the second half
+            const int e0 = uu * 8;
+            const int row = e0 / p.W;
+            const int xin = e0 - row * p.W;
+            uint2 ev, od;
+            ev.x = __byte_perm(v.x, v.y, 0x5410); ev.y = __byte_perm(v.z, v.w, 0x5410);
+            od.x = __byte_perm(v.x, v.y, 0x7632); od.y = __byte_perm(v.z, v.w, 0x7632);
+            *reinterpret_cast<uint2*>(dst + row * p.W + (xin >> 1)) = ev;
+            *reinterpret_cast<uint2*>(dst + row * p.W + half_w + (xin >> 1)) = od;
+          }
         }
         group_sync(g);
-        g_store(0);
-        if (g_batches > 1) g_issue(1);
         // ---- im2col view: one task = (channel, filter row r, chunk) -> columns s = 0, 1, 2 ----
         const int tasks = n_ch * 24;
         for (int q = gtid; q < tasks; q += kGroupThreads) {
@@ -311,59 +319,60 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
           const int rem = q - ci * 24;
           const int r = rem >> 3, chunk = rem & 7;
           const int pp = t.p0 + chunk * 8;
-          const int y = pp / p.W;
-          const int x0 = pp - y * p.W;
-          const int iy = y + r - 1;
-          uint4 c4 = make_uint4(0, 0, 0, 0);
-          uint32_t left = 0, right = 0;
+          const int y = pp / p.OW;
+          const int x0 = pp - y * p.OW;
+          const int iy = y * p.stride + r - 1;
+          uint4 s0 = make_uint4(0, 0, 0, 0), s1 = s0, s2 = s0;
           if (pp < p.P && iy >= 0 && iy < p.H) {
-            const unsigned short* src = patch + ci * t.range_len + (iy - t.iy_lo) * p.W + x0;
-            c4 = *reinterpret_cast<const uint4*>(src);
-            if (x0 > 0) left = src[-1];
-            if (x0 + 8 < p.W) right = src[8];
+            const unsigned short* rowp = patch + ci * t.range_len + (iy - t.iy_lo) * p.W;
+            if (p.stride == 1) {
+              const unsigned short* src = rowp + x0;
+              const uint4 c4 = *reinterpret_cast<const uint4*>(src);
+              const uint32_t left = (x0 > 0) ? src[-1] : 0u;
+              const uint32_t right = (x0 + 8 < p.W) ? src[8] : 0u;
+              s1 = c4;
+              s0.x = (c4.x << 16) | left;
+              s0.y = __funnelshift_l(c4.x, c4.y, 16);
+              s0.z = __funnelshift_l(c4.y, c4.z, 16);
+              s0.w = __funnelshift_l(c4.z, c4.w, 16);
+              s2.x = __funnelshift_r(c4.x, c4.y, 16);
+              s2.y = __funnelshift_r(c4.y, c4.z, 16);
+              s2.z = __funnelshift_r(c4.z, c4.w, 16);
+              s2.w = (c4.w >> 16) | (right << 16);
+            } else {
+              // input column 2x + s - 1: s = 1 -> even plane[x], s = 2 -> odd plane[x],
+              // s = 0 -> odd plane[x - 1]
+              s1 = *reinterpret_cast<const uint4*>(rowp + x0);
+              const unsigned short* odd = rowp + half_w + x0;
+              s2 = *reinterpret_cast<const uint4*>(odd);
+              const uint32_t left = (x0 > 0) ? odd[-1] : 0u;
+              s0.x = (s2.x << 16) | left;
+              s0.y = __funnelshift_l(s2.x, s2.y, 16);
+              s0.z = __funnelshift_l(s2.y, s2.z, 16);
+              s0.w = __funnelshift_l(s2.z, s2.w, 16);
+            }
           }
           const int row0 = (first_c + ci) * 9 + r * 3 - nn0;
-          uint4 lo4, hi4;   // shifted by -1 (s = 0) and by +1 (s = 2)
-          lo4.x = (c4.x << 16) | left;
-          lo4.y = __funnelshift_l(c4.x, c4.y, 16);
-          lo4.z = __funnelshift_l(c4.y, c4.z, 16);
-          lo4.w = __funnelshift_l(c4.z, c4.w, 16);
-          hi4.x = __funnelshift_r(c4.x, c4.y, 16);
-          hi4.y = __funnelshift_r(c4.y, c4.z, 16);
-          hi4.z = __funnelshift_r(c4.z, c4.w, 16);
-          hi4.w = (c4.w >> 16) | (right << 16);
           if (row0 >= 0 && row0 < rows_valid)
-            *reinterpret_cast<uint4*>(a_tile + tile_off(row0, chunk)) = lo4;
+            *reinterpret_cast<uint4*>(a_tile + tile_off(row0, chunk)) = s0;
           if (row0 + 1 >= 0 && row0 + 1 < rows_valid)
-            *reinterpret_cast<uint4*>(a_tile + tile_off(row0 + 1, chunk)) = c4;
+            *reinterpret_cast<uint4*>(a_tile + tile_off(row0 + 1, chunk)) = s1;
           if (row0 + 2 >= 0 && row0 + 2 < rows_valid)
-            *reinterpret_cast<uint4*>(a_tile + tile_off(row0 + 2, chunk)) = hi4;
+            *reinterpret_cast<uint4*>(a_tile + tile_off(row0 + 2, chunk)) = s2;
         }
       } else {
-        // ---- 1x1: decompress straight into the operand tile; row = channel, chunk = unit ----
+        // ---- 1x1: decompress straight into the operand tile; row = channel, chunk = 8 outputs
         const int units = rows_valid * 8;
         for (int u = gtid; u < units; u += kGroupThreads) {
           const int ri = u >> 3, chunk = u & 7;
-          uint4 v = make_uint4(0, 0, 0, 0);
-          if (chunk * 8 < t.k_valid) {
-            const int bit0 = static_cast<int>(range_start(t, ri) & 31);
-            v = decompress_unit<DT>(m_words + ri * 4, m_rank + ri * 4, bit0 + chunk * 8, values);
-          }
+          const uint4 v = gather8<DT>(m_words[u], m_rank[u], p.stride, values);
           *reinterpret_cast<uint4*>(a_tile + tile_off(ri, chunk)) = v;
         }
-        g_store(0);
-        if (g_batches > 1) g_issue(1);
-      }
-      for (int b = 1; b < g_batches; ++b) {
-        g_store(b);
-        if (b + 1 < g_batches) g_issue(b + 1);
+        group_sync(g);    // everyone is done with this tile's metadata
       }
       fence_proxy_async();
       __syncwarp();
       if (lane == 0) mbar_arrive(full_bar + 8 * s);
-      // metadata of this group's next tile (the group_sync at the top of the loop publishes it;
-      // the one after the decompression above guarantees nobody still reads the old one)
-      if (p.mode == 1) group_sync(g);
       if (it + kGroups < n_kt) stage_meta(tile_of(it + kGroups));
     }
   }
@@ -397,20 +406,49 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
   if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
 }
 
+// fp32 -> bf16 (round to nearest even), 8 elements per thread.
+__global__ void __launch_bounds__(256)
+grad_to_bf16_kernel(const float* __restrict__ g, long long n, unsigned short* __restrict__ out) {
+  const long long n8 = n >> 3;
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n8;
+       i += stride) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(g) + 2 * i);
+    const float4 b = __ldg(reinterpret_cast<const float4*>(g) + 2 * i + 1);
+    uint4 o;
+    o.x = pack_bf16x2(a.x, a.y); o.y = pack_bf16x2(a.z, a.w);
+    o.z = pack_bf16x2(b.x, b.y); o.w = pack_bf16x2(b.z, b.w);
+    reinterpret_cast<uint4*>(out)[i] = o;
+  }
+  if (blockIdx.x == 0)
+    for (long long j = (n8 << 3) + threadIdx.x; j < n; j += blockDim.x)
+      out[j] = static_cast<unsigned short>(pack_bf16x2(g[j], 0.0f) & 0xFFFFu);
+}
+
 }  // namespace
 
 bool plan_conv_fast(const surgeon_layer_desc& d, FastParams* out) {
-  if (d.kind != 1 || d.stride != 1) return false;
+  if (d.kind != 1 || (d.stride != 1 && d.stride != 2)) return false;
   int mode;
   if (d.kh == 3 && d.kw == 3 && d.pad == 1) mode = 0;
   else if (d.kh == 1 && d.kw == 1 && d.pad == 0) mode = 1;
   else return false;
-  if (d.w % 8 != 0) return false;
   FastParams p{};
   p.mode = mode;
+  p.stride = d.stride;
   p.B = d.batch; p.C = d.c_in; p.H = d.h; p.W = d.w; p.O = d.c_out;
-  p.P = d.h * d.w;
+  p.OH = (d.h + 2 * d.pad - d.kh) / d.stride + 1;
+  p.OW = (d.w + 2 * d.pad - d.kw) / d.stride + 1;
+  p.P = p.OH * p.OW;
   p.n_gemm = d.c_in * d.kh * d.kw;
+  if (mode == 0) {
+    if (d.w % (8 * d.stride) != 0 || p.OW % 8 != 0) return false;
+  } else if (d.stride == 1) {
+    if ((d.h * d.w) % 8 != 0) return false;      // chunks of 8 never straddle an image
+  } else {
+    if (d.w % 16 != 0 || p.OW % 8 != 0) return false;
+  }
+  if (p.P % 8 != 0) return false;                 // TMA row pitch of the bf16 gradient: 16 bytes
   // accumulator width: the widest multiple of 16 up to 256 that divides O, else 256 with padding
   int acc_n = 0;
   for (int c = 256; c >= 128; c -= 16)
@@ -426,8 +464,8 @@ bool plan_conv_fast(const surgeon_layer_desc& d, FastParams* out) {
   if (total > 2147483647LL) return false;
   p.total_ktiles = static_cast<int>(total);
   if (mode == 0) {
-    const int out_rows = (kTileK + p.W - 2) / p.W + 1;
-    int in_rows = out_rows + 2;
+    const int out_rows = (kTileK + p.OW - 2) / p.OW + 1;
+    int in_rows = (out_rows - 1) * d.stride + 3;
     if (in_rows > p.H) in_rows = p.H;
     const int range_len = in_rows * p.W;
     if (range_len + 31 > 32 * 32) return false;
@@ -462,9 +500,36 @@ bool plan_conv_fast(const surgeon_layer_desc& d, FastParams* out) {
   return true;
 }
 
+size_t conv_fast_grad_bf16_bytes(const FastParams& p) {
+  const size_t b = static_cast<size_t>(p.B) * p.O * p.P * 2;
+  return (b + 255) & ~static_cast<size_t>(255);
+}
+
 cudaError_t launch_conv_fast(const surgeon_compressed& act, const FastParams& p,
-                             const float* grad_out, float* partial, uint32_t* status,
-                             cudaStream_t stream) {
+                             const float* grad_out, void* grad_bf16, float* partial,
+                             uint32_t* status, cudaStream_t stream) {
+  // 1. gradient fp32 -> bf16 (scratch), then a 3-D tensor map over [B][O][P] for the TMA loads
+  const long long gn = static_cast<long long>(p.B) * p.O * p.P;
+  {
+    const long long want = (gn / 8 + 255) / 256;
+    const long long cap = 16LL * sm_count();
+    const int grid = static_cast<int>(want < 1 ? 1 : (want > cap ? cap : want));
+    grad_to_bf16_kernel<<<grid, 256, 0, stream>>>(grad_out, gn,
+                                                  static_cast<unsigned short*>(grad_bf16));
+  }
+  CUtensorMap map;
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(p.P), static_cast<cuuint64_t>(p.O),
+                              static_cast<cuuint64_t>(p.B)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(p.P) * 2,
+                                 static_cast<cuuint64_t>(p.P) * p.O * 2};
+  const cuuint32_t box[3] = {static_cast<cuuint32_t>(kTileK), static_cast<cuuint32_t>(p.acc_n), 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = cuTensorMapEncodeTiled(
+      &map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, grad_bf16, dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+
   const unsigned long long* offs = reinterpret_cast<const unsigned long long*>(act.block_offsets);
   dim3 grid(p.m_tiles, p.n_tiles, p.splits);
   cudaError_t e;
@@ -473,14 +538,15 @@ cudaError_t launch_conv_fast(const surgeon_compressed& act, const FastParams& p,
                              p.smem_bytes);
     if (e != cudaSuccess) return e;
     dw_conv_fast_kernel<0><<<grid, kThreads, p.smem_bytes, stream>>>(
-        act.bitmap, act.values, offs, grad_out, partial, status, p);
+        act.bitmap, act.values, offs, map, partial, status, p);
   } else {
     e = cudaFuncSetAttribute(dw_conv_fast_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              p.smem_bytes);
     if (e != cudaSuccess) return e;
     dw_conv_fast_kernel<1><<<grid, kThreads, p.smem_bytes, stream>>>(
-        act.bitmap, act.values, offs, grad_out, partial, status, p);
+        act.bitmap, act.values, offs, map, partial, status, p);
   }
+  note_launches(2);
   return cudaGetLastError();
 }
 

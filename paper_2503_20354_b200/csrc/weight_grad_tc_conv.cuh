@@ -7,8 +7,9 @@ namespace surgeon {
 
 struct FastParams {
   int mode;                 // 0 = 3x3 pad 1 through a shared-memory patch, 1 = 1x1 direct
-  int B, C, H, W, O;
-  int P;                    // output positions per image (= H*W)
+  int stride;               // 1 or 2
+  int B, C, H, W, O, OH, OW;
+  int P;                    // output positions per image (= OH*OW)
   int n_gemm;               // C*KH*KW
   int acc_n, n_acc;         // columns per accumulator, accumulators per CTA (1 or 2)
   int n_tiles, m_tiles;
@@ -19,9 +20,13 @@ struct FastParams {
 // False when the layer is not one the fast kernel handles.
 bool plan_conv_fast(const surgeon_layer_desc& d, FastParams* out);
 
-// Enqueues the kernel; partial = [splits][O][n_gemm] fp32, status = one zeroed word.
+// Bytes of scratch for the bf16 copy of the output gradient.
+size_t conv_fast_grad_bf16_bytes(const FastParams& p);
+
+// Enqueues the bf16 conversion of grad_out into grad_bf16 and the kernel;
+// partial = [splits][O][n_gemm] fp32, status = one zeroed word.
 cudaError_t launch_conv_fast(const surgeon_compressed& act, const FastParams& p,
-                             const float* grad_out, float* partial, uint32_t* status,
-                             cudaStream_t stream);
+                             const float* grad_out, void* grad_bf16, float* partial,
+                             uint32_t* status, cudaStream_t stream);
 
 }  // namespace surgeon

@@ -65,6 +65,10 @@ SHAPES = [
     W.conv("f1x1_w8", 5, 200, 8, 48, 1, 1, 0),
     W.conv("f1x1_w56", 2, 64, 56, 256, 1, 1, 0),
     W.Layer("f1x1_h12w8_tail_ktile", 1, 3, 40, 12, 8, 32, 1, 1, 1, 0),
+    W.conv("f3x3_s2_w32", 3, 20, 32, 40, 3, 2),
+    W.conv("f3x3_s2_w16_two_acc", 4, 16, 16, 320, 3, 2),
+    W.conv("f1x1_s2_w32", 3, 150, 32, 48, 1, 2, 0),
+    W.conv("f1x1_s2_w16", 5, 24, 16, 320, 1, 2, 0),
     W.linear("fc", 64, 2048, 1000, dist="abs_normal", dt=W.F32),
     W.linear("tokens", 2 * 197, 768, 256, dist="normal", dt=W.F32),
     W.linear("tiny", 5, 7, 3, dist="normal", dt=W.F32),
