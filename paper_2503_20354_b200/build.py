@@ -39,7 +39,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         flags += ["-Xptxas", "-v"]
     tmp = LIB + ".tmp%d" % os.getpid()
     cmd = [nvcc] + flags + ["-I", os.path.join(ROOT, "include"), "-I", CSRC] + sources() + [
-        "-o", tmp, "-lcuda"]
+        "-o", tmp]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)
     return LIB

@@ -425,6 +425,24 @@ grad_to_bf16_kernel(const float* __restrict__ g, long long n, unsigned short* __
       out[j] = static_cast<unsigned short>(pack_bf16x2(g[j], 0.0f) & 0xFFFFu);
 }
 
+// The driver's tensor-map encoder, looked up through the runtime so that the library carries no
+// link-time dependency on the driver library (it must load on machines without a GPU).
+using TensorMapEncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                       const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                       const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                       CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+TensorMapEncodeFn tensor_map_encoder() {
+  static TensorMapEncodeFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<TensorMapEncodeFn>(p);
+  }();
+  return fn;
+}
+
 }  // namespace
 
 bool plan_conv_fast(const surgeon_layer_desc& d, FastParams* out) {
@@ -524,7 +542,9 @@ cudaError_t launch_conv_fast(const surgeon_compressed& act, const FastParams& p,
                                  static_cast<cuuint64_t>(p.P) * p.O * 2};
   const cuuint32_t box[3] = {static_cast<cuuint32_t>(kTileK), static_cast<cuuint32_t>(p.acc_n), 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult r = cuTensorMapEncodeTiled(
+  const TensorMapEncodeFn encode = tensor_map_encoder();
+  if (!encode) return cudaErrorNotSupported;
+  const CUresult r = encode(
       &map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, grad_bf16, dims, strides, box, estr,
       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
