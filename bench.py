@@ -3,8 +3,8 @@
 
 One step = one pass of the whole path over one batch of the WideResNet-28-10-shaped stack
 (batch 200, 28 conv layers, fp32 activations): per-layer ratios (Eq. 5-7), prune+compact of every
-saved activation (Algorithm 1 lines 6-7), and the weight gradient of every layer from its
-compressed store (lines 11-12).  Prints ONE JSON line (rank 0).
+saved activation (Algorithm 1: prune and decompose steps), and the weight gradient of every layer from its
+compressed store (its Reshape and gradient steps).  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                   [--workload wrn28|tiny|resnet50|vit] [--batch B] [--path tc|fp32]

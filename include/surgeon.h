@@ -5,10 +5,10 @@
  * Adaptation via Dynamic Activation Sparsity" (arXiv 2503.20354):
  *
  *   per-layer pruning ratio (Eq. 5-7)  ->  prune the saved activation A_i at
- *   that ratio (Algorithm 1, line 6)   ->  store it as packed kept values plus a
- *   1-bit-per-element index (Algorithm 1, line 7; Section 4.2, "Algorithm"
+ *   that ratio (Algorithm 1: prune step)   ->  store it as packed kept values plus a
+ *   1-bit-per-element index (Algorithm 1: decompose step; Section 4.2, "Algorithm"
  *   paragraph)  ->  rebuild the sparse activation and form the weight gradient
- *   from it (Algorithm 1, lines 11-12; Eq. 2).
+ *   from it (Algorithm 1: Reshape and gradient steps; Eq. 2).
  *
  * Conventions shared by every entry point
  *   - Every function returns a surgeon_status; argument errors are found on the
@@ -70,7 +70,7 @@ surgeon_status surgeon_layer_ratios(const double* gi, const double* lam, int32_t
                                     double* ratios_out);
 
 /* ------------------------------------------------------------------------------------------
- * Algorithm 1, line 6 ("prune A_i with ratio p"): the kept count and the buffer sizes.
+ * Algorithm 1: prune step ("prune A_i with ratio p"): the kept count and the buffer sizes.
  * Pure host arithmetic.  n_prune = floor(ratio * n) evaluated in IEEE double, n_keep = n -
  * n_prune.  Any out pointer may be NULL.  bitmap_bytes = 4*ceil(n/32); values_bytes =
  * n_keep*sizeof(dt); offsets_bytes = 8*(ceil(n/SURGEON_BLOCK)+1); workspace_bytes = scratch
@@ -109,7 +109,7 @@ typedef struct surgeon_compressed {
 } surgeon_compressed;
 
 /* ------------------------------------------------------------------------------------------
- * Algorithm 1, lines 6-7: prune the activation x (n elements of dt, device pointer, not
+ * Algorithm 1: prune and decompose steps: prune the activation x (n elements of dt, device pointer, not
  * modified) by magnitude at `ratio` and write the compressed store.
  * Kept set: the n_keep elements with the largest magnitude key (bit pattern with the sign bit
  * cleared, compared as an unsigned integer: equals |x| order on finite data, -0 ties with +0,
@@ -139,7 +139,7 @@ typedef struct surgeon_layer_desc {
 size_t surgeon_weight_grad_workspace(const surgeon_layer_desc* d);
 
 /* ------------------------------------------------------------------------------------------
- * Algorithm 1, lines 11-12 with Eq. 2 (weight gradient only): rebuild the sparse activation
+ * Algorithm 1: Reshape and gradient steps with Eq. 2 (weight gradient only): rebuild the sparse activation
  * from the store on chip and contract it with the output gradient.
  *   linear:  dw[o, c]       = sum_t        grad_out[t, o]       * A[t, c]
  *   conv2d:  dw[o, c, r, s] = sum_{b,y,x}  grad_out[b, o, y, x] * A[b, c, y*stride + r - pad,
@@ -160,7 +160,7 @@ surgeon_status surgeon_weight_grad(const surgeon_compressed* act, const surgeon_
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
- * Algorithm 1, line 11 ("Reshape") as a stand-alone utility: x_out[j] = kept ? value : +0 for
+ * Algorithm 1: Reshape step ("Reshape") as a stand-alone utility: x_out[j] = kept ? value : +0 for
  * all j < act->n, in act->dt.  x_out: device pointer to n elements.  surgeon_weight_grad does
  * not call this (it rebuilds tiles in shared memory); tests use it.  Asynchronous.
  * ---------------------------------------------------------------------------------------- */

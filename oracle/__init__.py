@@ -98,12 +98,12 @@ def layer_ratios(gi, lam):
 
 
 def n_keep(n: int, ratio: float) -> int:
-    """Algorithm 1 line 6: kept count for ``ratio`` = n - floor(ratio*n)."""
+    """Algorithm 1: prune step: kept count for ``ratio`` = n - floor(ratio*n)."""
     return int(_load().oracle_n_keep(int(n), float(ratio)))
 
 
 def select(x: np.ndarray, k: int, method: int = 1):
-    """Algorithm 1 line 6: the k largest-magnitude elements, ties by lowest flat index.
+    """Algorithm 1: prune step: the k largest-magnitude elements, ties by lowest flat index.
 
     Returns (keep uint8[n], tau, c_gt, q).  method 0 = full stable sort, 1 = nth_element."""
     x = np.ascontiguousarray(x).reshape(-1)
@@ -118,7 +118,7 @@ def select(x: np.ndarray, k: int, method: int = 1):
 
 
 def compact(x: np.ndarray, keep: np.ndarray, block: int = BLOCK):
-    """Algorithm 1 line 7: (bitmap uint32[ceil(n/32)], values[k], offsets uint64[ceil(n/block)+1])."""
+    """Algorithm 1: decompose step: (bitmap uint32[ceil(n/32)], values[k], offsets uint64[ceil(n/block)+1])."""
     x = np.ascontiguousarray(x).reshape(-1)
     dt = _dt_of(x)
     keep = np.ascontiguousarray(keep, dtype=np.uint8)
@@ -134,7 +134,7 @@ def compact(x: np.ndarray, keep: np.ndarray, block: int = BLOCK):
 
 
 def decompress(bitmap: np.ndarray, values: np.ndarray, n: int) -> np.ndarray:
-    """Algorithm 1 line 11: dense tensor (flat) from the store, +0 where the bit is clear."""
+    """Algorithm 1: Reshape step: dense tensor (flat) from the store, +0 where the bit is clear."""
     bitmap = np.ascontiguousarray(bitmap, dtype=np.uint32)
     values = np.ascontiguousarray(values)
     dt = _dt_of(values)
@@ -144,7 +144,7 @@ def decompress(bitmap: np.ndarray, values: np.ndarray, n: int) -> np.ndarray:
 
 
 def prune_compact(x: np.ndarray, ratio: float, method: int = 1, block: int = BLOCK):
-    """Algorithm 1 lines 6-7 in one call: dict with tau, k, c_gt, q, keep, bitmap, values, offsets."""
+    """Algorithm 1: prune and decompose steps in one call: dict with tau, k, c_gt, q, keep, bitmap, values, offsets."""
     x = np.ascontiguousarray(x).reshape(-1)
     k = n_keep(x.size, ratio)
     keep, tau, cgt, q = select(x, k, method)

@@ -25,7 +25,7 @@ namespace {
 // Magnitude key: the element's bit pattern with the sign bit cleared, read as an unsigned
 // integer.  For finite values this orders exactly like |x|; -0 equals +0; Inf sits above every
 // finite value and NaN above Inf.  (The paper gives no pruning criterion beyond "prune with
-// ratio p", Algorithm 1 line 6; magnitude is the criterion of the activation-pruning works it
+// ratio p", Algorithm 1: prune step; magnitude is the criterion of the activation-pruning works it
 // builds on, Section 2.)
 inline uint32_t key_of(const void* x, int64_t j, int dt) {
   if (dt == 0) {
@@ -98,7 +98,7 @@ int oracle_layer_ratios(const double* G, const double* m, int l, double* p) {
   return 0;
 }
 
-// Algorithm 1, line 6: how many elements "ratio p" removes.  The paper does not state the
+// Algorithm 1: prune step: how many elements "ratio p" removes.  The paper does not state the
 // rounding; the reading is n_prune = floor(p*n) with the product taken once in double, and
 // the kept count is what remains.
 int64_t oracle_n_keep(int64_t n, double p) {
@@ -108,7 +108,7 @@ int64_t oracle_n_keep(int64_t n, double p) {
   return n - n_prune;
 }
 
-// Algorithm 1, line 6: the kept set = the k elements that come first when all elements are
+// Algorithm 1: prune step: the kept set = the k elements that come first when all elements are
 // ordered by magnitude key descending, equal keys by ascending flat index.
 //   method 0: stable sort of all indices by key (the definition written out);
 //   method 1: std::nth_element on (key, index) pairs under the same total order (same result,
@@ -144,7 +144,7 @@ void oracle_select(const void* x, int64_t n, int dt, int64_t k, int method, uint
   *q = k - greater;
 }
 
-// Algorithm 1, line 7 / Section 4.2: decompose the pruned activation into the vector of kept
+// Algorithm 1: decompose step / Section 4.2: decompose the pruned activation into the vector of kept
 // elements (ascending flat index, bit copies) and an index of 1 bit per element.  Bit (j & 31)
 // of 32-bit word (j >> 5) belongs to flat index j.  offsets[b] = kept elements below b*block;
 // offsets[ceil(n/block)] = total kept.  Returns the kept count.
@@ -166,7 +166,7 @@ int64_t oracle_compact(const void* x, int64_t n, int dt, const uint8_t* keep, in
   return r;
 }
 
-// Algorithm 1, line 11: Reshape(values, index) -> dense tensor with +0 where nothing is kept.
+// Algorithm 1: Reshape step: Reshape(values, index) -> dense tensor with +0 where nothing is kept.
 void oracle_decompress(const uint32_t* bitmap, const void* values, int64_t n, int dt,
                        void* x_out) {
   const size_t es = (dt == 0) ? 4 : 2;

@@ -116,7 +116,7 @@ def dtype_code(t: torch.dtype) -> int:
 
 
 # ---------------------------------------------------------------------------------------------
-# surgeon_layer_ratios (Eq. 5-7) and surgeon_compact_sizes (Algorithm 1 line 6): host arithmetic
+# surgeon_layer_ratios (Eq. 5-7) and surgeon_compact_sizes (Algorithm 1: prune step): host arithmetic
 # ---------------------------------------------------------------------------------------------
 
 def surgeon_layer_ratios(gi, lam, allow_degenerate: bool = False) -> np.ndarray:
@@ -150,7 +150,7 @@ def surgeon_compact_sizes(n: int, dt: int, ratio: float) -> CompactSizes:
 
 
 # ---------------------------------------------------------------------------------------------
-# The compressed store and surgeon_prune_compact (Algorithm 1 lines 6-7)
+# The compressed store and surgeon_prune_compact (Algorithm 1: prune and decompose steps)
 # ---------------------------------------------------------------------------------------------
 
 class CompressedActivation:
@@ -216,7 +216,7 @@ def surgeon_prune_compact(x: torch.Tensor, ratio: float, out: Optional[Compresse
 
 
 def surgeon_decompress(act: CompressedActivation, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
-    """Dense flat tensor rebuilt from the store (test utility; Algorithm 1 line 11)."""
+    """Dense flat tensor rebuilt from the store (test utility; Algorithm 1: Reshape step)."""
     vt = torch.float32 if act.dt == SURGEON_F32 else torch.bfloat16
     out = torch.empty(max(act.n, 1), dtype=vt, device=act.bitmap.device)
     st = lib().surgeon_decompress(C.byref(act.c), out.data_ptr(), _stream_ptr(stream))
@@ -225,7 +225,7 @@ def surgeon_decompress(act: CompressedActivation, stream: Optional[torch.cuda.St
 
 
 # ---------------------------------------------------------------------------------------------
-# surgeon_weight_grad (Algorithm 1 lines 11-12, Eq. 2)
+# surgeon_weight_grad (Algorithm 1: Reshape and gradient steps, Eq. 2)
 # ---------------------------------------------------------------------------------------------
 
 def layer_desc(layer, path: int) -> LayerDesc:

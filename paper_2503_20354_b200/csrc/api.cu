@@ -29,7 +29,7 @@ namespace {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Algorithm 1 line 6: kept count for `ratio`; one double multiply, one floor.
+// Algorithm 1: prune step: kept count for `ratio`; one double multiply, one floor.
 inline int64_t kept_count(int64_t n, double ratio) {
   double pruned = floor(ratio * static_cast<double>(n));
   if (pruned < 0.0) pruned = 0.0;

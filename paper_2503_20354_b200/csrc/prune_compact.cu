@@ -1,7 +1,7 @@
 // Threshold select and compaction kernels of surgeon_prune_compact, and surgeon_decompress.
 //
-// Algorithm 1, line 6: the kept set of a layer is its n_keep largest-magnitude elements, ties
-// at the threshold broken by lowest flat index.  Line 7 / Section 4.2: the pruned activation is
+// Algorithm 1: prune step: the kept set of a layer is its n_keep largest-magnitude elements, ties
+// at the threshold broken by lowest flat index.  Its decompose step / Section 4.2: the pruned activation is
 // cached as the vector of kept elements plus one index bit per element.
 //
 //   select  : radix select on the magnitude key.  Each pass histograms one digit of the keys
@@ -273,7 +273,7 @@ __global__ void offsets_empty_kernel(unsigned long long* offsets) { offsets[0] =
 
 // ---- decompress -------------------------------------------------------------------------------
 
-// Algorithm 1, line 11: one warp rebuilds one SURGEON_BLOCK of the dense tensor.
+// Algorithm 1: Reshape step: one warp rebuilds one SURGEON_BLOCK of the dense tensor.
 template <int DT>
 __global__ void __launch_bounds__(256)
 decompress_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ values_v,

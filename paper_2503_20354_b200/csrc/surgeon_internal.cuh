@@ -9,7 +9,7 @@
 namespace surgeon {
 
 // Storage type and magnitude-key mask per dtype.  The key is the bit pattern with the sign
-// bit cleared, compared as an unsigned integer (Algorithm 1 line 6 prunes by magnitude).
+// bit cleared, compared as an unsigned integer (Algorithm 1: prune step prunes by magnitude).
 template <int DT> struct Elem;
 template <> struct Elem<0> {
   using type = uint32_t;
@@ -41,7 +41,7 @@ constexpr size_t kWsStateBytes = 256;
 constexpr int kMaxBins = 2048;
 constexpr size_t kWsHistBytes = 3 * kMaxBins * sizeof(uint32_t);  // one histogram per pass
 
-inline size_t prune_workspace_bytes(int64_t n) {
+constexpr size_t prune_workspace_bytes(int64_t n) {
   const int64_t tiles = (n + kTileElems - 1) / kTileElems;
   size_t b = kWsStateBytes + kWsHistBytes + static_cast<size_t>(tiles) * 8;
   return (b + 255) & ~static_cast<size_t>(255);

@@ -1,4 +1,4 @@
-// fp32 CUDA-core path of surgeon_weight_grad (Algorithm 1 lines 11-12, Eq. 2).
+// fp32 CUDA-core path of surgeon_weight_grad (Algorithm 1: Reshape and gradient steps, Eq. 2).
 //
 // Implicit GEMM  dW[m, nn] = sum_k G[k, m] * Acol[k, nn]  with m = output channel,
 // nn = (c, r, s) and k = (b, y, x) (or the row t of a linear layer).  The im2col operand is

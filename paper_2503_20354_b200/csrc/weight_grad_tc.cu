@@ -1,4 +1,4 @@
-// Tensor-core path of surgeon_weight_grad (Algorithm 1 lines 11-12, Eq. 2) for sm_100a.
+// Tensor-core path of surgeon_weight_grad (Algorithm 1: Reshape and gradient steps, Eq. 2) for sm_100a.
 //
 // Implicit GEMM on tcgen05:  D[nn, o] = sum_k Acol[nn, k] * G[o, k]
 //   nn = (c, r, s)  im2col column of the activation  -> MMA M (128 rows per CTA tile, TMEM lanes)
@@ -9,7 +9,7 @@
 //
 // Nothing dense comes from HBM: producer warps read the bitmap, the block offsets and the packed
 // values, rebuild the rows of the pruned activation a K-tile needs in a shared-memory patch
-// (Algorithm 1 line 11, "Reshape"), and write the im2col view of that patch into the operand
+// (Algorithm 1: Reshape step, "Reshape"), and write the im2col view of that patch into the operand
 // tile.  The same warps convert the fp32 output gradient to bf16 on the way into its tile.  One
 // elected thread issues the MMAs; tcgen05.commit hands stages back to the producers.
 // The reduction is split over CTAs in contiguous K ranges; partial tiles go to scratch and are
@@ -59,7 +59,7 @@ __device__ __forceinline__ void producer_sync() {
 }
 
 // ---- decompression of one contiguous flat range into shared memory (one warp) ---------------
-// dst[i] = bf16 of the pruned activation at flat index start + i, i < len  (Algorithm 1 line 11).
+// dst[i] = bf16 of the pruned activation at flat index start + i, i < len  (Algorithm 1: Reshape step).
 template <int DT>
 __device__ __forceinline__ void decompress_range(const uint32_t* __restrict__ bitmap,
                                                  const void* __restrict__ values,

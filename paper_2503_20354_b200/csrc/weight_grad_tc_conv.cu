@@ -1,6 +1,6 @@
 // Fast tensor-core weight-gradient kernel for 3x3 / pad 1 ("patch" mode) and 1x1 / pad 0
 // ("direct" mode) convolutions of stride 1 or 2 whose rows are a multiple of 8 (stride 1) or
-// 16 (stride 2) elements wide.  Algorithm 1 lines 11-12 with Eq. 2; same GEMM view as
+// 16 (stride 2) elements wide.  Algorithm 1: Reshape and gradient steps with Eq. 2; same GEMM view as
 // weight_grad_tc.cu:  D[nn, o] = sum_k Acol[nn, k] * G[o, k],  nn = (c, r, s),  k = (b, y, x).
 //
 // What differs from the general kernel:

@@ -1,4 +1,4 @@
-"""Pins for the oracle's weight gradient (Eq. 2; Algorithm 1 lines 11-12).
+"""Pins for the oracle's weight gradient (Eq. 2; Algorithm 1: Reshape and gradient steps).
 
 Independent references: PyTorch's fp64 autograd through conv2d / matmul (a library routine, not
 the oracle's loops), finite differences of a scalar loss, the 1x1-conv == linear identity,

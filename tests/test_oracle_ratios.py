@@ -1,4 +1,4 @@
-"""Pins for the oracle's per-layer ratio rule (Eq. 5-7) and kept count (Algorithm 1 line 6).
+"""Pins for the oracle's per-layer ratio rule (Eq. 5-7) and kept count (Algorithm 1: prune step).
 
 The expected values come from hand-worked fixtures, from a closed form that follows from the
 equations (the two inner normalisations cancel: p_i = 1 - M_i G_i / max_j M_j G_j), and from

@@ -1,4 +1,4 @@
-"""Pins for the oracle's magnitude top-k selection and compressed store (Algorithm 1 lines 6-7, 11).
+"""Pins for the oracle's magnitude top-k selection and compressed store (Algorithm 1: prune, decompose and Reshape steps).
 
 Brute force in pure Python on tiny tensors, invariants that fix the result uniquely, the
 round trip at ratio 0, and special values.  Both selection routes (full stable sort and
