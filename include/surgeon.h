@@ -125,6 +125,32 @@ surgeon_status surgeon_prune_compact(const void* x, int64_t n, surgeon_dtype dt,
                                      surgeon_compressed* out, void* workspace,
                                      size_t workspace_bytes, void* cuda_stream);
 
+/* ------------------------------------------------------------------------------------------
+ * No counterpart in the paper: surgeon_prune_compact for callers that cannot allocate device
+ * memory.  A hook that runs while the framework's allocator is locked or its pool is frozen, a
+ * plug-in behind an interface that forbids cudaMalloc, or a process that gave away its whole
+ * memory budget at start-up still owns x and the four output buffers of *out, but has no scratch
+ * to pass as `workspace`.  This variant takes none: the scratch is a fixed array inside the
+ * library (less than 1 MB of global data on every GPU that loads the library, held until the
+ * process exits), so neither the caller nor the library allocates or frees anything.
+ * Same arguments, results, ordering on cuda_stream and error codes as surgeon_prune_compact,
+ * except:
+ *   - n may not exceed SURGEON_STATIC_MAX_N elements; a larger n returns
+ *     SURGEON_ERR_UNSUPPORTED before anything is launched (use surgeon_prune_compact with your
+ *     own workspace for such tensors);
+ *   - the first call on each device looks up the array's device address (one host-side
+ *     runtime query, with that device current).  Make that first call outside any stream
+ *     capture; later calls on the device do no set-up;
+ *   - all calls on one device share the one array.  Each call clears what it needs before use,
+ *     so calls that follow each other on a stream, or are otherwise ordered, are independent;
+ *     two calls whose kernels can run at the same time on one GPU (different streams without an
+ *     event between them) race on the array and give undefined results.
+ * ---------------------------------------------------------------------------------------- */
+#define SURGEON_STATIC_MAX_N (1LL << 22)
+surgeon_status surgeon_prune_compact_static(const void* x, int64_t n, surgeon_dtype dt,
+                                            double ratio, surgeon_compressed* out,
+                                            void* cuda_stream);
+
 /* Layer geometry for the weight gradient.  dilation 1, groups 1. */
 typedef struct surgeon_layer_desc {
   int32_t kind;  /* 0 = linear: activation [batch, c_in] (batch = rows T; h = w = kh = kw = 1,

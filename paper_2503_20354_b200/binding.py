@@ -72,6 +72,9 @@ def lib():
         l.surgeon_prune_compact.restype = C.c_int
         l.surgeon_prune_compact.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_double,
                                             C.POINTER(Compressed), C.c_void_p, C.c_size_t, C.c_void_p]
+        l.surgeon_prune_compact_static.restype = C.c_int
+        l.surgeon_prune_compact_static.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_double,
+                                                   C.POINTER(Compressed), C.c_void_p]
         l.surgeon_weight_grad_workspace.restype = C.c_size_t
         l.surgeon_weight_grad_workspace.argtypes = [C.POINTER(LayerDesc)]
         l.surgeon_weight_grad.restype = C.c_int
@@ -212,6 +215,34 @@ def surgeon_prune_compact(x: torch.Tensor, ratio: float, out: Optional[Compresse
                                      workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                      _stream_ptr(stream))
     _check(st, "surgeon_prune_compact")
+    return out
+
+
+SURGEON_STATIC_MAX_N = 1 << 22
+
+
+def surgeon_prune_compact_static(x: torch.Tensor, ratio: float, out: CompressedActivation,
+                                 stream: Optional[torch.cuda.Stream] = None) -> CompressedActivation:
+    """``surgeon_prune_compact`` without a workspace, for callers that must not allocate device
+    memory (a hook running while the allocator is locked, a frozen memory pool): the scratch is
+    a fixed array inside the library.  ``out`` must already exist and be large enough for this
+    ratio (build it once with ``CompressedActivation(n, dt, 0.0, device)``); this function
+    creates no tensor.  Tensors of more than ``SURGEON_STATIC_MAX_N`` elements are refused.
+    Calls on one GPU share the scratch, so they must not overlap in time."""
+    if not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x must be a contiguous CUDA tensor")
+    dt = dtype_code(x.dtype)
+    n = x.numel()
+    if n > SURGEON_STATIC_MAX_N:
+        raise SurgeonError(SURGEON_ERR_UNSUPPORTED, "surgeon_prune_compact_static: %d elements "
+                           "exceed the built-in scratch (limit %d)" % (n, SURGEON_STATIC_MAX_N))
+    sizes = surgeon_compact_sizes(n, dt, ratio)
+    if out.n != n or out.dt != dt or out.values.numel() < sizes.n_keep:
+        raise ValueError("output store does not fit this tensor / ratio")
+    out.ratio, out.sizes = float(ratio), sizes
+    st = lib().surgeon_prune_compact_static(x.data_ptr(), n, dt, float(ratio), C.byref(out.c),
+                                            _stream_ptr(stream))
+    _check(st, "surgeon_prune_compact_static")
     return out
 
 
