@@ -51,7 +51,7 @@ typedef enum {
 typedef enum { SURGEON_F32 = 0, SURGEON_BF16 = 1 } surgeon_dtype;
 
 /* Elements covered by one entry of surgeon_compressed::block_offsets. */
-#define SURGEON_BLOCK 1024
+#define SURGEON_BLOCK 128
 /* Largest supported element count of one activation tensor (counts are packed in 31 bits). */
 #define SURGEON_MAX_N 2147483647LL
 
@@ -73,8 +73,8 @@ surgeon_status surgeon_layer_ratios(const double* gi, const double* lam, int32_t
  * Algorithm 1: prune step ("prune A_i with ratio p"): the kept count and the buffer sizes.
  * Pure host arithmetic.  n_prune = floor(ratio * n) evaluated in IEEE double, n_keep = n -
  * n_prune.  Any out pointer may be NULL.  bitmap_bytes = 4*ceil(n/32); values_bytes =
- * n_keep*sizeof(dt); offsets_bytes = 8*(ceil(n/SURGEON_BLOCK)+1); workspace_bytes = scratch
- * surgeon_prune_compact needs for this n (independent of ratio).
+ * n_keep*sizeof(dt); offsets_bytes = 4*(ceil(n/SURGEON_BLOCK)+1); workspace_bytes = scratch
+ * surgeon_prune_compact needs for this n and dt (independent of ratio).
  * Errors: INVALID_ARG (n < 0, ratio not in [0,1], bad dt), UNSUPPORTED (n > SURGEON_MAX_N).
  * ---------------------------------------------------------------------------------------- */
 surgeon_status surgeon_compact_sizes(int64_t n, surgeon_dtype dt, double ratio, int64_t* n_keep,
@@ -103,7 +103,7 @@ typedef struct surgeon_compressed {
   uint32_t* bitmap;        /* ceil(n/32) words; bit (j & 31) of word (j >> 5) is 1 iff flat
                               index j is kept; pad bits of the last word are 0                  */
   void* values;            /* n_keep elements of dt in ascending flat index, bit copies of x    */
-  uint64_t* block_offsets; /* ceil(n/SURGEON_BLOCK)+1 entries; entry b = number of kept elements
+  uint32_t* block_offsets; /* ceil(n/SURGEON_BLOCK)+1 entries; entry b = number of kept elements
                               with flat index < b*SURGEON_BLOCK; the last entry = n_keep        */
   surgeon_header* header;  /* 32 bytes                                                          */
 } surgeon_compressed;
@@ -131,7 +131,7 @@ surgeon_status surgeon_prune_compact(const void* x, int64_t n, surgeon_dtype dt,
  * plug-in behind an interface that forbids cudaMalloc, or a process that gave away its whole
  * memory budget at start-up still owns x and the four output buffers of *out, but has no scratch
  * to pass as `workspace`.  This variant takes none: the scratch is a fixed array inside the
- * library (less than 1 MB of global data on every GPU that loads the library, held until the
+ * library (about 2.5 MB of global data on every GPU that loads the library, held until the
  * process exits), so neither the caller nor the library allocates or frees anything.
  * Same arguments, results, ordering on cuda_stream and error codes as surgeon_prune_compact,
  * except:

@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "surgeon_oracle.cpp")
 _LIB = os.path.join(_HERE, "libsurgeon_oracle.so")
 
-BLOCK = 1024  # elements per block-offset entry of the store that is compared with the library's
+BLOCK = 128  # elements per block-offset entry of the store that is compared with the library's
 F32, BF16 = 0, 1
 
 

@@ -26,7 +26,7 @@ SURGEON_ERR_CUDA = 5
 SURGEON_ERR_TIMEOUT = 6
 SURGEON_ERR_INTERNAL = 7
 SURGEON_F32, SURGEON_BF16 = 0, 1
-SURGEON_BLOCK = 1024
+SURGEON_BLOCK = 128
 PATH_TENSOR_CORE, PATH_FP32 = 0, 1
 
 
@@ -165,7 +165,7 @@ class CompressedActivation:
         self.bitmap = torch.empty(max(s.bitmap_bytes // 4, 1), dtype=torch.int32, device=device)
         vt = torch.float32 if dt == SURGEON_F32 else torch.bfloat16
         self.values = torch.empty(max(s.n_keep, 1), dtype=vt, device=device)
-        self.block_offsets = torch.empty(s.offsets_bytes // 8, dtype=torch.int64, device=device)
+        self.block_offsets = torch.empty(s.offsets_bytes // 4, dtype=torch.int32, device=device)
         self.header = torch.zeros(4, dtype=torch.int64, device=device)
         self.c = Compressed(self.n, self.dt, 0, self.bitmap.data_ptr(), self.values.data_ptr(),
                             self.block_offsets.data_ptr(), self.header.data_ptr())
@@ -185,12 +185,12 @@ class CompressedActivation:
         return Header.from_buffer_copy(raw)
 
     def to_numpy(self):
-        """Host copies for comparison: (bitmap uint32, values, offsets uint64, Header)."""
+        """Host copies for comparison: (bitmap uint32, values, offsets uint32, Header)."""
         nw = (self.n + 31) // 32
         bitmap = self.bitmap[:nw].cpu().numpy().view(np.uint32)
         vals = self.values[: self.n_keep].cpu()
         vals = vals.view(torch.int16).numpy().view(np.uint16) if self.dt == SURGEON_BF16 else vals.numpy()
-        offs = self.block_offsets[: self.sizes.offsets_bytes // 8].cpu().numpy().view(np.uint64)
+        offs = self.block_offsets[: self.sizes.offsets_bytes // 4].cpu().numpy().view(np.uint32)
         return bitmap, vals, offs, self.read_header()
 
 

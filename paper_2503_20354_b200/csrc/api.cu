@@ -112,8 +112,8 @@ surgeon_status surgeon_compact_sizes(int64_t n, surgeon_dtype dt, double ratio, 
   if (bitmap_bytes) *bitmap_bytes = static_cast<size_t>((n + 31) / 32) * 4;
   if (values_bytes) *values_bytes = static_cast<size_t>(k) * (dt == SURGEON_F32 ? 4 : 2);
   if (offsets_bytes)
-    *offsets_bytes = static_cast<size_t>((n + SURGEON_BLOCK - 1) / SURGEON_BLOCK + 1) * 8;
-  if (workspace_bytes) *workspace_bytes = prune_workspace_bytes(n);
+    *offsets_bytes = static_cast<size_t>((n + SURGEON_BLOCK - 1) / SURGEON_BLOCK + 1) * 4;
+  if (workspace_bytes) *workspace_bytes = prune_workspace_bytes(n, static_cast<int>(dt));
   return SURGEON_OK;
 }
 
@@ -131,7 +131,7 @@ surgeon_status surgeon_prune_compact(const void* x, int64_t n, surgeon_dtype dt,
   if (!aligned16(x) || !aligned16(out->bitmap) || !aligned16(out->values) ||
       !aligned16(out->block_offsets) || !aligned16(out->header) || !aligned16(workspace))
     return SURGEON_ERR_INVALID_ARG;
-  if (workspace_bytes < prune_workspace_bytes(n)) return SURGEON_ERR_BUFFER_TOO_SMALL;
+  if (workspace_bytes < prune_workspace_bytes(n, static_cast<int>(dt))) return SURGEON_ERR_BUFFER_TOO_SMALL;
   out->n = n;
   out->dt = static_cast<int32_t>(dt);
   out->reserved = 0;

@@ -1,112 +1,456 @@
 // Threshold select and compaction kernels of surgeon_prune_compact, and surgeon_decompress.
 //
-// Algorithm 1: prune step: the kept set of a layer is its n_keep largest-magnitude elements, ties
-// at the threshold broken by lowest flat index.  Its decompose step / Section 4.2: the pruned activation is
-// cached as the vector of kept elements plus one index bit per element.
+// Algorithm 1, prune step: the kept set of a layer is its n_keep largest-magnitude elements, ties
+// at the threshold broken by lowest flat index.  Its decompose step / Section 4.2: the pruned
+// activation is cached as the vector of kept elements plus one index bit per element.
 //
-//   select  : radix select on the magnitude key.  Each pass histograms one digit of the keys
-//             that still match the prefix found so far; the last CTA to finish a pass scans the
-//             histogram from the top and fixes the next digit.  The result (threshold key,
-//             count above it, tie quota) is exact and unique, so it is deterministic whatever
-//             the atomics' order.
-//   compact : one streaming pass.  A warp owns one SURGEON_BLOCK (1024 elements); ballots turn
-//             the per-element decisions directly into bitmap words; an ordered exclusive scan
-//             over tiles (decoupled look-back on one packed 64-bit word per tile) gives every
-//             tile its position in the packed vector and its rank among the ties.
+// The tensor is read twice: once to find the threshold, once to emit the store.  No kernel waits
+// on another CTA: everything the emitting pass needs to place a tile's output (how many elements
+// before the tile are kept, how many ties precede it) is counted during the first read.
+//
+//   sample   : a strided sample (about 1/32 of the tensor) gives a bracket [blo, bhi] of
+//              histogram buckets that contains the threshold with overwhelming probability.
+//   histogram: one streaming read, fed by bulk asynchronous copies into a shared-memory ring.
+//              A 32768-bin shared-memory histogram over the top 15 key bits gives the exact
+//              bucket b1 of the threshold (for bf16 the key has 15 bits, so that is the
+//              threshold itself).  The same read counts, per compaction tile, the keys above the
+//              bracket and the exact zeros, and appends every key inside the bracket, tagged
+//              with its tile, to a candidate list (1-3 % of the elements).
+//   refine   : fp32 only; a 65536-bin histogram over the low 16 bits of the listed keys of
+//              bucket b1 fixes the threshold.
+//   count    : the listed keys above / equal to the threshold are added to the per-tile counts;
+//              the last CTA turns the counts into an exclusive scan over tiles.
+//   compact  : one streaming read with 128-bit loads; a tile's CTA starts from its entry of the
+//              scan, builds bitmap words with warp OR-reductions, stages the kept values in
+//              shared memory and stores them as aligned 16-byte vectors.
+//
+// If the threshold's bucket falls outside the bracket, or the list overflows (massive ties at a
+// non-zero value), refine and count read the tensor once more instead of the list.  The result
+// is exact and unique either way; only the cost differs.
+// Every count fits 32 bits because n <= SURGEON_MAX_N < 2^31.
 #include "surgeon_internal.cuh"
+#include "tc_common.cuh"
 
 namespace surgeon {
 
 namespace {
 
-constexpr int kHistThreads = 512;
+using tc::smem_u32;
 
-template <int DT, int SHIFT, int BITS, bool LAST>
-__global__ void __launch_bounds__(kHistThreads)
-radix_hist_kernel(const void* __restrict__ xv, long long n, long long k_total, int pass,
-                  SelectState* __restrict__ st, uint32_t* __restrict__ ghist,
-                  surgeon_header* __restrict__ hdr) {
-  using E = typename Elem<DT>::type;
+constexpr int kSelThreads = 1024;
+constexpr uint32_t kFull = 0xFFFFFFFFu;
+// Histogram pass: 31 consumer warps read what one producer thread streams into a ring of stages
+// with bulk asynchronous copies; a stage holds one 16-byte vector per consumer thread.
+constexpr int kHistConsumerWarps = 31;
+constexpr int kStageVecs = kHistConsumerWarps * 32;
+constexpr int kStageBytes = kStageVecs * 16;
+constexpr int kHistStages = 3;
+constexpr int kWarpBuf = 192;          // candidate staging entries per warp
+constexpr int kFlushAt = 64;           // a half vector adds at most 128 entries
+constexpr int kHistWords = kBuckets + 32;   // + one private bin per lane that swallows zeros
+constexpr size_t kHistSmem = static_cast<size_t>(kHistWords) * 4 + kHistStages * kStageBytes +
+                             static_cast<size_t>(kHistConsumerWarps) * kWarpBuf * 8;
+static_assert((kHistWords * 4) % 128 == 0, "ring alignment");
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+  return v;
+}
+
+// dst[0 .. kBuckets) = src[0 .. kBuckets) with all loads of a thread in flight together
+// (1024 threads; src is global memory written by other CTAs, dst shared memory).
+__device__ __forceinline__ void load_hist_to_smem(const uint32_t* __restrict__ src, uint32_t* dst) {
+  constexpr int kPer = kBuckets / 4 / kSelThreads;   // 8 vectors per thread
+  uint4 v[kPer];
+#pragma unroll
+  for (int i = 0; i < kPer; ++i)
+    v[i] = __ldcg(reinterpret_cast<const uint4*>(src) + i * kSelThreads + threadIdx.x);
+#pragma unroll
+  for (int i = 0; i < kPer; ++i)
+    reinterpret_cast<uint4*>(dst)[i * kSelThreads + threadIdx.x] = v[i];
+}
+__device__ __forceinline__ void zero_hist_smem(uint32_t* dst) {
+#pragma unroll
+  for (int i = 0; i < kBuckets / 4 / kSelThreads; ++i)
+    reinterpret_cast<uint4*>(dst)[i * kSelThreads + threadIdx.x] = make_uint4(0, 0, 0, 0);
+}
+// Adds the non-zero bins of a CTA's shared-memory histogram to the global one.
+__device__ __forceinline__ void flush_hist(const uint32_t* hist, uint32_t* __restrict__ ghist) {
+#pragma unroll 4
+  for (int i = 0; i < kBuckets / 4 / kSelThreads; ++i) {
+    const int v = i * kSelThreads + threadIdx.x;
+    const uint4 h = reinterpret_cast<const uint4*>(hist)[v];
+    if (h.x) atomicAdd(&ghist[4 * v + 0], h.x);
+    if (h.y) atomicAdd(&ghist[4 * v + 1], h.y);
+    if (h.z) atomicAdd(&ghist[4 * v + 2], h.z);
+    if (h.w) atomicAdd(&ghist[4 * v + 3], h.w);
+  }
+}
+
+// Cooperative search from the top of a histogram of NB bins (NB a multiple of 1024) by a CTA of
+// 1024 threads: finds the bin b with  #(bins above b) < rank <= #(bins >= b)  and writes
+// res[0] = b, res[1] = count in the bins above b.  `ld(i)` returns bin i.  rank >= 1 and the
+// histogram holds at least `rank` entries.  scratch: 32 words of shared memory.
+template <int NB, typename Load>
+__device__ void find_from_top(Load ld, uint32_t rank, uint32_t* scratch, uint32_t* res) {
+  constexpr int PER_WARP = NB / 32;
+  constexpr int PER_LANE = PER_WARP / 32;
+  const int warp = threadIdx.x >> 5;
+  const uint32_t lane = lane_id();
+  // level 1: warp w owns the PER_WARP bins below NB - w*PER_WARP
+  const int top = NB - warp * PER_WARP;   // exclusive upper end
+  uint32_t s = 0;
+#pragma unroll 8
+  for (int i = lane; i < PER_WARP; i += 32) s += ld(top - 1 - i);
+  s = warp_sum(s);
+  if (lane == 0) scratch[warp] = s;
+  __syncthreads();
+  uint32_t acc = 0;
+  int W = 0;
+  for (; W < 31; ++W) {
+    const uint32_t t = scratch[W];
+    if (acc + t >= rank) break;
+    acc += t;
+  }
+  if (warp == W) {
+    // level 2: lane L owns the PER_LANE bins below top - L*PER_LANE
+    const int ltop = top - static_cast<int>(lane) * PER_LANE;
+    uint32_t ls = 0;
+#pragma unroll 8
+    for (int i = 0; i < PER_LANE; ++i) ls += ld(ltop - 1 - ((i + lane) % PER_LANE));
+    const uint32_t excl = warp_excl_scan(ls);
+    const uint32_t want = rank - acc;
+    if (excl < want && want <= excl + ls) {
+      uint32_t a = excl;
+      int b = ltop - 1;
+      for (int i = 0; i < PER_LANE - 1; ++i, --b) {
+        const uint32_t c = ld(b);
+        if (a + c >= want) break;
+        a += c;
+      }
+      res[0] = static_cast<uint32_t>(b);
+      res[1] = acc + a;
+    }
+  }
+  __syncthreads();
+}
+
+__device__ __forceinline__ uint32_t hash_u32(uint32_t v) {
+  v ^= v >> 16; v *= 0x7FEB352Du; v ^= v >> 15; v *= 0x846CA68Bu; v ^= v >> 16;
+  return v;
+}
+
+// ---- bracket of buckets around the threshold, predicted from a strided sample ------------------
+template <int DT>
+__global__ void __launch_bounds__(kSelThreads, 1)
+sample_kernel(const uint4* __restrict__ xq, long long n, uint32_t k, uint32_t n_seg,
+              uint32_t seg_stride, SelectState* __restrict__ st, uint32_t* __restrict__ shist) {
   constexpr uint32_t kMask = Elem<DT>::kKeyMask;
-  constexpr int NB = 1 << BITS;
-  constexpr int HI = SHIFT + BITS;  // bits above this position are the prefix
-  __shared__ uint32_t hist[NB];
+  constexpr int EPV = (DT == 0) ? 4 : 8;
+  extern __shared__ __align__(128) uint32_t hist[];   // kHistWords
+  __shared__ uint32_t scratch[32];
+  __shared__ uint32_t res[2];
   __shared__ bool s_last;
   const int tid = threadIdx.x;
-  for (int i = tid; i < NB; i += kHistThreads) hist[i] = 0;
+  const uint32_t lane = lane_id();
+  zero_hist_smem(hist);
   __syncthreads();
-
-  const uint32_t prefix = st->prefix;
-  const uint32_t want = (HI < 32) ? (prefix >> (HI & 31)) : 0u;
-  uint32_t zero_cnt = 0;  // digit 0 is counted in a register: post-ReLU data is half zeros
-  auto add = [&](uint32_t key) {
-    const uint32_t hi = (HI < 32) ? (key >> (HI & 31)) : 0u;
-    if (hi == want) {
-      const uint32_t d = (key >> SHIFT) & (NB - 1);
-      if (d == 0) ++zero_cnt;
-      else atomicAdd(&hist[d], 1u);
+  uint32_t zero_cnt = 0;
+#pragma unroll 4
+  for (uint32_t seg = blockIdx.x * 32 + (tid >> 5); seg < n_seg; seg += gridDim.x * 32) {
+    // one segment = 32 lanes x 16 bytes, at a hashed position inside its stride
+    const unsigned long long pos =
+        static_cast<unsigned long long>(seg) * seg_stride + hash_u32(seg) % seg_stride;
+    const uint4 q = __ldg(xq + pos * 32 + lane);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) {
+      const uint32_t bits = (DT == 0) ? w[e % 4] : (w[e >> 1] >> (16 * (e & 1)));
+      const uint32_t key = bits & kMask;
+      const bool isz = key == 0;
+      zero_cnt += isz ? 1u : 0u;
+      atomicAdd(&hist[isz ? kBuckets + lane : (DT == 0 ? key >> 16 : key)], 1u);
     }
-  };
-
-  constexpr int VEC = 16 / sizeof(E);
-  const long long nvec = n / VEC;
-  const uint4* __restrict__ xq = reinterpret_cast<const uint4*>(xv);
-  const long long stride = static_cast<long long>(gridDim.x) * kHistThreads;
-  for (long long v = static_cast<long long>(blockIdx.x) * kHistThreads + tid; v < nvec;
-       v += stride) {
-    const uint4 q = __ldg(xq + v);
-    if (DT == 0) {
-      add(q.x & kMask); add(q.y & kMask); add(q.z & kMask); add(q.w & kMask);
-    } else {
-      add(q.x & kMask); add((q.x >> 16) & kMask);
-      add(q.y & kMask); add((q.y >> 16) & kMask);
-      add(q.z & kMask); add((q.z >> 16) & kMask);
-      add(q.w & kMask); add((q.w >> 16) & kMask);
-    }
-  }
-  if (blockIdx.x == 0) {
-    const E* __restrict__ xe = reinterpret_cast<const E*>(xv);
-    for (long long j = nvec * VEC + tid; j < n; j += kHistThreads)
-      add(static_cast<uint32_t>(xe[j]) & kMask);
   }
   zero_cnt = warp_sum(zero_cnt);
-  if (lane_id() == 0 && zero_cnt) atomicAdd(&hist[0], zero_cnt);
+  if (lane == 0 && zero_cnt) atomicAdd(&hist[0], zero_cnt);
   __syncthreads();
-  for (int i = tid; i < NB; i += kHistThreads)
-    if (hist[i]) atomicAdd(&ghist[i], hist[i]);
+  flush_hist(hist, shist);
   __threadfence();
   __syncthreads();
-  if (tid == 0) {
-    const uint32_t t = atomicAdd(&st->pass_ticket[pass], 1u);
-    s_last = (t == gridDim.x - 1);
+  if (tid == 0) s_last = (atomicAdd(&st->ticket_sample, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  load_hist_to_smem(shist, hist);
+  __syncthreads();
+  // rank of the threshold inside the sample, +- 5 standard deviations of a binomial count
+  const double S = static_cast<double>(32 * EPV) * n_seg;
+  const double q = static_cast<double>(k) / static_cast<double>(n);
+  const double r = q * S;
+  const double delta = 5.0 * sqrt(S * q * (1.0 - q)) + 8.0;
+  uint32_t bhi = kBuckets - 1, blo = 0;
+  auto ld = [&](int i) { return hist[i]; };
+  if (r - delta >= 1.0) {
+    find_from_top<kBuckets>(ld, static_cast<uint32_t>(r - delta), scratch, res);
+    bhi = res[0];
+    __syncthreads();
   }
+  if (r + delta <= S - 1.0) {
+    find_from_top<kBuckets>(ld, static_cast<uint32_t>(r + delta) + 1u, scratch, res);
+    blo = res[0];
+  }
+  if (tid == 0) { st->blo = blo; st->bhi = bhi; }
+}
+
+// ---- the select's read of the tensor ---------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(kSelThreads, 1)
+hist_kernel(const void* __restrict__ xv, long long n, uint32_t k, int use_bracket,
+            SelectState* __restrict__ st, uint32_t* __restrict__ ghist,
+            uint32_t* __restrict__ hist2, uint32_t* __restrict__ cnt_gt,
+            uint32_t* __restrict__ cnt_zero, unsigned long long* __restrict__ list,
+            uint32_t list_cap, surgeon_header* __restrict__ hdr) {
+  using E = typename Elem<DT>::type;
+  constexpr uint32_t kMask = Elem<DT>::kKeyMask;
+  constexpr int VEC = 16 / sizeof(E);
+  // dynamic shared memory: hist[kHistWords] | ring[kHistStages][kStageBytes] | wbuf[31][kWarpBuf]
+  extern __shared__ __align__(128) uint32_t hist[];
+  __shared__ __align__(8) unsigned long long bars[2 * kHistStages];
+  __shared__ uint32_t scratch[32];
+  __shared__ uint32_t s_wcnt[32];
+  __shared__ uint32_t res[2];
+  __shared__ bool s_last;
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  const uint32_t lane = lane_id();
+  unsigned char* ring = reinterpret_cast<unsigned char*>(hist + kHistWords);
+  unsigned long long* wbuf =
+      reinterpret_cast<unsigned long long*>(ring + kHistStages * kStageBytes) + warp * kWarpBuf;
+  const uint32_t full_bar = smem_u32(bars);
+  const uint32_t empty_bar = smem_u32(bars + kHistStages);
+  if (tid == 0) {
+    for (int s = 0; s < kHistStages; ++s) {
+      tc::mbar_init(full_bar + 8 * s, 1);
+      tc::mbar_init(empty_bar + 8 * s, kHistConsumerWarps);
+    }
+    tc::fence_barrier_init();
+  }
+  zero_hist_smem(hist);
+  if (lane == 0) s_wcnt[warp] = 0;
+  __syncthreads();
+
+  uint32_t blo = 0, bhi = kBuckets - 1;
+  if (use_bracket) { blo = st->blo; bhi = st->bhi; }
+  const uint32_t span = bhi - blo;
+  uint32_t zero_total = 0;
+
+  // Candidate staging: lanes append through a per-warp cursor in shared memory; the buffer goes
+  // to the global list once it holds kFlushAt entries.
+  auto maybe_flush = [&](uint32_t limit) {
+    __syncwarp();
+    const uint32_t cnt = *reinterpret_cast<volatile uint32_t*>(&s_wcnt[warp]);
+    if (cnt >= limit && cnt > 0) {
+      uint32_t base = 0;
+      if (lane == 0) base = atomicAdd(&st->list_count, cnt);
+      base = __shfl_sync(kFull, base, 0);
+      for (uint32_t i = lane; i < cnt; i += 32) {
+        if (base + i < list_cap) list[base + i] = wbuf[i];
+        else st->list_overflow = 1u;
+      }
+      __syncwarp();
+      if (lane == 0) s_wcnt[warp] = 0;
+      __syncwarp();
+    }
+  };
+  uint32_t above_v = 0, zero_v = 0;   // per vector and lane: keys above the bracket, exact zeros
+  unsigned long long tile_tag = 0;    // tile index << 32
+  auto add = [&](uint32_t bits) {
+    const uint32_t key = bits & kMask;
+    const uint32_t bucket = (DT == 0) ? (key >> 16) : key;
+    const bool isz = key == 0;
+    zero_v += isz ? 1u : 0u;
+    above_v += (bucket > bhi) ? 1u : 0u;
+    // zeros (half of post-ReLU data) go to a bin private to the lane: no conflicts, no branch
+    atomicAdd(&hist[isz ? kBuckets + lane : bucket], 1u);
+    if (!isz && (bucket - blo) <= span) wbuf[atomicAdd(&s_wcnt[warp], 1u)] = tile_tag | key;
+  };
+  auto add_vec = [&](const uint4& q) {
+    if (DT == 0) {
+      add(q.x); add(q.y); add(q.z); add(q.w);
+    } else {
+      add(q.x); add(q.x >> 16); add(q.y); add(q.y >> 16);
+    }
+  };
+  auto add_vec_hi = [&](const uint4& q) {   // bf16: second half of the vector
+    add(q.z); add(q.z >> 16); add(q.w); add(q.w >> 16);
+  };
+  // Per-tile counters of one warp step (all 32 lanes hold elements of the same tile).
+  auto tile_counts = [&](uint32_t tile) {
+    const uint32_t a = __reduce_add_sync(kFull, above_v);
+    const uint32_t z = __reduce_add_sync(kFull, zero_v);
+    if (lane == 0) {
+      if (a) atomicAdd(&cnt_gt[tile], a);
+      if (z) atomicAdd(&cnt_zero[tile], z);
+    }
+    zero_total += zero_v;
+    above_v = 0;
+    zero_v = 0;
+  };
+
+  // Chunks of kStageVecs vectors, handed out from the END of the tensor towards its start: what
+  // this pass leaves in L2 is then the part the compaction pass reads first.
+  const long long nvec = n / VEC;
+  const uint4* __restrict__ xq = reinterpret_cast<const uint4*>(xv);
+  const long long n_chunks = (nvec + kStageVecs - 1) / kStageVecs;
+  const long long first_chunk = n_chunks - 1 - blockIdx.x;
+  const int n_it = first_chunk < 0 ? 0 : static_cast<int>(first_chunk / gridDim.x) + 1;
+  bool timed_out = false;
+  if (warp == kHistConsumerWarps) {
+    // ---- producer: one thread keeps the ring full ----
+    if (lane == 0) {
+      for (int it = 0; it < n_it; ++it) {
+        const int s = it % kHistStages;
+        if (it >= kHistStages &&
+            !tc::mbar_wait(empty_bar + 8 * s, ((it / kHistStages) - 1) & 1, 20)) {
+          timed_out = true;
+          break;
+        }
+        const long long v0 = (first_chunk - static_cast<long long>(it) * gridDim.x) * kStageVecs;
+        const long long left = nvec - v0;
+        const uint32_t bytes = static_cast<uint32_t>(left < kStageVecs ? left : kStageVecs) * 16u;
+        tc::mbar_arrive_expect_tx(full_bar + 8 * s, bytes);
+        tc::bulk_load(smem_u32(ring + s * kStageBytes), xq + v0, bytes, full_bar + 8 * s);
+      }
+    }
+  } else {
+    // ---- consumers ----
+    for (int it = 0; it < n_it; ++it) {
+      const int s = it % kHistStages;
+      if (!tc::mbar_wait(full_bar + 8 * s, (it / kHistStages) & 1, 20)) { timed_out = true; break; }
+      const long long vw = (first_chunk - static_cast<long long>(it) * gridDim.x) * kStageVecs +
+                           warp * 32;                     // first vector of this warp's step
+      const bool valid = vw + lane < nvec;
+      uint4 q = make_uint4(0, 0, 0, 0);
+      if (valid) q = reinterpret_cast<const uint4*>(ring + s * kStageBytes)[warp * 32 + lane];
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(empty_bar + 8 * s);
+      const uint32_t tile = static_cast<uint32_t>(vw / kTileVecs);
+      tile_tag = static_cast<unsigned long long>(tile) << 32;
+      if (valid) add_vec(q);
+      if (DT == 1) {
+        maybe_flush(kFlushAt);
+        if (valid) add_vec_hi(q);
+      }
+      tile_counts(tile);
+      maybe_flush(kFlushAt);
+    }
+    if (blockIdx.x == 0 && warp == 0) {   // elements past the last full vector
+      const E* __restrict__ xe = reinterpret_cast<const E*>(xv);
+      const uint32_t tile = static_cast<uint32_t>(nvec / kTileVecs);
+      tile_tag = static_cast<unsigned long long>(tile) << 32;
+      const long long j = nvec * VEC + lane;
+      if (j < n) add(static_cast<uint32_t>(xe[j]));
+      tile_counts(tile);
+    }
+    maybe_flush(1);
+    zero_total = warp_sum(zero_total);
+    if (lane == 0 && zero_total) {
+      atomicAdd(&hist[0], zero_total);
+      atomicAdd(&st->zero_count, zero_total);
+    }
+  }
+  if (timed_out) atomicMax(&st->error, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+  __syncthreads();
+  flush_hist(hist, ghist);
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&st->ticket_hist, 1u) == gridDim.x - 1);
   __syncthreads();
   if (!s_last) return;
 
-  // Last CTA of the pass: every other CTA's histogram is in ghist.
+  // Last CTA: the complete histogram is in ghist.
   __threadfence();
-  for (int i = tid; i < NB; i += kHistThreads) hist[i] = __ldcg(ghist + i);
+  load_hist_to_smem(ghist, hist);
   __syncthreads();
+  find_from_top<kBuckets>([&](int i) { return hist[i]; }, k, scratch, res);
   if (tid == 0) {
-    const long long kr = (pass == 0) ? k_total : st->k_remaining;
-    long long above = 0;
-    int b = NB - 1;
-    for (; b > 0; --b) {
-      const long long c = hist[b];
-      if (above + c >= kr) break;
-      above += c;
+    const uint32_t b = res[0], above = res[1];
+    const bool overflow = __ldcg(&st->list_overflow) != 0;
+    const bool inside = b >= blo && b <= bhi;
+    st->b1 = b;
+    st->k1 = k - above;
+    st->above = above;
+    st->mode = (!overflow && inside) ? 0u : 1u;
+    if (DT == 1) {
+      hdr->threshold_key = b;
+      hdr->status = __ldcg(&st->error);
+      hdr->n_keep = k;
+      hdr->n_greater = above;
+      hdr->tie_quota = static_cast<long long>(k) - above;
+    } else if (b == 0) {
+      // exact zeros are never listed or re-read: they enter the refinement here
+      hist2[0] = __ldcg(&st->zero_count);
     }
-    const uint32_t new_prefix = prefix | (static_cast<uint32_t>(b) << SHIFT);
-    const long long ng = ((pass == 0) ? 0 : st->n_greater) + above;
-    st->prefix = new_prefix;
-    st->k_remaining = kr - above;
-    st->n_greater = ng;
-    if (LAST) {
-      hdr->threshold_key = new_prefix;
-      hdr->n_keep = k_total;
-      hdr->n_greater = ng;
-      hdr->tie_quota = k_total - ng;
+    __threadfence();
+  }
+}
+
+// ---- fp32: low 16 key bits of the elements in bucket b1 ---------------------------------------
+__global__ void __launch_bounds__(kSelThreads)
+refine_kernel(const uint4* __restrict__ xq, long long n, uint32_t k, SelectState* __restrict__ st,
+              uint32_t* __restrict__ hist2, const unsigned long long* __restrict__ list,
+              uint32_t list_cap, surgeon_header* __restrict__ hdr) {
+  __shared__ uint32_t scratch[32];
+  __shared__ uint32_t res[2];
+  __shared__ bool s_last;
+  const int tid = threadIdx.x;
+  const uint32_t lane = lane_id();
+  const uint32_t b1 = st->b1;
+  const uint32_t mode = st->mode;
+  uint32_t round_cnt = 0;   // keys at the bottom of the bucket (low bits 0): round values tie a lot
+  auto add = [&](uint32_t key) {
+    if (key != 0 && (key >> 16) == b1) {
+      const uint32_t low = key & 0xFFFFu;
+      if (low == 0) ++round_cnt;
+      else atomicAdd(&hist2[low], 1u);
     }
+  };
+  const long long gtid = static_cast<long long>(blockIdx.x) * kSelThreads + tid;
+  const long long gsz = static_cast<long long>(gridDim.x) * kSelThreads;
+  if (mode == 0) {
+    uint32_t cnt = st->list_count;
+    if (cnt > list_cap) cnt = list_cap;
+    for (long long i = gtid; i < cnt; i += gsz) add(static_cast<uint32_t>(__ldg(list + i)));
+  } else {
+    const long long nvec = n / 4;
+    for (long long v = gtid; v < nvec; v += gsz) {
+      const uint4 q = __ldg(xq + v);
+      add(q.x & 0x7FFFFFFFu); add(q.y & 0x7FFFFFFFu); add(q.z & 0x7FFFFFFFu); add(q.w & 0x7FFFFFFFu);
+    }
+    if (blockIdx.x == 0) {
+      const uint32_t* xe = reinterpret_cast<const uint32_t*>(xq);
+      for (long long j = nvec * 4 + tid; j < n; j += kSelThreads) add(xe[j] & 0x7FFFFFFFu);
+    }
+  }
+  round_cnt = warp_sum(round_cnt);
+  if (lane == 0 && round_cnt) atomicAdd(&hist2[0], round_cnt);
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&st->ticket_refine, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const uint32_t k1 = st->k1;
+  find_from_top<kLowBins>([&](int i) { return __ldcg(hist2 + i); }, k1, scratch, res);
+  if (tid == 0) {
+    const uint32_t ng = st->above + res[1];
+    hdr->threshold_key = (b1 << 16) | res[0];
+    hdr->status = __ldcg(&st->error);
+    hdr->n_keep = k;
+    hdr->n_greater = ng;
+    hdr->tie_quota = static_cast<long long>(k) - ng;
     __threadfence();
   }
 }
@@ -114,22 +458,149 @@ radix_hist_kernel(const void* __restrict__ xv, long long n, long long k_total, i
 // n_keep == 0 (ratio 1, or an empty tensor): nothing to select.
 __global__ void header_empty_kernel(surgeon_header* hdr, uint32_t sentinel) {
   hdr->threshold_key = sentinel;
+  hdr->status = SURGEON_OK;
   hdr->n_keep = 0;
   hdr->n_greater = 0;
   hdr->tie_quota = 0;
 }
 
+// ---- per-tile counts -> exclusive scan over tiles -------------------------------------------
+// prefix[t] = (keys above the threshold before tile t) << 31 | (keys equal to it before tile t).
+template <int DT>
+__global__ void __launch_bounds__(kSelThreads)
+count_kernel(const void* __restrict__ xv, long long n, SelectState* __restrict__ st,
+             surgeon_header* __restrict__ hdr, const unsigned long long* __restrict__ list,
+             uint32_t list_cap, uint32_t* __restrict__ cnt_gt, uint32_t* __restrict__ cnt_eq,
+             const uint32_t* __restrict__ cnt_zero, uint32_t* __restrict__ full_gt,
+             uint32_t* __restrict__ full_eq, unsigned long long* __restrict__ prefix, int tiles) {
+  using E = typename Elem<DT>::type;
+  constexpr uint32_t kMask = Elem<DT>::kKeyMask;
+  constexpr int EPV = 16 / sizeof(E);
+  __shared__ unsigned long long s_tot[32];
+  __shared__ bool s_last;
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  const uint32_t lane = lane_id();
+  const uint32_t tau = hdr->threshold_key;
+  const uint32_t mode = st->mode;
+  if (mode == 0) {
+    // listed keys: runs of entries share a tile, so a warp usually issues one atomic per count
+    uint32_t cnt = st->list_count;
+    if (cnt > list_cap) cnt = list_cap;
+    const long long rounded = (static_cast<long long>(cnt) + 31) & ~31LL;
+    for (long long i = static_cast<long long>(blockIdx.x) * kSelThreads + tid; i < rounded;
+         i += static_cast<long long>(gridDim.x) * kSelThreads) {
+      const bool valid = i < cnt;
+      const unsigned long long e = valid ? __ldg(list + i) : 0ull;
+      const uint32_t tile = static_cast<uint32_t>(e >> 32);
+      const uint32_t key = static_cast<uint32_t>(e);
+      const bool gt = valid && key > tau;
+      const bool eq = valid && key == tau;
+      const uint32_t t0 = __shfl_sync(kFull, tile, 0);
+      if (__all_sync(kFull, !valid || tile == t0)) {
+        const uint32_t g = __popc(__ballot_sync(kFull, gt));
+        const uint32_t q = __popc(__ballot_sync(kFull, eq));
+        if (lane == 0) {
+          if (g) atomicAdd(&cnt_gt[t0], g);
+          if (q) atomicAdd(&cnt_eq[t0], q);
+        }
+      } else {
+        if (gt) atomicAdd(&cnt_gt[tile], 1u);
+        if (eq) atomicAdd(&cnt_eq[tile], 1u);
+      }
+    }
+  } else {
+    // the list is unusable: count every tile from the tensor itself (one vector per thread)
+    const E* __restrict__ x = reinterpret_cast<const E*>(xv);
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x) {
+      const long long base = (static_cast<long long>(t) * kTileVecs + tid) * EPV;
+      uint32_t g = 0, q = 0;
+      if (base + EPV <= n) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + base));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) {
+          const uint32_t key = ((DT == 0) ? w[i % 4] : (w[i >> 1] >> (16 * (i & 1)))) & kMask;
+          g += key > tau ? 1u : 0u;
+          q += key == tau ? 1u : 0u;
+        }
+      } else {
+        for (int i = 0; i < EPV; ++i) {
+          if (base + i < n) {
+            const uint32_t key = static_cast<uint32_t>(x[base + i]) & kMask;
+            g += key > tau ? 1u : 0u;
+            q += key == tau ? 1u : 0u;
+          }
+        }
+      }
+      g = __reduce_add_sync(kFull, g);
+      q = __reduce_add_sync(kFull, q);
+      if (lane == 0) {
+        if (g) atomicAdd(&full_gt[t], g);
+        if (q) atomicAdd(&full_eq[t], q);
+      }
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&st->ticket_count, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+
+  // Last CTA: exclusive scan.  Warp w owns a contiguous range of tiles.
+  auto value = [&](int t) -> unsigned long long {
+    unsigned long long g, q;
+    if (mode == 0) {
+      g = __ldcg(cnt_gt + t);
+      q = __ldcg(cnt_eq + t) + (tau == 0 ? __ldcg(cnt_zero + t) : 0u);
+    } else {
+      g = __ldcg(full_gt + t);
+      q = __ldcg(full_eq + t);
+    }
+    return (g << 31) | q;
+  };
+  const int chunk = ((tiles + 31) / 32 + 31) & ~31;
+  const int begin = warp * chunk < tiles ? warp * chunk : tiles;
+  const int end = begin + chunk < tiles ? begin + chunk : tiles;
+  unsigned long long acc = 0;
+#pragma unroll 4
+  for (int t = begin + lane; t < end; t += 32) acc += value(t);
+  acc = warp_sum_u64(acc);
+  if (lane == 0) s_tot[warp] = acc;
+  __syncthreads();
+  unsigned long long carry = 0, total = 0;
+  for (int w = 0; w < 32; ++w) {
+    if (w < warp) carry += s_tot[w];
+    total += s_tot[w];
+  }
+  for (int t0 = begin; t0 < end; t0 += 32) {
+    const int t = t0 + lane;
+    const unsigned long long v = t < end ? value(t) : 0ull;
+    unsigned long long incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long up = __shfl_up_sync(kFull, incl, o);
+      if (lane >= static_cast<uint32_t>(o)) incl += up;
+    }
+    if (t < end) prefix[t] = carry + incl - v;
+    carry += __shfl_sync(kFull, incl, 31);
+  }
+  if (tid == 0) {
+    // self-check: the counts must add up to what the select found
+    const long long gt_all = static_cast<long long>(total >> 31);
+    const long long eq_all = static_cast<long long>(total & 0x7FFFFFFFull);
+    if (gt_all != hdr->n_greater || eq_all < hdr->tie_quota)
+      atomicMax(&hdr->status, static_cast<uint32_t>(SURGEON_ERR_INTERNAL));
+  }
+}
+
 // ---- compaction -----------------------------------------------------------------------------
 
-constexpr unsigned long long kStAggregate = 1ull << 62;
-constexpr unsigned long long kStPrefix = 2ull << 62;
 constexpr unsigned long long kCountMask = 0x7FFFFFFFull;
-constexpr uint32_t kSpinCap = 1u << 22;  // bounded look-back wait (each poll sleeps ~50 ns)
-
-__device__ __forceinline__ unsigned long long pack_counts(unsigned long long gt,
-                                                          unsigned long long eq) {
-  return (gt << 31) | eq;
-}
+constexpr int kCompactThreads = 256;
+constexpr int kRows = 4;                 // rows of 32 lanes x 16 bytes per warp
+static_assert(8 * kRows * 32 == kTileVecs, "compaction tile");
 
 // Keep only the lowest `allowed` set bits of `m`.
 __device__ __forceinline__ uint32_t lowest_set_bits(uint32_t m, long long allowed) {
@@ -142,162 +613,233 @@ __device__ __forceinline__ uint32_t lowest_set_bits(uint32_t m, long long allowe
   return m;
 }
 
+// One CTA per tile; nothing is exchanged between CTAs.
 template <int DT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kCompactThreads)
 compact_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restrict__ hdr,
                uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
-               unsigned long long* __restrict__ offsets, uint32_t* __restrict__ ticket,
-               unsigned long long* __restrict__ tile_state, int num_tiles) {
+               uint32_t* __restrict__ offsets, const unsigned long long* __restrict__ prefix) {
   using E = typename Elem<DT>::type;
   constexpr uint32_t kMask = Elem<DT>::kKeyMask;
+  constexpr int EPV = 16 / sizeof(E);          // elements per lane and row: 4 (fp32) / 8 (bf16)
+  constexpr int ROW = 32 * EPV;                // elements per row: 128 / 256
+  constexpr int WPR = ROW / 32;                // bitmap words per row: 4 / 8
+  constexpr int LPW = 32 / EPV;                // lanes per bitmap word: 8 / 4
+  constexpr int BPR = ROW / SURGEON_BLOCK;     // offset blocks per row: 1 / 2
+  constexpr int TILE = 8 * kRows * ROW;
+  constexpr uint32_t kEMask = (1u << EPV) - 1u;
   const E* __restrict__ x = reinterpret_cast<const E*>(xv);
   E* __restrict__ values = reinterpret_cast<E*>(values_v);
-  __shared__ uint32_t s_gt[kTileBlocks], s_eq[kTileBlocks];
-  __shared__ int s_tile;
-  __shared__ unsigned long long s_excl;
+  __shared__ __align__(16) E stage[TILE + EPV];   // kept values of the tile, aligned like the output
+  __shared__ uint32_t s_gt[8], s_eq[8];
 
-  const uint32_t tau = hdr->threshold_key;
-  const long long quota = hdr->tie_quota;
   const int tid = threadIdx.x;
   const uint32_t lane = lane_id();
   const int warp = tid >> 5;
-  const long long n_blocks = (n + SURGEON_BLOCK - 1) / SURGEON_BLOCK;
+  const int tile = blockIdx.x;
+  const long long n_blocks = (n + SURGEON_BLOCK - 1) >> kBlockShift;
   const long long n_words = (n + 31) / 32;
+  const int my_word = lane / LPW;
+  const int my_shift = EPV * (lane % LPW);
 
-  while (true) {
-    if (tid == 0) s_tile = static_cast<int>(atomicAdd(ticket, 1u));
-    __syncthreads();
-    const int tile = s_tile;
-    if (tile >= num_tiles) break;
-
-    const long long block = static_cast<long long>(tile) * kTileBlocks + warp;
-    const long long base = block * SURGEON_BLOCK;
-    E xs[32];
-    uint32_t gt_word = 0, eq_word = 0;  // lane i ends up holding the masks of word i
-    if (base < n) {
+  // ---- load kRows rows; the header and the tile's scan entry travel alongside ----
+  const long long row0 = (static_cast<long long>(tile) * 8 + warp) * kRows;
+  uint4 q[kRows];
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const long long idx = base + i * 32 + lane;
-        xs[i] = (idx < n) ? x[idx] : static_cast<E>(0);
-      }
+  for (int r = 0; r < kRows; ++r) {
+    const long long base = (row0 + r) * ROW + static_cast<long long>(lane) * EPV;
+    if (base + EPV <= n) {
+      q[r] = __ldg(reinterpret_cast<const uint4*>(x + base));
+    } else {
+      uint32_t t[8];
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const long long idx = base + i * 32 + lane;
-        const uint32_t key = static_cast<uint32_t>(xs[i]) & kMask;
-        const bool valid = idx < n;
-        const uint32_t g = __ballot_sync(0xFFFFFFFFu, valid && key > tau);
-        const uint32_t e = __ballot_sync(0xFFFFFFFFu, valid && key == tau);
-        if (lane == static_cast<uint32_t>(i)) { gt_word = g; eq_word = e; }
-      }
+      for (int i = 0; i < 8; ++i)
+        t[i] = (i < EPV && base + i < n) ? static_cast<uint32_t>(x[base + i]) : 0u;
+      if (DT == 0) q[r] = make_uint4(t[0], t[1], t[2], t[3]);
+      else q[r] = make_uint4(t[0] | (t[1] << 16), t[2] | (t[3] << 16), t[4] | (t[5] << 16),
+                             t[6] | (t[7] << 16));
     }
-    const uint32_t gt_warp = warp_sum(__popc(gt_word));
-    const uint32_t eq_warp = warp_sum(__popc(eq_word));
-    if (lane == 0) { s_gt[warp] = gt_warp; s_eq[warp] = eq_warp; }
-    __syncthreads();
+  }
+  const uint32_t tau = hdr->threshold_key;
+  const long long quota = hdr->tie_quota;
+  const unsigned long long excl = prefix[tile];
 
-    if (tid == 0) {
-      unsigned long long gt_tile = 0, eq_tile = 0;
+  // ---- per row and lane EPV decisions "above tau" and "equal to tau" ----
+  uint32_t g_all = 0, e_all = 0;      // kRows fields of EPV bits
 #pragma unroll
-      for (int w = 0; w < kTileBlocks; ++w) { gt_tile += s_gt[w]; eq_tile += s_eq[w]; }
-      const unsigned long long mine = pack_counts(gt_tile, eq_tile);
-      volatile unsigned long long* vs = tile_state;
-      unsigned long long excl = 0;
-      if (tile == 0) {
-        vs[0] = kStPrefix | mine;
+  for (int r = 0; r < kRows; ++r) {
+    const long long base = (row0 + r) * ROW + static_cast<long long>(lane) * EPV;
+    const uint32_t w[4] = {q[r].x, q[r].y, q[r].z, q[r].w};
+    uint32_t g = 0, e = 0;
+#pragma unroll
+    for (int i = 0; i < EPV; ++i) {
+      const uint32_t bits = (DT == 0) ? w[i % 4] : (w[i >> 1] >> (16 * (i & 1)));
+      const uint32_t key = bits & kMask;
+      const bool valid = base + i < n;
+      g |= (valid && key > tau) ? (1u << i) : 0u;
+      e |= (valid && key == tau) ? (1u << i) : 0u;
+    }
+    g_all |= g << (EPV * r);
+    e_all |= e << (EPV * r);
+  }
+  const uint32_t gt_warp = __reduce_add_sync(kFull, __popc(g_all));
+  const uint32_t eq_warp = __reduce_add_sync(kFull, __popc(e_all));
+  if (lane == 0) { s_gt[warp] = gt_warp; s_eq[warp] = eq_warp; }
+  __syncthreads();
+
+  const long long gt_tile_before = static_cast<long long>(excl >> 31);
+  const long long eq_tile_before = static_cast<long long>(excl & kCountMask);
+  long long gt_before = gt_tile_before, eq_before = eq_tile_before;
+  long long gt_all = gt_tile_before, eq_all = eq_tile_before;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) {
+    if (w < warp) { gt_before += s_gt[w]; eq_before += s_eq[w]; }
+    gt_all += s_gt[w]; eq_all += s_eq[w];
+  }
+  // kept before = all greater + the ties that fit the quota
+  const long long tile_kept_before = gt_tile_before + (eq_tile_before < quota ? eq_tile_before : quota);
+  const long long tile_kept_end = gt_all + (eq_all < quota ? eq_all : quota);
+  long long kept_before = gt_before + (eq_before < quota ? eq_before : quota);
+  // 0: no tie of this warp is kept, 1: all are, 2: the quota ends inside these rows
+  const int tie_mode = (eq_before >= quota) ? 0 : (eq_before + eq_warp <= quota ? 1 : 2);
+  // the stage mirrors the 16-byte alignment of the tile's range in the packed vector
+  const int align = static_cast<int>(tile_kept_before % EPV);
+  const long long stage_origin = tile_kept_before - align;   // packed index of stage[0]
+
+  uint32_t my_words[WPR];      // lane r keeps the bitmap words of row r
+  uint32_t my_off[BPR];        // and the offsets of its blocks
+  uint32_t my_cnt[BPR];
+#pragma unroll
+  for (int j = 0; j < WPR; ++j) my_words[j] = 0;
+#pragma unroll
+  for (int j = 0; j < BPR; ++j) { my_off[j] = 0; my_cnt[j] = 0; }
+
+  if (row0 * ROW < n) {
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+      const uint32_t g = (g_all >> (EPV * r)) & kEMask;
+      const uint32_t e = (e_all >> (EPV * r)) & kEMask;
+      uint32_t keep = g;
+      if (tie_mode == 1) {
+        keep |= e;
+      } else if (tie_mode == 2) {
+        const uint32_t ec = __popc(e);
+        const uint32_t before = warp_excl_scan(ec);      // ties of this row in lower lanes
+        keep |= lowest_set_bits(e, quota - eq_before - before);
+        eq_before += warp_sum(ec);
+      }
+      // bitmap words of the row, known to every lane
+      const uint32_t shifted = keep << my_shift;
+      uint32_t words[WPR];
+#pragma unroll
+      for (int j = 0; j < WPR; ++j)
+        words[j] = __reduce_or_sync(kFull, my_word == j ? shifted : 0u);
+      uint32_t pre = 0, total = 0, half = 0;
+#pragma unroll
+      for (int j = 0; j < WPR; ++j) {
+        const uint32_t pc = __popc(words[j]);
+        if (j < my_word) pre += pc;
+        if (j == my_word) pre += __popc(words[j] & ((1u << my_shift) - 1u));
+        if (j < WPR / 2) half += pc;
+        total += pc;
+      }
+      if (static_cast<int>(lane) == r) {
+#pragma unroll
+        for (int j = 0; j < WPR; ++j) my_words[j] = words[j];
+        my_off[0] = static_cast<uint32_t>(kept_before);
+        if (BPR == 2) {
+          my_off[BPR - 1] = static_cast<uint32_t>(kept_before) + half;
+          my_cnt[0] = half;
+          my_cnt[BPR - 1] = total - half;
+        } else {
+          my_cnt[0] = total;
+        }
+      }
+      // kept values into the stage, in packed order
+      int dst = static_cast<int>(kept_before - stage_origin) + static_cast<int>(pre);
+      const uint32_t w[4] = {q[r].x, q[r].y, q[r].z, q[r].w};
+#pragma unroll
+      for (int i = 0; i < EPV; ++i) {
+        if ((keep >> i) & 1u) {
+          stage[dst++] = (DT == 0) ? static_cast<E>(w[i % 4])
+                                   : static_cast<E>((w[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
+        }
+      }
+      kept_before += total;
+    }
+    // lanes 0..kRows-1 store the words and offsets of their rows: contiguous 16-byte pieces
+    if (lane < kRows) {
+      const long long row = row0 + lane;
+      const long long w0 = row * WPR;
+      if (w0 + WPR <= n_words) {
+#pragma unroll
+        for (int j = 0; j < WPR; j += 4)
+          *reinterpret_cast<uint4*>(bitmap + w0 + j) =
+              make_uint4(my_words[j], my_words[j + 1], my_words[j + 2], my_words[j + 3]);
       } else {
-        vs[tile] = kStAggregate | mine;
-        int p = tile - 1;
-        while (true) {
-          unsigned long long v = vs[p];
-          uint32_t spins = 0;
-          while ((v >> 62) == 0 && spins < kSpinCap) {
-            __nanosleep(50);
-            v = vs[p];
-            ++spins;
-          }
-          if ((v >> 62) == 0) {  // gave up: report, stop waiting, let successors pass
-            atomicMax(&hdr->status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
-            break;
-          }
-          excl += v & ~(3ull << 62);
-          if ((v >> 62) == 2 || p == 0) break;
-          --p;
-        }
-        vs[tile] = kStPrefix | (excl + mine);
-      }
-      s_excl = excl;
-    }
-    __syncthreads();
-
-    const unsigned long long excl = s_excl;
-    long long gt_before = static_cast<long long>(excl >> 31);
-    long long eq_before = static_cast<long long>(excl & kCountMask);
 #pragma unroll
-    for (int w = 0; w < kTileBlocks; ++w) {
-      if (w < warp) { gt_before += s_gt[w]; eq_before += s_eq[w]; }
-    }
-    // kept before this warp's block = all greater + the ties that fit the quota
-    const long long kept_before = gt_before + (eq_before < quota ? eq_before : quota);
-
-    if (base < n) {
-      // rank of this word's first tie among all ties of the tensor
-      const long long eq_word_before = eq_before + warp_excl_scan(__popc(eq_word));
-      const uint32_t keep_word = gt_word | lowest_set_bits(eq_word, quota - eq_word_before);
-      const uint32_t kc = __popc(keep_word);
-      const uint32_t word_excl = warp_excl_scan(kc);
-      const uint32_t kept_warp = warp_sum(kc);
-      const long long w_idx = block * 32 + lane;
-      if (w_idx < n_words) bitmap[w_idx] = keep_word;
-      if (lane == 0) {
-        offsets[block] = static_cast<unsigned long long>(kept_before);
-        if (block == n_blocks - 1) {
-          const long long total = kept_before + kept_warp;
-          offsets[n_blocks] = static_cast<unsigned long long>(total);
-          if (total != hdr->n_keep)
-            atomicMax(&hdr->status, static_cast<uint32_t>(SURGEON_ERR_INTERNAL));
+        for (int j = 0; j < WPR; ++j)
+          if (w0 + j < n_words) bitmap[w0 + j] = my_words[j];
+      }
+#pragma unroll
+      for (int j = 0; j < BPR; ++j) {
+        const long long blk = row * BPR + j;
+        if (blk < n_blocks) {
+          offsets[blk] = my_off[j];
+          if (blk == n_blocks - 1) {
+            const long long total = static_cast<long long>(my_off[j]) + my_cnt[j];
+            offsets[n_blocks] = static_cast<uint32_t>(total);
+            if (total != hdr->n_keep)
+              atomicMax(&hdr->status, static_cast<uint32_t>(SURGEON_ERR_INTERNAL));
+          }
         }
       }
-      const uint32_t lt = lanemask_lt();
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const uint32_t kw = __shfl_sync(0xFFFFFFFFu, keep_word, i);
-        const uint32_t wb = __shfl_sync(0xFFFFFFFFu, word_excl, i);
-        if ((kw >> lane) & 1u) values[kept_before + wb + __popc(kw & lt)] = xs[i];
-      }
     }
-    __syncthreads();  // s_tile / s_gt / s_eq are rewritten by the next iteration
+  }
+  __syncthreads();
+
+  // ---- stage -> packed vector: whole 16-byte vectors where the tile owns all of them ----
+  const int span_end = align + static_cast<int>(tile_kept_end - tile_kept_before);   // stage[align, span_end)
+  const int n_slots = (span_end + EPV - 1) / EPV;
+  for (int j = tid; j < n_slots; j += kCompactThreads) {
+    const int lo = j * EPV, hi = lo + EPV;
+    if (lo >= align && hi <= span_end) {
+      *reinterpret_cast<uint4*>(values + stage_origin + lo) = *reinterpret_cast<const uint4*>(stage + lo);
+    } else {
+      for (int i = (lo < align ? align : lo); i < (hi < span_end ? hi : span_end); ++i)
+        values[stage_origin + i] = stage[i];
+    }
   }
 }
 
-__global__ void offsets_empty_kernel(unsigned long long* offsets) { offsets[0] = 0ull; }
+__global__ void offsets_empty_kernel(uint32_t* offsets) { offsets[0] = 0u; }
 
 // ---- decompress -------------------------------------------------------------------------------
 
-// Algorithm 1: Reshape step: one warp rebuilds one SURGEON_BLOCK of the dense tensor.
+// Algorithm 1, Reshape step: one warp rebuilds 1024 elements (32 bitmap words) of the dense tensor.
 template <int DT>
 __global__ void __launch_bounds__(256)
 decompress_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ values_v,
-                  const unsigned long long* __restrict__ offsets, long long n,
-                  void* __restrict__ out_v) {
+                  const uint32_t* __restrict__ offsets, long long n, void* __restrict__ out_v) {
   using E = typename Elem<DT>::type;
   const E* __restrict__ values = reinterpret_cast<const E*>(values_v);
   E* __restrict__ out = reinterpret_cast<E*>(out_v);
   const uint32_t lane = lane_id();
-  const long long n_blocks = (n + SURGEON_BLOCK - 1) / SURGEON_BLOCK;
+  const long long n_chunks = (n + 1023) / 1024;
   const long long n_words = (n + 31) / 32;
   const long long warps = (static_cast<long long>(gridDim.x) * blockDim.x) >> 5;
-  for (long long block = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
-       block < n_blocks; block += warps) {
-    const long long w_idx = block * 32 + lane;
+  for (long long chunk = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+       chunk < n_chunks; chunk += warps) {
+    const long long w_idx = chunk * 32 + lane;
     const uint32_t word = (w_idx < n_words) ? bitmap[w_idx] : 0u;
     const uint32_t word_excl = warp_excl_scan(__popc(word));
-    const unsigned long long first = offsets[block];
+    const long long first = offsets[chunk * (1024 / SURGEON_BLOCK)];
     const uint32_t lt = lanemask_lt();
-    const long long base = block * SURGEON_BLOCK;
+    const long long base = chunk * 1024;
 #pragma unroll 4
     for (int i = 0; i < 32; ++i) {
-      const uint32_t w = __shfl_sync(0xFFFFFFFFu, word, i);
-      const uint32_t wb = __shfl_sync(0xFFFFFFFFu, word_excl, i);
+      const uint32_t w = __shfl_sync(kFull, word, i);
+      const uint32_t wb = __shfl_sync(kFull, word_excl, i);
       const long long idx = base + i * 32 + lane;
       if (idx < n) out[idx] = ((w >> lane) & 1u) ? values[first + wb + __popc(w & lt)]
                                                  : static_cast<E>(0);
@@ -309,52 +851,87 @@ template <int DT>
 cudaError_t run_prune_compact(const void* x, long long n, long long k,
                               const surgeon_compressed& out, void* workspace,
                               cudaStream_t stream) {
+  constexpr int VEC = 16 / static_cast<int>(sizeof(typename Elem<DT>::type));
+  const PruneLayout L = prune_layout(n, DT);
   char* ws = static_cast<char*>(workspace);
   SelectState* st = reinterpret_cast<SelectState*>(ws);
-  uint32_t* ghist = reinterpret_cast<uint32_t*>(ws + kWsStateBytes);
-  unsigned long long* tile_state =
-      reinterpret_cast<unsigned long long*>(ws + kWsStateBytes + kWsHistBytes);
-  cudaError_t e = cudaMemsetAsync(workspace, 0, prune_workspace_bytes(n), stream);
+  uint32_t* hist1 = reinterpret_cast<uint32_t*>(ws + L.hist1);
+  uint32_t* hist_s = reinterpret_cast<uint32_t*>(ws + L.hist_s);
+  uint32_t* hist2 = reinterpret_cast<uint32_t*>(ws + L.hist2);
+  uint32_t* cnt_gt = reinterpret_cast<uint32_t*>(ws + L.cnt_gt);
+  uint32_t* cnt_eq = reinterpret_cast<uint32_t*>(ws + L.cnt_eq);
+  uint32_t* cnt_zero = reinterpret_cast<uint32_t*>(ws + L.cnt_zero);
+  uint32_t* full_gt = reinterpret_cast<uint32_t*>(ws + L.full_gt);
+  uint32_t* full_eq = reinterpret_cast<uint32_t*>(ws + L.full_eq);
+  unsigned long long* prefix = reinterpret_cast<unsigned long long*>(ws + L.prefix);
+  unsigned long long* list = reinterpret_cast<unsigned long long*>(ws + L.list);
+  const uint32_t list_cap = static_cast<uint32_t>(L.list_cap);
+  cudaError_t e = cudaMemsetAsync(workspace, 0, L.zero_bytes, stream);
   if (e != cudaSuccess) return e;
-  e = cudaMemsetAsync(out.header, 0, sizeof(surgeon_header), stream);
-  if (e != cudaSuccess) return e;
+  const int sms = sm_count();
+  static bool attrs_done_on[64] = {false};   // per device; a race only repeats idempotent calls
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+  bool& attrs_done = attrs_done_on[dev];
+  if (!attrs_done) {
+    e = cudaFuncSetAttribute(sample_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kHistWords * 4);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(hist_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(kHistSmem));
+    if (e != cudaSuccess) return e;
+    attrs_done = true;
+  }
 
   if (k == 0) {
     header_empty_kernel<<<1, 1, 0, stream>>>(out.header, Elem<DT>::kSentinel);
     note_launches(1);
   } else {
-    constexpr int VEC = 16 / static_cast<int>(sizeof(typename Elem<DT>::type));
     const long long nvec = n / VEC;
-    long long want = (nvec + kHistThreads * 4 - 1) / (kHistThreads * 4);
-    const int grid = static_cast<int>(want < 1 ? 1 : (want > 2LL * sm_count() ? 2LL * sm_count() : want));
-    if (DT == 0) {
-      radix_hist_kernel<0, 20, 11, false><<<grid, kHistThreads, 0, stream>>>(
-          x, n, k, 0, st, ghist, out.header);
-      radix_hist_kernel<0, 9, 11, false><<<grid, kHistThreads, 0, stream>>>(
-          x, n, k, 1, st, ghist + kMaxBins, out.header);
-      radix_hist_kernel<0, 0, 9, true><<<grid, kHistThreads, 0, stream>>>(
-          x, n, k, 2, st, ghist + 2 * kMaxBins, out.header);
-      note_launches(3);
-    } else {
-      radix_hist_kernel<1, 4, 11, false><<<grid, kHistThreads, 0, stream>>>(
-          x, n, k, 0, st, ghist, out.header);
-      radix_hist_kernel<1, 0, 4, true><<<grid, kHistThreads, 0, stream>>>(
-          x, n, k, 1, st, ghist + kMaxBins, out.header);
-      note_launches(2);
+    int use_bracket = 0;
+    if (n > kSampleMinN) {
+      // sample: segments of 32 vectors, about 1/32 of the tensor, at most 16384 segments
+      const long long n_seg_all = nvec / 32;
+      long long n_seg = n_seg_all / 32;
+      if (n_seg < 256) n_seg = 256;
+      if (n_seg > 16384) n_seg = 16384;
+      const long long seg_stride = n_seg_all / n_seg;   // >= 1 because n > 65536
+      const long long want = (n_seg + 63) / 64;
+      const int grid = static_cast<int>(want < sms ? want : sms);
+      sample_kernel<DT><<<grid, kSelThreads, kHistWords * 4, stream>>>(
+          reinterpret_cast<const uint4*>(x), n, static_cast<uint32_t>(k),
+          static_cast<uint32_t>(n_seg), static_cast<uint32_t>(seg_stride), st, hist_s);
+      note_launches(1);
+      use_bracket = 1;
     }
+    {
+      const long long chunks = (nvec + kStageVecs - 1) / kStageVecs;
+      const int grid = static_cast<int>(chunks < 1 ? 1 : (chunks < sms ? chunks : sms));
+      hist_kernel<DT><<<grid, kSelThreads, kHistSmem, stream>>>(
+          x, n, static_cast<uint32_t>(k), use_bracket, st, hist1, hist2, cnt_gt, cnt_zero, list,
+          list_cap, out.header);
+      note_launches(1);
+    }
+    const long long want = (nvec + 4 * kSelThreads - 1) / (4 * kSelThreads);
+    const long long cap = 2LL * sms;
+    const int grid = static_cast<int>(want < 1 ? 1 : (want < cap ? want : cap));
+    if (DT == 0) {
+      refine_kernel<<<grid, kSelThreads, 0, stream>>>(
+          reinterpret_cast<const uint4*>(x), n, static_cast<uint32_t>(k), st, hist2, list, list_cap,
+          out.header);
+      note_launches(1);
+    }
+    count_kernel<DT><<<grid, kSelThreads, 0, stream>>>(
+        x, n, st, out.header, list, list_cap, cnt_gt, cnt_eq, cnt_zero, full_gt, full_eq, prefix,
+        static_cast<int>(L.tiles));
+    note_launches(1);
   }
   if (n == 0) {
-    offsets_empty_kernel<<<1, 1, 0, stream>>>(
-        reinterpret_cast<unsigned long long*>(out.block_offsets));
+    offsets_empty_kernel<<<1, 1, 0, stream>>>(out.block_offsets);
     note_launches(1);
   } else {
-    const long long tiles = (n + kTileElems - 1) / kTileElems;
-    const long long cap = 8LL * sm_count();
-    const int grid = static_cast<int>(tiles < cap ? tiles : cap);
-    compact_kernel<DT><<<grid, 256, 0, stream>>>(
-        x, n, out.header, out.bitmap, out.values,
-        reinterpret_cast<unsigned long long*>(out.block_offsets), &st->compact_ticket, tile_state,
-        static_cast<int>(tiles));
+    compact_kernel<DT><<<static_cast<unsigned>(L.tiles), kCompactThreads, 0, stream>>>(
+        x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix);
     note_launches(1);
   }
   return cudaGetLastError();
@@ -371,15 +948,16 @@ cudaError_t launch_prune_compact(const void* x, int64_t n, int dt, int64_t k,
 
 cudaError_t launch_decompress(const surgeon_compressed& act, void* x_out, cudaStream_t stream) {
   if (act.n == 0) return cudaSuccess;
-  const long long n_blocks = (act.n + SURGEON_BLOCK - 1) / SURGEON_BLOCK;
-  const long long ctas = (n_blocks + 7) / 8;
+  const long long n_chunks = (act.n + 1023) / 1024;
+  const long long ctas = (n_chunks + 7) / 8;
   const long long cap = 16LL * sm_count();
   const int grid = static_cast<int>(ctas < cap ? ctas : cap);
-  const unsigned long long* offs = reinterpret_cast<const unsigned long long*>(act.block_offsets);
   if (act.dt == 0)
-    decompress_kernel<0><<<grid, 256, 0, stream>>>(act.bitmap, act.values, offs, act.n, x_out);
+    decompress_kernel<0><<<grid, 256, 0, stream>>>(act.bitmap, act.values, act.block_offsets, act.n,
+                                                   x_out);
   else
-    decompress_kernel<1><<<grid, 256, 0, stream>>>(act.bitmap, act.values, offs, act.n, x_out);
+    decompress_kernel<1><<<grid, 256, 0, stream>>>(act.bitmap, act.values, act.block_offsets, act.n,
+                                                   x_out);
   note_launches(1);
   return cudaGetLastError();
 }

@@ -6,7 +6,7 @@
 // (for instance while a stream is being captured), a plug-in behind a host API that forbids
 // cudaMalloc, or a process whose memory budget was handed out in full at start-up.  Such a
 // caller already owns the input and the output buffers of the store, but the select and the
-// compaction also need a few hundred kilobytes of scratch.  This entry point keeps that
+// compaction also need a couple of megabytes of scratch.  This entry point keeps that
 // scratch inside the library image, so nothing is allocated by anybody.
 #include <mutex>
 
@@ -15,7 +15,9 @@
 namespace surgeon {
 namespace {
 
-constexpr size_t kStaticScratchBytes = prune_workspace_bytes(SURGEON_STATIC_MAX_N);
+// fp32 needs the larger scratch of the two dtypes
+constexpr size_t kStaticScratchBytes = prune_workspace_bytes(SURGEON_STATIC_MAX_N, 0);
+static_assert(kStaticScratchBytes >= prune_workspace_bytes(SURGEON_STATIC_MAX_N, 1), "scratch");
 
 // The scratch itself: part of the module's global data, present once on every device that
 // loads the library, for the life of the process.  In host code this name is only a handle for

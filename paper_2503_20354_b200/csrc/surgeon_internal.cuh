@@ -24,28 +24,65 @@ template <> struct Elem<1> {
   static constexpr int kKeyBits = 15;
 };
 
-constexpr int kTileBlocks = 8;                         // offset blocks per compaction tile
-constexpr int kTileElems = kTileBlocks * SURGEON_BLOCK;  // 8192 elements per CTA tile
+constexpr int kBlockShift = 7;                       // log2(SURGEON_BLOCK)
+constexpr int kBlockWords = SURGEON_BLOCK / 32;      // bitmap words per offset block
+static_assert((1 << kBlockShift) == SURGEON_BLOCK, "SURGEON_BLOCK must be 128");
 
-// Scratch layout of surgeon_prune_compact (offsets in bytes from the workspace base).
+// ---- scratch of surgeon_prune_compact ---------------------------------------------------------
+// Compaction tile = 1024 16-byte vectors: 8 warps x 4 rows of 32 lanes x 16 bytes.
+constexpr int kTileVecs = 1024;
+constexpr int64_t compact_tile_elems(int dt) { return dt == 0 ? 4096 : 8192; }
+constexpr int kBuckets = 32768;        // histogram bins of the select pass (top 15 key bits)
+constexpr int kLowBins = 65536;        // bins of the fp32 refinement (low 16 key bits)
+constexpr int64_t kSampleMinN = 65536; // tensors up to this size list every non-zero element
+
 struct SelectState {
-  uint32_t prefix;        // key bits fixed so far (lower bits zero)
-  uint32_t compact_ticket;
-  long long k_remaining;  // rank still to find inside the current prefix bucket
-  long long n_greater;    // keys known to be strictly above the bucket
-  uint32_t pass_ticket[4];
+  uint32_t ticket_sample, ticket_hist, ticket_refine, ticket_count;
+  uint32_t blo, bhi;             // bucket bracket around the threshold, predicted from the sample
+  uint32_t list_count, list_overflow;
+  uint32_t b1, mode;             // bucket of the threshold; 0 = candidate list usable, 1 = re-read x
+  uint32_t k1, above;            // rank of the threshold inside bucket b1; keys in buckets above b1
+  uint32_t zero_count;           // elements whose key is exactly 0
+  uint32_t error;                // surgeon_status raised by a bounded wait of the select kernels
   uint32_t pad[2];
 };
-static_assert(sizeof(SelectState) == 48, "SelectState layout");
+static_assert(sizeof(SelectState) == 64, "SelectState layout");
 constexpr size_t kWsStateBytes = 256;
-constexpr int kMaxBins = 2048;
-constexpr size_t kWsHistBytes = 3 * kMaxBins * sizeof(uint32_t);  // one histogram per pass
 
-constexpr size_t prune_workspace_bytes(int64_t n) {
-  const int64_t tiles = (n + kTileElems - 1) / kTileElems;
-  size_t b = kWsStateBytes + kWsHistBytes + static_cast<size_t>(tiles) * 8;
-  return (b + 255) & ~static_cast<size_t>(255);
+// Byte offsets of the parts of the scratch buffer; everything in [0, zero_bytes) must be zero
+// when the first kernel starts.  Per compaction tile: cnt_gt / cnt_zero are filled by the
+// histogram pass (keys above the bracket, exact zeros), cnt_gt / cnt_eq are completed from the
+// candidate list once the threshold is known; full_gt / full_eq are used instead when the
+// tensor had to be re-read; prefix holds the exclusive scan the compaction kernel starts from.
+struct PruneLayout {
+  size_t hist1, hist_s, hist2, cnt_gt, cnt_eq, cnt_zero, full_gt, full_eq, prefix, zero_bytes,
+      list, total;
+  int64_t tiles, list_cap;
+};
+constexpr PruneLayout prune_layout(int64_t n, int dt) {
+  PruneLayout L{};
+  L.tiles = (n + compact_tile_elems(dt) - 1) / compact_tile_elems(dt);
+  const size_t per_tile = static_cast<size_t>(L.tiles) * 4;
+  size_t off = kWsStateBytes;
+  L.hist1 = off; off += static_cast<size_t>(kBuckets) * 4;
+  L.hist_s = off; off += static_cast<size_t>(kBuckets) * 4;
+  L.hist2 = off; if (dt == 0) off += static_cast<size_t>(kLowBins) * 4;
+  L.cnt_gt = off; off += per_tile;
+  L.cnt_eq = off; off += per_tile;
+  L.cnt_zero = off; off += per_tile;
+  L.full_gt = off; off += per_tile;
+  L.full_eq = off; off += per_tile;
+  off = (off + 15) & ~static_cast<size_t>(15);
+  L.prefix = off; off += per_tile * 2;
+  off = (off + 255) & ~static_cast<size_t>(255);
+  L.zero_bytes = off;
+  L.list = off;
+  L.list_cap = n <= kSampleMinN ? n : n / 32 + kSampleMinN;
+  off += static_cast<size_t>(L.list_cap) * 8;
+  L.total = (off + 255) & ~static_cast<size_t>(255);
+  return L;
 }
+constexpr size_t prune_workspace_bytes(int64_t n, int dt) { return prune_layout(n, dt).total; }
 
 // Host launchers (each enqueues on `stream` and returns the last CUDA error).
 cudaError_t launch_prune_compact(const void* x, int64_t n, int dt, int64_t k,

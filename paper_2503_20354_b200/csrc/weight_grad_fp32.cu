@@ -37,15 +37,15 @@ __host__ __device__ inline Geom make_geom(const surgeon_layer_desc& d) {
 template <int DT>
 __device__ __forceinline__ float fetch_act(const uint32_t* __restrict__ bitmap,
                                            const void* __restrict__ values,
-                                           const unsigned long long* __restrict__ offsets,
+                                           const uint32_t* __restrict__ offsets,
                                            long long j) {
   const long long wi = j >> 5;
   const uint32_t w = __ldg(bitmap + wi);
   const uint32_t bit = static_cast<uint32_t>(j) & 31u;
   if (!((w >> bit) & 1u)) return 0.0f;
-  const long long blk = j >> 10;
+  const long long blk = j >> kBlockShift;
   long long r = static_cast<long long>(__ldg(offsets + blk));
-  for (long long t = blk * 32; t < wi; ++t) r += __popc(__ldg(bitmap + t));
+  for (long long t = blk * kBlockWords; t < wi; ++t) r += __popc(__ldg(bitmap + t));
   r += __popc(w & ((1u << bit) - 1u));
   if (DT == 0) return __ldg(reinterpret_cast<const float*>(values) + r);
   const uint32_t h = __ldg(reinterpret_cast<const unsigned short*>(values) + r);
@@ -55,7 +55,7 @@ __device__ __forceinline__ float fetch_act(const uint32_t* __restrict__ bitmap,
 template <int DT>
 __global__ void __launch_bounds__(256)
 dw_fp32_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ values,
-               const unsigned long long* __restrict__ offsets, const float* __restrict__ grad,
+               const uint32_t* __restrict__ offsets, const float* __restrict__ grad,
                float* __restrict__ partial, Geom g) {
   __shared__ float Gs[TK][TM + 4];
   __shared__ float As[TK][TN + 4];
@@ -172,7 +172,7 @@ cudaError_t launch_weight_grad_fp32(const surgeon_compressed& act, const surgeon
   const Geom g = make_geom(d);
   const long long chunks = (g.K + kChunk - 1) / kChunk;
   float* partial = static_cast<float*>(workspace);
-  const unsigned long long* offs = reinterpret_cast<const unsigned long long*>(act.block_offsets);
+  const uint32_t* offs = act.block_offsets;
   if (chunks > 0) {
     dim3 grid(static_cast<unsigned>((g.N + TN - 1) / TN), static_cast<unsigned>((g.M + TM - 1) / TM),
               static_cast<unsigned>(chunks));

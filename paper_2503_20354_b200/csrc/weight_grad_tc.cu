@@ -63,15 +63,15 @@ __device__ __forceinline__ void producer_sync() {
 template <int DT>
 __device__ __forceinline__ void decompress_range(const uint32_t* __restrict__ bitmap,
                                                  const void* __restrict__ values,
-                                                 const unsigned long long* __restrict__ offsets,
+                                                 const uint32_t* __restrict__ offsets,
                                                  long long start, int len,
                                                  unsigned short* __restrict__ dst) {
   const uint32_t lane = lane_id();
   const uint32_t lt = lanemask_lt();
   const long long first_word = start >> 5;
   const long long last_word = (start + len - 1) >> 5;
-  const long long blk = start >> 10;
-  const long long blk_word0 = blk << 5;
+  const long long blk = start >> kBlockShift;
+  const long long blk_word0 = blk * kBlockWords;
   uint32_t w = 0;
   if (blk_word0 + lane < first_word) w = __ldg(bitmap + blk_word0 + lane);
   long long rank = static_cast<long long>(__ldg(offsets + blk)) + warp_sum(__popc(w));
@@ -98,7 +98,7 @@ struct RowInfo {   // one im2col row (nn) of the CTA's M tile
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 1)
 dw_tc_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ values,
-             const unsigned long long* __restrict__ offsets, const float* __restrict__ grad,
+             const uint32_t* __restrict__ offsets, const float* __restrict__ grad,
              float* __restrict__ partial, uint32_t* __restrict__ status, TcParams p) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   // carve: [stages][A 16 KB | B tile_n*128] | patch | barriers | row table
@@ -479,7 +479,7 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
   TcParams p;
   if (!plan(d, act.dt, &p)) return cudaErrorNotSupported;
   const size_t smem = smem_bytes(p);
-  const unsigned long long* offs = reinterpret_cast<const unsigned long long*>(act.block_offsets);
+  const uint32_t* offs = act.block_offsets;
   dim3 grid(p.m_tiles, p.n_tiles, p.splits);
   if (act.dt == 0) {
     e = cudaFuncSetAttribute(dw_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -77,7 +77,7 @@ __device__ __forceinline__ uint4 gather8(uint32_t bits, uint32_t r0, int step,
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 1)
 dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ values,
-                    const unsigned long long* __restrict__ offsets,
+                    const uint32_t* __restrict__ offsets,
                     const __grid_constant__ CUtensorMap grad_map, float* __restrict__ partial,
                     uint32_t* __restrict__ status, FastParams p) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -202,8 +202,8 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
         for (int ri = gwarp; ri < n_ch; ri += kGroupWarps) {
           const long long start = plane_of(t, ri) + static_cast<long long>(t.iy_lo) * p.W;
           const long long first_word = start >> 5;
-          const long long blk = start >> 10;
-          const long long blk_word0 = blk << 5;
+          const long long blk = start >> kBlockShift;
+          const long long blk_word0 = blk * kBlockWords;
           uint32_t wb = 0;
           if (blk_word0 + lane < first_word) wb = __ldg(bitmap + blk_word0 + lane);
           const int nwords = static_cast<int>(((start + t.range_len - 1) >> 5) - first_word) + 1;
@@ -223,13 +223,13 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
           const int y0 = t.p0 / p.OW;
           const int x00 = t.p0 - y0 * p.OW;
           long long pos = plane + static_cast<long long>(y0 * p.stride) * p.W + x00 * p.stride;
-          const long long blk = pos >> 10;
+          const long long blk = pos >> kBlockShift;
           uint32_t rank = static_cast<uint32_t>(__ldg(offsets + blk));
           {
-            const long long blk_word0 = blk << 5;
+            const long long blk_word0 = blk * kBlockWords;
             const int before = static_cast<int>((pos >> 5) - blk_word0);
-#pragma unroll 8
-            for (int w = 0; w < 31; ++w)
+#pragma unroll
+            for (int w = 0; w < kBlockWords - 1; ++w)
               if (w < before) rank += __popc(__ldg(bitmap + blk_word0 + w));
             const uint32_t w0 = __ldg(bitmap + (pos >> 5));
             rank += __popc(w0 & ((1u << (pos & 31)) - 1u));
@@ -550,7 +550,7 @@ cudaError_t launch_conv_fast(const surgeon_compressed& act, const FastParams& p,
       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
 
-  const unsigned long long* offs = reinterpret_cast<const unsigned long long*>(act.block_offsets);
+  const uint32_t* offs = act.block_offsets;
   dim3 grid(p.m_tiles, p.n_tiles, p.splits);
   cudaError_t e;
   if (act.dt == 0) {

@@ -100,7 +100,7 @@ def test_non_default_stream_and_canaries():
     pad = 64
     big_bitmap = torch.full((sizes.bitmap_bytes // 4 + pad,), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
     big_vals = torch.full((sizes.n_keep + pad,), 12345.0, dtype=torch.float32, device="cuda")
-    big_offs = torch.full((sizes.offsets_bytes // 8 + pad,), 0x1234567, dtype=torch.int64, device="cuda")
+    big_offs = torch.full((sizes.offsets_bytes // 4 + pad,), 0x1234567, dtype=torch.int32, device="cuda")
     comp.bitmap, comp.values, comp.block_offsets = big_bitmap, big_vals, big_offs
     comp.c.bitmap, comp.c.values, comp.c.block_offsets = (big_bitmap.data_ptr(), big_vals.data_ptr(),
                                                           big_offs.data_ptr())
@@ -111,7 +111,7 @@ def test_non_default_stream_and_canaries():
     assert_store_equals_oracle(x.cpu(), 0.4, comp=comp)
     assert torch.all(big_bitmap[sizes.bitmap_bytes // 4:] == 0x5A5A5A5A)
     assert torch.all(big_vals[sizes.n_keep:] == 12345.0)
-    assert torch.all(big_offs[sizes.offsets_bytes // 8:] == 0x1234567)
+    assert torch.all(big_offs[sizes.offsets_bytes // 4:] == 0x1234567)
 
 
 def test_argument_errors_on_device():

@@ -70,7 +70,7 @@ def test_compact_sizes_match_oracle_kept_count():
                 assert s.n_keep == oracle.n_keep(n, ratio)
                 assert s.bitmap_bytes == 4 * ((n + 31) // 32)
                 assert s.values_bytes == s.n_keep * es
-                assert s.offsets_bytes == 8 * ((n + 1023) // 1024 + 1)
+                assert s.offsets_bytes == 4 * ((n + 127) // 128 + 1)
                 assert s.workspace_bytes > 0 and s.workspace_bytes % 256 == 0
     for bad in ((-1, 0, 0.5), (10, 0, 1.5), (10, 0, -0.1), (10, 2, 0.5), (10, 0, float("nan"))):
         with pytest.raises(B.SurgeonError) as e:
