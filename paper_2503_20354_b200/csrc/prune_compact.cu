@@ -465,7 +465,8 @@ __global__ void header_empty_kernel(surgeon_header* hdr, uint32_t sentinel) {
 }
 
 // ---- per-tile counts -> exclusive scan over tiles -------------------------------------------
-// prefix[t] = (keys above the threshold before tile t) << 31 | (keys equal to it before tile t).
+// prefix[t] = (keys above the threshold before tile t) << 31 | (keys equal to it before tile t),
+// t = 0 .. tiles (the last entry holds the totals).
 template <int DT>
 __global__ void __launch_bounds__(kSelThreads)
 count_kernel(const void* __restrict__ xv, long long n, SelectState* __restrict__ st,
@@ -587,6 +588,7 @@ count_kernel(const void* __restrict__ xv, long long n, SelectState* __restrict__
     carry += __shfl_sync(kFull, incl, 31);
   }
   if (tid == 0) {
+    prefix[tiles] = total;
     // self-check: the counts must add up to what the select found
     const long long gt_all = static_cast<long long>(total >> 31);
     const long long eq_all = static_cast<long long>(total & 0x7FFFFFFFull);
@@ -613,12 +615,18 @@ __device__ __forceinline__ uint32_t lowest_set_bits(uint32_t m, long long allowe
   return m;
 }
 
-// One CTA per tile; nothing is exchanged between CTAs.
-template <int DT>
-__global__ void __launch_bounds__(kCompactThreads)
-compact_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restrict__ hdr,
-               uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
-               uint32_t* __restrict__ offsets, const unsigned long long* __restrict__ prefix) {
+// Emits one tile.  SLOW = false: every tie of the tile is kept, or none is (`ties`), so one
+// decision per element suffices.  SLOW = true: the tie quota ends inside this tile; ties are
+// ranked by flat index.  Nothing is exchanged between CTAs.
+template <int DT, bool SLOW>
+__device__ __forceinline__ void compact_tile(const typename Elem<DT>::type* __restrict__ x,
+                                             long long n, const uint4 (&q)[kRows], int tile,
+                                             uint32_t tau, long long quota, bool ties,
+                                             long long gt_tile_before, long long eq_tile_before,
+                                             surgeon_header* __restrict__ hdr,
+                                             uint32_t* __restrict__ bitmap,
+                                             typename Elem<DT>::type* __restrict__ values,
+                                             uint32_t* __restrict__ offsets) {
   using E = typename Elem<DT>::type;
   constexpr uint32_t kMask = Elem<DT>::kKeyMask;
   constexpr int EPV = 16 / sizeof(E);          // elements per lane and row: 4 (fp32) / 8 (bf16)
@@ -626,45 +634,17 @@ compact_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restr
   constexpr int WPR = ROW / 32;                // bitmap words per row: 4 / 8
   constexpr int LPW = 32 / EPV;                // lanes per bitmap word: 8 / 4
   constexpr int BPR = ROW / SURGEON_BLOCK;     // offset blocks per row: 1 / 2
-  constexpr int TILE = 8 * kRows * ROW;
   constexpr uint32_t kEMask = (1u << EPV) - 1u;
-  const E* __restrict__ x = reinterpret_cast<const E*>(xv);
-  E* __restrict__ values = reinterpret_cast<E*>(values_v);
-  __shared__ __align__(16) E stage[TILE + EPV];   // kept values of the tile, aligned like the output
   __shared__ uint32_t s_gt[8], s_eq[8];
-
-  const int tid = threadIdx.x;
   const uint32_t lane = lane_id();
-  const int warp = tid >> 5;
-  const int tile = blockIdx.x;
+  const int warp = threadIdx.x >> 5;
   const long long n_blocks = (n + SURGEON_BLOCK - 1) >> kBlockShift;
   const long long n_words = (n + 31) / 32;
   const int my_word = lane / LPW;
   const int my_shift = EPV * (lane % LPW);
-
-  // ---- load kRows rows; the header and the tile's scan entry travel alongside ----
   const long long row0 = (static_cast<long long>(tile) * 8 + warp) * kRows;
-  uint4 q[kRows];
-#pragma unroll
-  for (int r = 0; r < kRows; ++r) {
-    const long long base = (row0 + r) * ROW + static_cast<long long>(lane) * EPV;
-    if (base + EPV <= n) {
-      q[r] = __ldg(reinterpret_cast<const uint4*>(x + base));
-    } else {
-      uint32_t t[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i)
-        t[i] = (i < EPV && base + i < n) ? static_cast<uint32_t>(x[base + i]) : 0u;
-      if (DT == 0) q[r] = make_uint4(t[0], t[1], t[2], t[3]);
-      else q[r] = make_uint4(t[0] | (t[1] << 16), t[2] | (t[3] << 16), t[4] | (t[5] << 16),
-                             t[6] | (t[7] << 16));
-    }
-  }
-  const uint32_t tau = hdr->threshold_key;
-  const long long quota = hdr->tie_quota;
-  const unsigned long long excl = prefix[tile];
 
-  // ---- per row and lane EPV decisions "above tau" and "equal to tau" ----
+  // per row and lane EPV decisions: g = kept for sure, e = tie at the threshold (SLOW only)
   uint32_t g_all = 0, e_all = 0;      // kRows fields of EPV bits
 #pragma unroll
   for (int r = 0; r < kRows; ++r) {
@@ -676,35 +656,29 @@ compact_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restr
       const uint32_t bits = (DT == 0) ? w[i % 4] : (w[i >> 1] >> (16 * (i & 1)));
       const uint32_t key = bits & kMask;
       const bool valid = base + i < n;
-      g |= (valid && key > tau) ? (1u << i) : 0u;
-      e |= (valid && key == tau) ? (1u << i) : 0u;
+      if (SLOW) {
+        g |= (valid && key > tau) ? (1u << i) : 0u;
+        e |= (valid && key == tau) ? (1u << i) : 0u;
+      } else {
+        g |= (valid && (key > tau || (ties && key == tau))) ? (1u << i) : 0u;
+      }
     }
     g_all |= g << (EPV * r);
     e_all |= e << (EPV * r);
   }
   const uint32_t gt_warp = __reduce_add_sync(kFull, __popc(g_all));
-  const uint32_t eq_warp = __reduce_add_sync(kFull, __popc(e_all));
+  const uint32_t eq_warp = SLOW ? __reduce_add_sync(kFull, __popc(e_all)) : 0u;
   if (lane == 0) { s_gt[warp] = gt_warp; s_eq[warp] = eq_warp; }
   __syncthreads();
 
-  const long long gt_tile_before = static_cast<long long>(excl >> 31);
-  const long long eq_tile_before = static_cast<long long>(excl & kCountMask);
   long long gt_before = gt_tile_before, eq_before = eq_tile_before;
-  long long gt_all = gt_tile_before, eq_all = eq_tile_before;
 #pragma unroll
   for (int w = 0; w < 8; ++w) {
     if (w < warp) { gt_before += s_gt[w]; eq_before += s_eq[w]; }
-    gt_all += s_gt[w]; eq_all += s_eq[w];
   }
-  // kept before = all greater + the ties that fit the quota
-  const long long tile_kept_before = gt_tile_before + (eq_tile_before < quota ? eq_tile_before : quota);
-  const long long tile_kept_end = gt_all + (eq_all < quota ? eq_all : quota);
+  // kept before = all greater + the ties that fit the quota.  In the fast path the kept ties of
+  // this tile are already inside the "greater" counts and eq_before stays the tile's value.
   long long kept_before = gt_before + (eq_before < quota ? eq_before : quota);
-  // 0: no tie of this warp is kept, 1: all are, 2: the quota ends inside these rows
-  const int tie_mode = (eq_before >= quota) ? 0 : (eq_before + eq_warp <= quota ? 1 : 2);
-  // the stage mirrors the 16-byte alignment of the tile's range in the packed vector
-  const int align = static_cast<int>(tile_kept_before % EPV);
-  const long long stage_origin = tile_kept_before - align;   // packed index of stage[0]
 
   uint32_t my_words[WPR];      // lane r keeps the bitmap words of row r
   uint32_t my_off[BPR];        // and the offsets of its blocks
@@ -717,12 +691,9 @@ compact_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restr
   if (row0 * ROW < n) {
 #pragma unroll
     for (int r = 0; r < kRows; ++r) {
-      const uint32_t g = (g_all >> (EPV * r)) & kEMask;
-      const uint32_t e = (e_all >> (EPV * r)) & kEMask;
-      uint32_t keep = g;
-      if (tie_mode == 1) {
-        keep |= e;
-      } else if (tie_mode == 2) {
+      uint32_t keep = (g_all >> (EPV * r)) & kEMask;
+      if (SLOW) {
+        const uint32_t e = (e_all >> (EPV * r)) & kEMask;
         const uint32_t ec = __popc(e);
         const uint32_t before = warp_excl_scan(ec);      // ties of this row in lower lanes
         keep |= lowest_set_bits(e, quota - eq_before - before);
@@ -755,14 +726,14 @@ compact_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restr
           my_cnt[0] = total;
         }
       }
-      // kept values into the stage, in packed order
-      int dst = static_cast<int>(kept_before - stage_origin) + static_cast<int>(pre);
+      // packed values: consecutive kept elements go to consecutive addresses
+      E* dst = values + kept_before + pre;
       const uint32_t w[4] = {q[r].x, q[r].y, q[r].z, q[r].w};
 #pragma unroll
       for (int i = 0; i < EPV; ++i) {
         if ((keep >> i) & 1u) {
-          stage[dst++] = (DT == 0) ? static_cast<E>(w[i % 4])
-                                   : static_cast<E>((w[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
+          *dst++ = (DT == 0) ? static_cast<E>(w[i % 4])
+                             : static_cast<E>((w[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
         }
       }
       kept_before += total;
@@ -796,20 +767,80 @@ compact_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restr
       }
     }
   }
-  __syncthreads();
+}
 
-  // ---- stage -> packed vector: whole 16-byte vectors where the tile owns all of them ----
-  const int span_end = align + static_cast<int>(tile_kept_end - tile_kept_before);   // stage[align, span_end)
-  const int n_slots = (span_end + EPV - 1) / EPV;
-  for (int j = tid; j < n_slots; j += kCompactThreads) {
-    const int lo = j * EPV, hi = lo + EPV;
-    if (lo >= align && hi <= span_end) {
-      *reinterpret_cast<uint4*>(values + stage_origin + lo) = *reinterpret_cast<const uint4*>(stage + lo);
+template <int DT>
+__device__ __forceinline__ void load_tile(const typename Elem<DT>::type* __restrict__ x,
+                                          long long n, int tile, uint4 (&q)[kRows]) {
+  constexpr int EPV = 16 / sizeof(typename Elem<DT>::type);
+  constexpr int ROW = 32 * EPV;
+  const long long row0 = (static_cast<long long>(tile) * 8 + (threadIdx.x >> 5)) * kRows;
+#pragma unroll
+  for (int r = 0; r < kRows; ++r) {
+    const long long base = (row0 + r) * ROW + static_cast<long long>(lane_id()) * EPV;
+    if (base + EPV <= n) {
+      q[r] = __ldg(reinterpret_cast<const uint4*>(x + base));
     } else {
-      for (int i = (lo < align ? align : lo); i < (hi < span_end ? hi : span_end); ++i)
-        values[stage_origin + i] = stage[i];
+      uint32_t t[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        t[i] = (i < EPV && base + i < n) ? static_cast<uint32_t>(x[base + i]) : 0u;
+      if (DT == 0) q[r] = make_uint4(t[0], t[1], t[2], t[3]);
+      else q[r] = make_uint4(t[0] | (t[1] << 16), t[2] | (t[3] << 16), t[4] | (t[5] << 16),
+                             t[6] | (t[7] << 16));
     }
   }
+}
+
+// One CTA per tile.  The one tile inside which the tie quota ends (if any) is left to
+// compact_boundary_kernel.
+template <int DT>
+__global__ void __launch_bounds__(kCompactThreads)
+compact_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restrict__ hdr,
+               uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
+               uint32_t* __restrict__ offsets, const unsigned long long* __restrict__ prefix) {
+  using E = typename Elem<DT>::type;
+  const E* __restrict__ x = reinterpret_cast<const E*>(xv);
+  const int tile = blockIdx.x;
+  uint4 q[kRows];
+  load_tile<DT>(x, n, tile, q);     // in flight while the header and the scan entries arrive
+  const uint32_t tau = hdr->threshold_key;
+  const long long quota = hdr->tie_quota;
+  const unsigned long long pb = prefix[tile], pe = prefix[tile + 1];
+  const long long eq_b = static_cast<long long>(pb & kCountMask);
+  const long long eq_e = static_cast<long long>(pe & kCountMask);
+  if (eq_b < quota && eq_e > quota) return;            // boundary tile
+  compact_tile<DT, false>(x, n, q, tile, tau, quota, /*ties=*/eq_e <= quota,
+                          static_cast<long long>(pb >> 31), eq_b, hdr, bitmap,
+                          reinterpret_cast<E*>(values_v), offsets);
+}
+
+// One CTA: finds the tile inside which the tie quota ends and emits it with ties ranked by index.
+template <int DT>
+__global__ void __launch_bounds__(kCompactThreads)
+compact_boundary_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restrict__ hdr,
+                        uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
+                        uint32_t* __restrict__ offsets,
+                        const unsigned long long* __restrict__ prefix, int tiles) {
+  using E = typename Elem<DT>::type;
+  const E* __restrict__ x = reinterpret_cast<const E*>(xv);
+  const long long quota = hdr->tie_quota;
+  // first tile whose inclusive tie count exceeds the quota (the counts never decrease)
+  int lo = 0, hi = tiles;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (static_cast<long long>(prefix[mid + 1] & kCountMask) > quota) hi = mid;
+    else lo = mid + 1;
+  }
+  if (lo >= tiles) return;
+  const unsigned long long pb = prefix[lo];
+  const long long eq_b = static_cast<long long>(pb & kCountMask);
+  if (eq_b >= quota) return;                            // the quota ends exactly between tiles
+  uint4 q[kRows];
+  load_tile<DT>(x, n, lo, q);
+  compact_tile<DT, true>(x, n, q, lo, hdr->threshold_key, quota, false,
+                         static_cast<long long>(pb >> 31), eq_b, hdr, bitmap,
+                         reinterpret_cast<E*>(values_v), offsets);
 }
 
 __global__ void offsets_empty_kernel(uint32_t* offsets) { offsets[0] = 0u; }
@@ -932,7 +963,10 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
   } else {
     compact_kernel<DT><<<static_cast<unsigned>(L.tiles), kCompactThreads, 0, stream>>>(
         x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix);
-    note_launches(1);
+    compact_boundary_kernel<DT><<<1, kCompactThreads, 0, stream>>>(
+        x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix,
+        static_cast<int>(L.tiles));
+    note_launches(2);
   }
   return cudaGetLastError();
 }

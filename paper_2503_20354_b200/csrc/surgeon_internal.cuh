@@ -73,7 +73,7 @@ constexpr PruneLayout prune_layout(int64_t n, int dt) {
   L.full_gt = off; off += per_tile;
   L.full_eq = off; off += per_tile;
   off = (off + 15) & ~static_cast<size_t>(15);
-  L.prefix = off; off += per_tile * 2;
+  L.prefix = off; off += per_tile * 2 + 8;   // tiles + 1 entries
   off = (off + 255) & ~static_cast<size_t>(255);
   L.zero_bytes = off;
   L.list = off;
