@@ -28,6 +28,8 @@
 // non-zero value), refine and count read the tensor once more instead of the list.  The result
 // is exact and unique either way; only the cost differs.
 // Every count fits 32 bits because n <= SURGEON_MAX_N < 2^31.
+#include <cuda.h>
+
 #include "surgeon_internal.cuh"
 #include "tc_common.cuh"
 
@@ -511,10 +513,14 @@ count_kernel(const void* __restrict__ xv, long long n, SelectState* __restrict__
       }
     }
   } else {
-    // the list is unusable: count every tile from the tensor itself (one vector per thread)
+    // the list is unusable: count every tile from the tensor itself (one vector per thread,
+    // a warp's 32 vectors lie inside one tile)
     const E* __restrict__ x = reinterpret_cast<const E*>(xv);
-    for (int t = blockIdx.x; t < tiles; t += gridDim.x) {
-      const long long base = (static_cast<long long>(t) * kTileVecs + tid) * EPV;
+    const long long n_steps = (static_cast<long long>(tiles) * kTileVecs + kSelThreads - 1) / kSelThreads;
+    for (long long s = blockIdx.x; s < n_steps; s += gridDim.x) {
+      const long long vec = s * kSelThreads + tid;
+      const long long t = vec / kTileVecs;
+      const long long base = vec * EPV;
       uint32_t g = 0, q = 0;
       if (base + EPV <= n) {
         const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + base));
@@ -536,7 +542,7 @@ count_kernel(const void* __restrict__ xv, long long n, SelectState* __restrict__
       }
       g = __reduce_add_sync(kFull, g);
       q = __reduce_add_sync(kFull, q);
-      if (lane == 0) {
+      if (lane == 0 && t < tiles) {
         if (g) atomicAdd(&full_gt[t], g);
         if (q) atomicAdd(&full_eq[t], q);
       }
@@ -600,9 +606,10 @@ count_kernel(const void* __restrict__ xv, long long n, SelectState* __restrict__
 // ---- compaction -----------------------------------------------------------------------------
 
 constexpr unsigned long long kCountMask = 0x7FFFFFFFull;
-constexpr int kCompactThreads = 256;
 constexpr int kRows = 4;                 // rows of 32 lanes x 16 bytes per warp
-static_assert(8 * kRows * 32 == kTileVecs, "compaction tile");
+constexpr int kTileWarps = kTileVecs / (kRows * 32);   // warps of the generic per-tile kernels
+static_assert(kTileWarps * kRows * 32 == kTileVecs, "compaction tile");
+constexpr int kCompactThreads = kTileWarps * 32;
 
 // Keep only the lowest `allowed` set bits of `m`.
 __device__ __forceinline__ uint32_t lowest_set_bits(uint32_t m, long long allowed) {
@@ -635,14 +642,14 @@ __device__ __forceinline__ void compact_tile(const typename Elem<DT>::type* __re
   constexpr int LPW = 32 / EPV;                // lanes per bitmap word: 8 / 4
   constexpr int BPR = ROW / SURGEON_BLOCK;     // offset blocks per row: 1 / 2
   constexpr uint32_t kEMask = (1u << EPV) - 1u;
-  __shared__ uint32_t s_gt[8], s_eq[8];
+  __shared__ uint32_t s_gt[kTileWarps], s_eq[kTileWarps];
   const uint32_t lane = lane_id();
   const int warp = threadIdx.x >> 5;
   const long long n_blocks = (n + SURGEON_BLOCK - 1) >> kBlockShift;
   const long long n_words = (n + 31) / 32;
   const int my_word = lane / LPW;
   const int my_shift = EPV * (lane % LPW);
-  const long long row0 = (static_cast<long long>(tile) * 8 + warp) * kRows;
+  const long long row0 = (static_cast<long long>(tile) * kTileWarps + warp) * kRows;
 
   // per row and lane EPV decisions: g = kept for sure, e = tie at the threshold (SLOW only)
   uint32_t g_all = 0, e_all = 0;      // kRows fields of EPV bits
@@ -673,7 +680,7 @@ __device__ __forceinline__ void compact_tile(const typename Elem<DT>::type* __re
 
   long long gt_before = gt_tile_before, eq_before = eq_tile_before;
 #pragma unroll
-  for (int w = 0; w < 8; ++w) {
+  for (int w = 0; w < kTileWarps; ++w) {
     if (w < warp) { gt_before += s_gt[w]; eq_before += s_eq[w]; }
   }
   // kept before = all greater + the ties that fit the quota.  In the fast path the kept ties of
@@ -774,7 +781,7 @@ __device__ __forceinline__ void load_tile(const typename Elem<DT>::type* __restr
                                           long long n, int tile, uint4 (&q)[kRows]) {
   constexpr int EPV = 16 / sizeof(typename Elem<DT>::type);
   constexpr int ROW = 32 * EPV;
-  const long long row0 = (static_cast<long long>(tile) * 8 + (threadIdx.x >> 5)) * kRows;
+  const long long row0 = (static_cast<long long>(tile) * kTileWarps + (threadIdx.x >> 5)) * kRows;
 #pragma unroll
   for (int r = 0; r < kRows; ++r) {
     const long long base = (row0 + r) * ROW + static_cast<long long>(lane_id()) * EPV;
@@ -792,11 +799,11 @@ __device__ __forceinline__ void load_tile(const typename Elem<DT>::type* __restr
   }
 }
 
-// One CTA per tile.  The one tile inside which the tie quota ends (if any) is left to
-// compact_boundary_kernel.
+// One small CTA per tile: used for tensors too small for the streaming kernel.  The one tile
+// inside which the tie quota ends (if any) is left to compact_boundary_kernel.
 template <int DT>
 __global__ void __launch_bounds__(kCompactThreads)
-compact_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restrict__ hdr,
+compact_small_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restrict__ hdr,
                uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
                uint32_t* __restrict__ offsets, const unsigned long long* __restrict__ prefix) {
   using E = typename Elem<DT>::type;
@@ -825,6 +832,8 @@ compact_boundary_kernel(const void* __restrict__ xv, long long n, surgeon_header
   using E = typename Elem<DT>::type;
   const E* __restrict__ x = reinterpret_cast<const E*>(xv);
   const long long quota = hdr->tie_quota;
+  if (threadIdx.x == 0)   // the sentinel entry of the block offsets
+    offsets[(n + SURGEON_BLOCK - 1) >> kBlockShift] = static_cast<uint32_t>(hdr->n_keep);
   // first tile whose inclusive tie count exceeds the quota (the counts never decrease)
   int lo = 0, hi = tiles;
   while (lo < hi) {
@@ -841,6 +850,220 @@ compact_boundary_kernel(const void* __restrict__ xv, long long n, surgeon_header
   compact_tile<DT, true>(x, n, q, lo, hdr->threshold_key, quota, false,
                          static_cast<long long>(pb >> 31), eq_b, hdr, bitmap,
                          reinterpret_cast<E*>(values_v), offsets);
+}
+
+// ---- streaming compaction ---------------------------------------------------------------------
+// Persistent CTAs.  One producer thread keeps a ring of 32 KB stages full with 2-D TMA loads of
+// [256 rows x 128 bytes] (128-byte swizzle, so that 32 lanes can each read their own row without
+// bank conflicts).  Each of the 8 consumer warps owns one 4 KB chunk of a stage; each LANE owns
+// one 128-byte row of it, i.e. 32 (fp32) or 64 (bf16) consecutive elements, and builds their
+// bitmap word(s) with no cross-lane traffic.  One warp scan places the lanes' kept values; they
+// are gathered in the warp's part of the stage (in place) and leave as 16-byte vectors.
+constexpr int kCsWarps = 8;
+constexpr int kCsThreads = (kCsWarps + 1) * 32;
+constexpr int kCsStageRows = kCsWarps * 32;
+constexpr int kCsStageBytes = kCsStageRows * 128;
+constexpr int kCsStages = 3;
+constexpr size_t kCsSmem = static_cast<size_t>(kCsStages) * kCsStageBytes + 1024;
+static_assert(kCsStageRows * 128 / 16 == kCsWarps * kTileVecs, "a warp's 32 rows are one chunk");
+
+template <int DT>
+__global__ void __launch_bounds__(kCsThreads, 2)
+compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict__ xv,
+                      long long n, long long n_rows_full, surgeon_header* __restrict__ hdr,
+                      uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
+                      uint32_t* __restrict__ offsets, const unsigned long long* __restrict__ prefix,
+                      int n_chunks, int n_stage_tiles) {
+  using E = typename Elem<DT>::type;
+  constexpr uint32_t kMask = Elem<DT>::kKeyMask;
+  constexpr int EPR = 128 / sizeof(E);         // elements per row (= per lane): 32 / 64
+  constexpr int EPV = 16 / sizeof(E);          // elements per 16-byte vector: 4 / 8
+  constexpr int WPL = EPR / 32;                // bitmap words per lane: 1 / 2
+  constexpr int BPC = 32 * EPR / SURGEON_BLOCK;   // offset blocks per chunk: 8 / 16
+  constexpr int LPB = 32 / BPC;                // lanes per offset block: 4 / 2
+  extern __shared__ __align__(1024) unsigned char cs_smem_raw[];
+  unsigned char* ring = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(cs_smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  __shared__ __align__(8) unsigned long long bars[2 * kCsStages];
+  const E* __restrict__ x = reinterpret_cast<const E*>(xv);
+  E* __restrict__ values = reinterpret_cast<E*>(values_v);
+  const int warp = threadIdx.x >> 5;
+  const uint32_t lane = lane_id();
+  const uint32_t full_bar = smem_u32(bars);
+  const uint32_t empty_bar = smem_u32(bars + kCsStages);
+  if (threadIdx.x == 0) {
+    tc::tma_prefetch_desc(&xmap);
+    for (int s = 0; s < kCsStages; ++s) {
+      tc::mbar_init(full_bar + 8 * s, 1);
+      tc::mbar_init(empty_bar + 8 * s, kCsWarps);
+    }
+    tc::fence_barrier_init();
+  }
+  __syncthreads();
+  const int first = blockIdx.x;
+  const int n_it = first < n_stage_tiles ? (n_stage_tiles - 1 - first) / static_cast<int>(gridDim.x) + 1 : 0;
+
+  if (warp == kCsWarps) {
+    // ---- producer ----
+    if (lane == 0) {
+      for (int it = 0; it < n_it; ++it) {
+        const int s = it % kCsStages;
+        if (it >= kCsStages && !tc::mbar_wait(empty_bar + 8 * s, ((it / kCsStages) - 1) & 1, 20)) {
+          atomicMax(&hdr->status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+          break;
+        }
+        const int t = first + it * static_cast<int>(gridDim.x);
+        tc::mbar_arrive_expect_tx(full_bar + 8 * s, kCsStageBytes);
+        tc::tma_load_2d(smem_u32(ring + s * kCsStageBytes), &xmap, 0, t * kCsStageRows,
+                        full_bar + 8 * s);
+      }
+    }
+    return;
+  }
+
+  // ---- consumers ----
+  const uint32_t tau = hdr->threshold_key;
+  const long long quota = hdr->tie_quota;
+  const bool none = hdr->n_keep == 0;
+  const long long n_words = (n + 31) / 32;
+  const long long n_blocks = (n + SURGEON_BLOCK - 1) >> kBlockShift;
+  auto chunk_of = [&](int it) { return (first + it * static_cast<int>(gridDim.x)) * kCsWarps + warp; };
+  unsigned long long pb = 0, pe = 0;    // scan entries of this iteration's chunk, fetched one ahead
+  if (n_it > 0 && chunk_of(0) < n_chunks) { pb = prefix[chunk_of(0)]; pe = prefix[chunk_of(0) + 1]; }
+  for (int it = 0; it < n_it; ++it) {
+    const int s = it % kCsStages;
+    const int chunk = chunk_of(it);
+    unsigned long long pb_next = 0, pe_next = 0;
+    if (it + 1 < n_it && chunk_of(it + 1) < n_chunks) {
+      pb_next = prefix[chunk_of(it + 1)];
+      pe_next = prefix[chunk_of(it + 1) + 1];
+    }
+    if (!tc::mbar_wait(full_bar + 8 * s, (it / kCsStages) & 1, 20)) {
+      if (lane == 0) atomicMax(&hdr->status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+      break;
+    }
+    unsigned char* region = ring + s * kCsStageBytes + warp * 4096;   // this warp's 32 rows
+    const long long eq_b = static_cast<long long>(pb & kCountMask);
+    const long long eq_e = static_cast<long long>(pe & kCountMask);
+    const bool boundary = eq_b < quota && eq_e > quota;   // left to compact_boundary_kernel
+    if (chunk < n_chunks && !boundary) {
+      // ---- this lane's row: 8 vectors, un-swizzled ----
+      uint4 q[8];
+      const unsigned char* row = region + lane * 128;
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        q[j] = *reinterpret_cast<const uint4*>(row + ((j ^ (lane & 7)) << 4));
+      const long long grow = static_cast<long long>(chunk) * 32 + lane;   // row index in the tensor
+      const long long e0 = grow * EPR;
+      long long nv = n - e0;                      // valid elements of the row
+      nv = nv < 0 ? 0 : (nv > EPR ? EPR : nv);
+      if (grow >= n_rows_full && nv > 0) {        // the ragged last row is not covered by the map
+        uint32_t t[64];
+#pragma unroll
+        for (int i = 0; i < 64; ++i) t[i] = (i < EPR && i < nv) ? static_cast<uint32_t>(x[e0 + i]) : 0u;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (DT == 0) q[j] = make_uint4(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3]);
+          else q[j] = make_uint4(t[8 * j] | (t[8 * j + 1] << 16), t[8 * j + 2] | (t[8 * j + 3] << 16),
+                                 t[8 * j + 4] | (t[8 * j + 5] << 16), t[8 * j + 6] | (t[8 * j + 7] << 16));
+        }
+      }
+      // ---- one decision per element: key >= thr ----
+      const bool ties = eq_e <= quota;            // every tie of this chunk is kept (else none is)
+      const uint32_t thr = ties ? tau : tau + 1u;
+      uint32_t word[WPL];
+#pragma unroll
+      for (int w = 0; w < WPL; ++w) word[w] = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t c[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (DT == 0) {
+            word[0] |= ((c[i] & kMask) >= thr ? 1u : 0u) << (4 * j + i);
+          } else {
+            const int e = 8 * j + 2 * i;          // element index inside the row
+            word[e >> 5] |= ((c[i] & kMask) >= thr ? 1u : 0u) << (e & 31);
+            word[e >> 5] |= (((c[i] >> 16) & kMask) >= thr ? 1u : 0u) << ((e + 1) & 31);
+          }
+        }
+      }
+#pragma unroll
+      for (int w = 0; w < WPL; ++w) {
+        const long long left = nv - 32 * w;
+        const uint32_t vmask = left >= 32 ? 0xFFFFFFFFu : (left <= 0 ? 0u : ((1u << left) - 1u));
+        word[w] = none ? 0u : (word[w] & vmask);
+      }
+      uint32_t cnt = 0;
+#pragma unroll
+      for (int w = 0; w < WPL; ++w) cnt += __popc(word[w]);
+      uint32_t incl = cnt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t up = __shfl_up_sync(kFull, incl, o);
+        if (lane >= static_cast<uint32_t>(o)) incl += up;
+      }
+      const uint32_t lane_pre = incl - cnt;
+      const uint32_t total = __shfl_sync(kFull, incl, 31);
+      const long long kept_before = static_cast<long long>(pb >> 31) + (eq_b < quota ? eq_b : quota);
+
+      // ---- bitmap words and block offsets: coalesced ----
+#pragma unroll
+      for (int w = 0; w < WPL; ++w) {
+        const long long wi = static_cast<long long>(chunk) * 32 * WPL + lane * WPL + w;
+        if (wi < n_words) bitmap[wi] = word[w];
+      }
+      const uint32_t off = __shfl_sync(kFull, lane_pre, (lane * LPB) & 31);
+      const long long blk = static_cast<long long>(chunk) * BPC + lane;
+      if (lane < BPC && blk < n_blocks) offsets[blk] = static_cast<uint32_t>(kept_before) + off;
+
+      // ---- kept values: gathered in place (packed order), then out as 16-byte vectors ----
+      __syncwarp();                                // every lane has its row in registers
+      E* outp = reinterpret_cast<E*>(region);
+      uint32_t pos = lane_pre;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t c[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (DT == 0) {
+            if ((word[0] >> (4 * j + i)) & 1u) outp[pos++] = static_cast<E>(c[i]);
+          } else {
+            const int e = 8 * j + 2 * i;
+            if ((word[e >> 5] >> (e & 31)) & 1u) outp[pos++] = static_cast<E>(c[i] & 0xFFFFu);
+            if ((word[e >> 5] >> ((e + 1) & 31)) & 1u) outp[pos++] = static_cast<E>(c[i] >> 16);
+          }
+        }
+      }
+      __syncwarp();
+      E* dst = values + kept_before;
+      const uint32_t mis = static_cast<uint32_t>(kept_before % EPV);
+      uint32_t head = mis ? EPV - mis : 0;
+      if (head > total) head = total;
+      const uint32_t n_vec = (total - head) / EPV;
+      if (lane < head) dst[lane] = outp[lane];
+      for (uint32_t v = lane; v < n_vec; v += 32) {
+        const E* src = outp + head + v * EPV;
+        uint4 o;
+        if (DT == 0) {
+          o = make_uint4(src[0], src[1], src[2], src[3]);
+        } else {
+          o = make_uint4(src[0] | (static_cast<uint32_t>(src[1]) << 16),
+                         src[2] | (static_cast<uint32_t>(src[3]) << 16),
+                         src[4 % EPV] | (static_cast<uint32_t>(src[5 % EPV]) << 16),
+                         src[6 % EPV] | (static_cast<uint32_t>(src[7 % EPV]) << 16));
+        }
+        *reinterpret_cast<uint4*>(dst + head + v * EPV) = o;
+      }
+      const uint32_t done = head + n_vec * EPV;
+      if (lane < total - done) dst[done + lane] = outp[done + lane];
+    }
+    tc::fence_proxy_async();     // this warp's writes to the stage precede the next TMA fill
+    __syncwarp();
+    if (lane == 0) tc::mbar_arrive(empty_bar + 8 * s);
+    pb = pb_next;
+    pe = pe_next;
+  }
 }
 
 __global__ void offsets_empty_kernel(uint32_t* offsets) { offsets[0] = 0u; }
@@ -911,6 +1134,9 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
     e = cudaFuncSetAttribute(hist_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(kHistSmem));
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(compact_stream_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(kCsSmem));
+    if (e != cudaSuccess) return e;
     attrs_done = true;
   }
 
@@ -961,8 +1187,34 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
     offsets_empty_kernel<<<1, 1, 0, stream>>>(out.block_offsets);
     note_launches(1);
   } else {
-    compact_kernel<DT><<<static_cast<unsigned>(L.tiles), kCompactThreads, 0, stream>>>(
-        x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix);
+    const long long n_rows_full = n * static_cast<long long>(sizeof(typename Elem<DT>::type)) / 128;
+    bool streamed = false;
+    if (n_rows_full >= kCsStageRows) {
+      using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                    const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                    const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+      const EncodeFn encode = reinterpret_cast<EncodeFn>(tensor_map_encode_fn());
+      CUtensorMap map;
+      const cuuint64_t dims[2] = {32, static_cast<cuuint64_t>(n_rows_full)};
+      const cuuint64_t strides[1] = {128};
+      const cuuint32_t box[2] = {32, static_cast<cuuint32_t>(kCsStageRows)};
+      const cuuint32_t estr[2] = {1, 1};
+      if (encode &&
+          encode(&map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(x), dims, strides, box,
+                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS) {
+        const int n_stage_tiles = static_cast<int>((L.tiles + kCsWarps - 1) / kCsWarps);
+        const int grid = n_stage_tiles < 2 * sms ? n_stage_tiles : 2 * sms;
+        compact_stream_kernel<DT><<<grid, kCsThreads, kCsSmem, stream>>>(
+            map, x, n, n_rows_full, out.header, out.bitmap, out.values, out.block_offsets, prefix,
+            static_cast<int>(L.tiles), n_stage_tiles);
+        streamed = true;
+      }
+    }
+    if (!streamed)
+      compact_small_kernel<DT><<<static_cast<unsigned>(L.tiles), kCompactThreads, 0, stream>>>(
+          x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix);
     compact_boundary_kernel<DT><<<1, kCompactThreads, 0, stream>>>(
         x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix,
         static_cast<int>(L.tiles));

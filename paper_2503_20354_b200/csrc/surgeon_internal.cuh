@@ -29,9 +29,10 @@ constexpr int kBlockWords = SURGEON_BLOCK / 32;      // bitmap words per offset 
 static_assert((1 << kBlockShift) == SURGEON_BLOCK, "SURGEON_BLOCK must be 128");
 
 // ---- scratch of surgeon_prune_compact ---------------------------------------------------------
-// Compaction tile = 1024 16-byte vectors: 8 warps x 4 rows of 32 lanes x 16 bytes.
-constexpr int kTileVecs = 1024;
-constexpr int64_t compact_tile_elems(int dt) { return dt == 0 ? 4096 : 8192; }
+// Compaction tile ("chunk") = 4 KB of input = 256 16-byte vectors: the unit one warp emits and
+// the unit of the exclusive scan that places it.
+constexpr int kTileVecs = 256;
+constexpr int64_t compact_tile_elems(int dt) { return dt == 0 ? 1024 : 2048; }
 constexpr int kBuckets = 32768;        // histogram bins of the select pass (top 15 key bits)
 constexpr int kLowBins = 65536;        // bins of the fp32 refinement (low 16 key bits)
 constexpr int64_t kSampleMinN = 65536; // tensors up to this size list every non-zero element
@@ -100,6 +101,9 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
                                   const float* grad_out, float* dw, int accumulate,
                                   void* workspace, cudaStream_t stream);
 
+// The driver's cuTensorMapEncodeTiled, looked up through the runtime (the library carries no
+// link-time dependency on the driver library); nullptr if unavailable.
+void* tensor_map_encode_fn();
 // Number of SMs of the current device (cached per device id).
 int sm_count();
 // Adds to the process-wide kernel-launch counter behind surgeon_launch_count().

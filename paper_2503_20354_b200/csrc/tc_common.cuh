@@ -61,6 +61,15 @@ __device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gsrc, u
       ::"r"(smem_dst), "l"(gsrc), "r"(bytes), "r"(bar)
       : "memory");
 }
+// TMA: 2-D tiled load global -> shared, completion counted in bytes on an mbarrier.
+__device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const void* tmap, int x, int y,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_dst), "l"(tmap), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }

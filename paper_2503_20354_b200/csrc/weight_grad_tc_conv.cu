@@ -425,22 +425,12 @@ grad_to_bf16_kernel(const float* __restrict__ g, long long n, unsigned short* __
       out[j] = static_cast<unsigned short>(pack_bf16x2(g[j], 0.0f) & 0xFFFFu);
 }
 
-// The driver's tensor-map encoder, looked up through the runtime so that the library carries no
-// link-time dependency on the driver library (it must load on machines without a GPU).
 using TensorMapEncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                        const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
                                        const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                        CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 TensorMapEncodeFn tensor_map_encoder() {
-  static TensorMapEncodeFn fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    return reinterpret_cast<TensorMapEncodeFn>(p);
-  }();
-  return fn;
+  return reinterpret_cast<TensorMapEncodeFn>(tensor_map_encode_fn());
 }
 
 }  // namespace
