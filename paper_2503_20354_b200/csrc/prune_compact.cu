@@ -4,29 +4,28 @@
 // at the threshold broken by lowest flat index.  Its decompose step / Section 4.2: the pruned
 // activation is cached as the vector of kept elements plus one index bit per element.
 //
-// The tensor is read twice: once to find the threshold, once to emit the store.  No kernel waits
-// on another CTA: everything the emitting pass needs to place a tile's output (how many elements
-// before the tile are kept, how many ties precede it) is counted during the first read.
+// The tensor is read twice: once to find the threshold, once to emit the store.  No CTA of the
+// emitting pass waits on another: everything it needs to place a chunk's output (how many
+// elements before the chunk are kept, how many ties precede it) is counted during the first read.
+// Both reads are persistent kernels fed by TMA into a shared-memory ring, in which every lane owns
+// 128 consecutive bytes, so bitmap words are built without cross-lane traffic.
 //
-//   sample   : a strided sample (about 1/32 of the tensor) gives a bracket [blo, bhi] of
-//              histogram buckets that contains the threshold with overwhelming probability.
-//   histogram: one streaming read, fed by bulk asynchronous copies into a shared-memory ring.
-//              A 32768-bin shared-memory histogram over the top 15 key bits gives the exact
-//              bucket b1 of the threshold (for bf16 the key has 15 bits, so that is the
-//              threshold itself).  The same read counts, per compaction tile, the keys above the
-//              bracket and the exact zeros, and appends every key inside the bracket, tagged
-//              with its tile, to a candidate list (1-3 % of the elements).
-//   refine   : fp32 only; a 65536-bin histogram over the low 16 bits of the listed keys of
-//              bucket b1 fixes the threshold.
-//   count    : the listed keys above / equal to the threshold are added to the per-tile counts;
-//              the last CTA turns the counts into an exclusive scan over tiles.
-//   compact  : one streaming read with 128-bit loads; a tile's CTA starts from its entry of the
-//              scan, builds bitmap words with warp OR-reductions, stages the kept values in
-//              shared memory and stores them as aligned 16-byte vectors.
+//   sample   : a strided sample (about 1/32 of the tensor) gives a bracket [lo_key, hi_key] of
+//              keys that contains the threshold with overwhelming probability and holds 1-3 %
+//              of the elements.
+//   classify : the first read.  Per 4 KB chunk: the number of keys above the bracket, the number
+//              inside, and the keys inside themselves (the chunk's slot).  Its last CTA decides
+//              where the threshold lies and, for bf16, which key it is.
+//   count    : fp32 resolves the threshold among the listed keys with two histogram levels;
+//              then the listed keys above / equal to the threshold complete the per-chunk counts,
+//              and an exclusive scan over chunks follows (cooperative launch, grid barriers).
+//   compact  : the second read.  A chunk's warp starts from its entry of the scan.  The one chunk
+//              inside which the tie quota ends is emitted by a separate small kernel that ranks
+//              ties by flat index.
 //
-// If the threshold's bucket falls outside the bracket, or the list overflows (massive ties at a
-// non-zero value), refine and count read the tensor once more instead of the list.  The result
-// is exact and unique either way; only the cost differs.
+// If the threshold falls outside the bracket, a slot overflows (massive ties at a non-zero
+// value) or the tensor is small, the count kernel runs an exact radix select over the tensor
+// and counts the chunks from the tensor.  The result is exact and unique either way.
 // Every count fits 32 bits because n <= SURGEON_MAX_N < 2^31.
 #include <cuda.h>
 
@@ -41,19 +40,7 @@ using tc::smem_u32;
 
 constexpr int kSelThreads = 1024;
 constexpr uint32_t kFull = 0xFFFFFFFFu;
-// Histogram pass: 31 consumer warps read what one producer thread streams into a ring of stages
-// with bulk asynchronous copies; a stage holds one 16-byte vector per consumer thread.
-constexpr int kHistConsumerWarps = 31;
-constexpr int kStageVecs = kHistConsumerWarps * 32;
-constexpr int kStageBytes = kStageVecs * 16;
-constexpr int kHistStages = 3;
-constexpr int kWarpBuf = 192;          // candidate staging entries per warp
-constexpr int kFlushAt = 64;           // a half vector adds at most 128 entries
 constexpr int kHistWords = kBuckets + 32;   // + one private bin per lane that swallows zeros
-constexpr size_t kHistSmem = static_cast<size_t>(kHistWords) * 4 + kHistStages * kStageBytes +
-                             static_cast<size_t>(kHistConsumerWarps) * kWarpBuf * 8;
-static_assert((kHistWords * 4) % 128 == 0, "ring alignment");
-
 __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
@@ -172,6 +159,7 @@ sample_kernel(const uint4* __restrict__ xq, long long n, uint32_t k, uint32_t n_
       const uint32_t key = bits & kMask;
       const bool isz = key == 0;
       zero_cnt += isz ? 1u : 0u;
+      // zeros (half of post-ReLU data) go to a bin private to the lane: no conflicts, no branch
       atomicAdd(&hist[isz ? kBuckets + lane : (DT == 0 ? key >> 16 : key)], 1u);
     }
   }
@@ -203,256 +191,286 @@ sample_kernel(const uint4* __restrict__ xq, long long n, uint32_t k, uint32_t n_
     find_from_top<kBuckets>(ld, static_cast<uint32_t>(r + delta) + 1u, scratch, res);
     blo = res[0];
   }
-  if (tid == 0) { st->blo = blo; st->bhi = bhi; }
+  if (tid == 0) {
+    st->blo = blo;
+    st->bhi = bhi;
+    // the bracket as keys; key 0 (exact zeros) is never a candidate
+    const uint32_t lo = (DT == 0) ? (blo << 16) : blo;
+    st->lo_key = lo < 1u ? 1u : lo;
+    st->hi_key = (DT == 0) ? ((bhi << 16) | 0xFFFFu) : bhi;
+    st->mode = (bhi - blo + 1u > static_cast<uint32_t>(kMaxSpan)) ? 1u : 0u;
+  }
+}
+
+// ---- geometry shared by the two streaming kernels -----------------------------------------------
+// Persistent CTAs.  One producer thread keeps a ring of 32 KB stages full with 2-D TMA loads of
+// [256 rows x 128 bytes] (128-byte swizzle, so that 32 lanes can each read their own row without
+// bank conflicts).  Each of the 8 consumer warps owns one 4 KB chunk of a stage; each LANE owns
+// one 128-byte row of it, i.e. 32 (fp32) or 64 (bf16) consecutive elements.
+constexpr int kCsWarps = 8;
+constexpr int kCsThreads = (kCsWarps + 1) * 32;
+constexpr int kCsStageRows = kCsWarps * 32;
+constexpr int kCsStageBytes = kCsStageRows * 128;
+constexpr int kCsStages = 3;
+constexpr size_t kCsSmem = static_cast<size_t>(kCsStages) * kCsStageBytes + 1024;
+static_assert(kCsStageRows * 128 / 16 == kCsWarps * kTileVecs, "a warp's 32 rows are one chunk");
+
+// This lane's row (8 vectors) out of the swizzled stage; the ragged last row of the tensor, which
+// the tensor map does not cover, comes from global memory.  Returns the row's valid element count.
+template <int DT>
+__device__ __forceinline__ int load_row(const unsigned char* region, const typename Elem<DT>::type* x,
+                                        long long n, long long n_rows_full, long long grow,
+                                        uint4 (&q)[8]) {
+  constexpr int EPR = 128 / sizeof(typename Elem<DT>::type);
+  const uint32_t lane = lane_id();
+  const unsigned char* row = region + lane * 128;
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    q[j] = *reinterpret_cast<const uint4*>(row + ((j ^ (lane & 7)) << 4));
+  const long long e0 = grow * EPR;
+  long long nv = n - e0;
+  nv = nv < 0 ? 0 : (nv > EPR ? EPR : nv);
+  if (grow >= n_rows_full && nv > 0) {
+    uint32_t t[64];
+#pragma unroll
+    for (int i = 0; i < 64; ++i) t[i] = (i < EPR && i < nv) ? static_cast<uint32_t>(x[e0 + i]) : 0u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (DT == 0) q[j] = make_uint4(t[4 * j], t[4 * j + 1], t[4 * j + 2], t[4 * j + 3]);
+      else q[j] = make_uint4(t[8 * j] | (t[8 * j + 1] << 16), t[8 * j + 2] | (t[8 * j + 3] << 16),
+                             t[8 * j + 4] | (t[8 * j + 5] << 16), t[8 * j + 6] | (t[8 * j + 7] << 16));
+    }
+  }
+  return static_cast<int>(nv);
+}
+__device__ __forceinline__ uint32_t valid_mask(int nv, int w) {
+  const int left = nv - 32 * w;
+  return left >= 32 ? 0xFFFFFFFFu : (left <= 0 ? 0u : ((1u << left) - 1u));
 }
 
 // ---- the select's read of the tensor ---------------------------------------------------------
+// Per chunk: how many keys lie above the bracket, how many inside; the keys inside go to the
+// chunk's slot.  A level-A histogram of the keys inside (relative to lo_key) is kept per CTA.
+// The last CTA places the threshold: above the bracket or a full slot -> fall back; inside ->
+// bin of level A (bf16: the threshold itself); below, with lo_key == 1 -> the threshold is 0.
 template <int DT>
-__global__ void __launch_bounds__(kSelThreads, 1)
-hist_kernel(const void* __restrict__ xv, long long n, uint32_t k, int use_bracket,
-            SelectState* __restrict__ st, uint32_t* __restrict__ ghist,
-            uint32_t* __restrict__ hist2, uint32_t* __restrict__ cnt_gt,
-            uint32_t* __restrict__ cnt_zero, unsigned long long* __restrict__ list,
-            uint32_t list_cap, surgeon_header* __restrict__ hdr) {
+__global__ void __launch_bounds__(kCsThreads, 2)
+classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict__ xv, long long n,
+                long long n_rows_full, uint32_t k, SelectState* __restrict__ st,
+                uint32_t* __restrict__ hist_a, uint32_t* __restrict__ cnt_gt,
+                uint32_t* __restrict__ cand_cnt, void* __restrict__ slots_v,
+                surgeon_header* __restrict__ hdr, int n_chunks, int n_stage_tiles) {
   using E = typename Elem<DT>::type;
   constexpr uint32_t kMask = Elem<DT>::kKeyMask;
-  constexpr int VEC = 16 / sizeof(E);
-  // dynamic shared memory: hist[kHistWords] | ring[kHistStages][kStageBytes] | wbuf[31][kWarpBuf]
-  extern __shared__ __align__(128) uint32_t hist[];
-  __shared__ __align__(8) unsigned long long bars[2 * kHistStages];
-  __shared__ uint32_t scratch[32];
-  __shared__ uint32_t s_wcnt[32];
-  __shared__ uint32_t res[2];
+  constexpr int EPR = 128 / sizeof(E);
+  constexpr int WPL = EPR / 32;
+  constexpr int kSlot = (DT == 0) ? 64 : 128;
+  constexpr int kShiftA = (DT == 0) ? 12 : 0;
+  extern __shared__ __align__(1024) unsigned char cs_smem_raw[];
+  unsigned char* ring = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(cs_smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  __shared__ __align__(8) unsigned long long bars[2 * kCsStages];
+  __shared__ uint32_t s_hist[kBinsA];
+  __shared__ uint32_t s_tot[2];
   __shared__ bool s_last;
+  const E* __restrict__ x = reinterpret_cast<const E*>(xv);
+  E* __restrict__ slots = reinterpret_cast<E*>(slots_v);   // fp32: 32-bit keys, bf16: 16-bit keys
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
   const uint32_t lane = lane_id();
-  unsigned char* ring = reinterpret_cast<unsigned char*>(hist + kHistWords);
-  unsigned long long* wbuf =
-      reinterpret_cast<unsigned long long*>(ring + kHistStages * kStageBytes) + warp * kWarpBuf;
+  if (st->mode == 1u) return;          // the sample found no usable bracket
+  const uint32_t lo_key = st->lo_key, hi_key = st->hi_key;
+  const uint32_t range = hi_key - lo_key;
   const uint32_t full_bar = smem_u32(bars);
-  const uint32_t empty_bar = smem_u32(bars + kHistStages);
+  const uint32_t empty_bar = smem_u32(bars + kCsStages);
   if (tid == 0) {
-    for (int s = 0; s < kHistStages; ++s) {
+    tc::tma_prefetch_desc(&xmap);
+    for (int s = 0; s < kCsStages; ++s) {
       tc::mbar_init(full_bar + 8 * s, 1);
-      tc::mbar_init(empty_bar + 8 * s, kHistConsumerWarps);
+      tc::mbar_init(empty_bar + 8 * s, kCsWarps);
     }
     tc::fence_barrier_init();
+    s_tot[0] = 0;
+    s_tot[1] = 0;
   }
-  zero_hist_smem(hist);
-  if (lane == 0) s_wcnt[warp] = 0;
+  for (int i = tid; i < kBinsA; i += kCsThreads) s_hist[i] = 0;
   __syncthreads();
+  const int first = blockIdx.x;
+  const int n_it = first < n_stage_tiles ? (n_stage_tiles - 1 - first) / static_cast<int>(gridDim.x) + 1 : 0;
 
-  uint32_t blo = 0, bhi = kBuckets - 1;
-  if (use_bracket) { blo = st->blo; bhi = st->bhi; }
-  const uint32_t span = bhi - blo;
-  uint32_t zero_total = 0;
-
-  // Candidate staging: lanes append through a per-warp cursor in shared memory; the buffer goes
-  // to the global list once it holds kFlushAt entries.
-  auto maybe_flush = [&](uint32_t limit) {
-    __syncwarp();
-    const uint32_t cnt = *reinterpret_cast<volatile uint32_t*>(&s_wcnt[warp]);
-    if (cnt >= limit && cnt > 0) {
-      uint32_t base = 0;
-      if (lane == 0) base = atomicAdd(&st->list_count, cnt);
-      base = __shfl_sync(kFull, base, 0);
-      for (uint32_t i = lane; i < cnt; i += 32) {
-        if (base + i < list_cap) list[base + i] = wbuf[i];
-        else st->list_overflow = 1u;
-      }
-      __syncwarp();
-      if (lane == 0) s_wcnt[warp] = 0;
-      __syncwarp();
-    }
-  };
-  uint32_t above_v = 0, zero_v = 0;   // per vector and lane: keys above the bracket, exact zeros
-  unsigned long long tile_tag = 0;    // tile index << 32
-  auto add = [&](uint32_t bits) {
-    const uint32_t key = bits & kMask;
-    const uint32_t bucket = (DT == 0) ? (key >> 16) : key;
-    const bool isz = key == 0;
-    zero_v += isz ? 1u : 0u;
-    above_v += (bucket > bhi) ? 1u : 0u;
-    // zeros (half of post-ReLU data) go to a bin private to the lane: no conflicts, no branch
-    atomicAdd(&hist[isz ? kBuckets + lane : bucket], 1u);
-    if (!isz && (bucket - blo) <= span) wbuf[atomicAdd(&s_wcnt[warp], 1u)] = tile_tag | key;
-  };
-  auto add_vec = [&](const uint4& q) {
-    if (DT == 0) {
-      add(q.x); add(q.y); add(q.z); add(q.w);
-    } else {
-      add(q.x); add(q.x >> 16); add(q.y); add(q.y >> 16);
-    }
-  };
-  auto add_vec_hi = [&](const uint4& q) {   // bf16: second half of the vector
-    add(q.z); add(q.z >> 16); add(q.w); add(q.w >> 16);
-  };
-  // Per-tile counters of one warp step (all 32 lanes hold elements of the same tile).
-  auto tile_counts = [&](uint32_t tile) {
-    const uint32_t a = __reduce_add_sync(kFull, above_v);
-    const uint32_t z = __reduce_add_sync(kFull, zero_v);
-    if (lane == 0) {
-      if (a) atomicAdd(&cnt_gt[tile], a);
-      if (z) atomicAdd(&cnt_zero[tile], z);
-    }
-    zero_total += zero_v;
-    above_v = 0;
-    zero_v = 0;
-  };
-
-  // Chunks of kStageVecs vectors, handed out from the END of the tensor towards its start: what
-  // this pass leaves in L2 is then the part the compaction pass reads first.
-  const long long nvec = n / VEC;
-  const uint4* __restrict__ xq = reinterpret_cast<const uint4*>(xv);
-  const long long n_chunks = (nvec + kStageVecs - 1) / kStageVecs;
-  const long long first_chunk = n_chunks - 1 - blockIdx.x;
-  const int n_it = first_chunk < 0 ? 0 : static_cast<int>(first_chunk / gridDim.x) + 1;
-  bool timed_out = false;
-  if (warp == kHistConsumerWarps) {
-    // ---- producer: one thread keeps the ring full ----
+  if (warp == kCsWarps) {
+    // ---- producer ----
     if (lane == 0) {
       for (int it = 0; it < n_it; ++it) {
-        const int s = it % kHistStages;
-        if (it >= kHistStages &&
-            !tc::mbar_wait(empty_bar + 8 * s, ((it / kHistStages) - 1) & 1, 20)) {
-          timed_out = true;
+        const int s = it % kCsStages;
+        if (it >= kCsStages && !tc::mbar_wait(empty_bar + 8 * s, ((it / kCsStages) - 1) & 1, 20)) {
+          atomicMax(&st->error, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
           break;
         }
-        const long long v0 = (first_chunk - static_cast<long long>(it) * gridDim.x) * kStageVecs;
-        const long long left = nvec - v0;
-        const uint32_t bytes = static_cast<uint32_t>(left < kStageVecs ? left : kStageVecs) * 16u;
-        tc::mbar_arrive_expect_tx(full_bar + 8 * s, bytes);
-        tc::bulk_load(smem_u32(ring + s * kStageBytes), xq + v0, bytes, full_bar + 8 * s);
+        const int t = first + it * static_cast<int>(gridDim.x);
+        tc::mbar_arrive_expect_tx(full_bar + 8 * s, kCsStageBytes);
+        tc::tma_load_2d(smem_u32(ring + s * kCsStageBytes), &xmap, 0, t * kCsStageRows,
+                        full_bar + 8 * s);
       }
     }
   } else {
     // ---- consumers ----
+    uint32_t w_above = 0, w_cand = 0;
     for (int it = 0; it < n_it; ++it) {
-      const int s = it % kHistStages;
-      if (!tc::mbar_wait(full_bar + 8 * s, (it / kHistStages) & 1, 20)) { timed_out = true; break; }
-      const long long vw = (first_chunk - static_cast<long long>(it) * gridDim.x) * kStageVecs +
-                           warp * 32;                     // first vector of this warp's step
-      const bool valid = vw + lane < nvec;
-      uint4 q = make_uint4(0, 0, 0, 0);
-      if (valid) q = reinterpret_cast<const uint4*>(ring + s * kStageBytes)[warp * 32 + lane];
+      const int s = it % kCsStages;
+      const int chunk = (first + it * static_cast<int>(gridDim.x)) * kCsWarps + warp;
+      if (!tc::mbar_wait(full_bar + 8 * s, (it / kCsStages) & 1, 20)) {
+        if (lane == 0) atomicMax(&st->error, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+        break;
+      }
+      const unsigned char* region = ring + s * kCsStageBytes + warp * 4096;
+      if (chunk < n_chunks) {
+        uint4 q[8];
+        const long long grow = static_cast<long long>(chunk) * 32 + lane;
+        const int nv = load_row<DT>(region, x, n, n_rows_full, grow, q);
+        uint32_t aw[WPL], cw[WPL];
+#pragma unroll
+        for (int w = 0; w < WPL; ++w) { aw[w] = 0; cw[w] = 0; }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t c[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            if (DT == 0) {
+              const uint32_t key = c[i] & kMask;
+              aw[0] |= (key > hi_key ? 1u : 0u) << (4 * j + i);
+              cw[0] |= (key - lo_key <= range ? 1u : 0u) << (4 * j + i);
+            } else {
+              const int e = 8 * j + 2 * i;
+              const uint32_t k0 = c[i] & kMask, k1 = (c[i] >> 16) & kMask;
+              aw[e >> 5] |= (k0 > hi_key ? 1u : 0u) << (e & 31);
+              aw[e >> 5] |= (k1 > hi_key ? 1u : 0u) << ((e + 1) & 31);
+              cw[e >> 5] |= (k0 - lo_key <= range ? 1u : 0u) << (e & 31);
+              cw[e >> 5] |= (k1 - lo_key <= range ? 1u : 0u) << ((e + 1) & 31);
+            }
+          }
+        }
+        uint32_t ac = 0, cc = 0;
+#pragma unroll
+        for (int w = 0; w < WPL; ++w) {
+          const uint32_t vm = valid_mask(nv, w);
+          aw[w] &= vm;
+          cw[w] &= vm;
+          ac += __popc(aw[w]);
+          cc += __popc(cw[w]);
+        }
+        const uint32_t a_tot = __reduce_add_sync(kFull, ac);
+        const uint32_t c_tot = __reduce_add_sync(kFull, cc);
+        if (lane == 0) { cnt_gt[chunk] = a_tot; cand_cnt[chunk] = c_tot; }
+        w_above += a_tot;
+        w_cand += c_tot;
+        if (c_tot > static_cast<uint32_t>(kSlot)) {
+          if (lane == 0) st->list_overflow = 1u;
+        } else if (c_tot) {
+          // keys inside the bracket -> the chunk's slot (order does not matter)
+          uint32_t pos = warp_excl_scan(cc);
+          E* slot = slots + static_cast<long long>(chunk) * kSlot;
+          const bool ragged = grow >= n_rows_full;
+          const unsigned char* row = region + lane * 128;
+#pragma unroll
+          for (int w = 0; w < WPL; ++w) {
+            uint32_t m = cw[w];
+            while (m) {
+              const int e = 32 * w + __ffs(m) - 1;
+              m &= m - 1;
+              uint32_t key;
+              if (ragged) {
+                key = static_cast<uint32_t>(x[grow * EPR + e]) & kMask;
+              } else {
+                const int byte = e * static_cast<int>(sizeof(E));
+                key = static_cast<uint32_t>(*reinterpret_cast<const E*>(
+                          row + (((byte >> 4) ^ (lane & 7)) << 4) + (byte & 15))) & kMask;
+              }
+              slot[pos++] = static_cast<E>(key);
+              atomicAdd(&s_hist[(key - lo_key) >> kShiftA], 1u);
+            }
+          }
+        }
+      }
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(empty_bar + 8 * s);
-      const uint32_t tile = static_cast<uint32_t>(vw / kTileVecs);
-      tile_tag = static_cast<unsigned long long>(tile) << 32;
-      if (valid) add_vec(q);
-      if (DT == 1) {
-        maybe_flush(kFlushAt);
-        if (valid) add_vec_hi(q);
-      }
-      tile_counts(tile);
-      maybe_flush(kFlushAt);
     }
-    if (blockIdx.x == 0 && warp == 0) {   // elements past the last full vector
-      const E* __restrict__ xe = reinterpret_cast<const E*>(xv);
-      const uint32_t tile = static_cast<uint32_t>(nvec / kTileVecs);
-      tile_tag = static_cast<unsigned long long>(tile) << 32;
-      const long long j = nvec * VEC + lane;
-      if (j < n) add(static_cast<uint32_t>(xe[j]));
-      tile_counts(tile);
-    }
-    maybe_flush(1);
-    zero_total = warp_sum(zero_total);
-    if (lane == 0 && zero_total) {
-      atomicAdd(&hist[0], zero_total);
-      atomicAdd(&st->zero_count, zero_total);
+    if (lane == 0) {
+      if (w_above) atomicAdd(&s_tot[0], w_above);
+      if (w_cand) atomicAdd(&s_tot[1], w_cand);
     }
   }
-  if (timed_out) atomicMax(&st->error, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
   __syncthreads();
-  flush_hist(hist, ghist);
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(&st->ticket_hist, 1u) == gridDim.x - 1);
-  __syncthreads();
-  if (!s_last) return;
-
-  // Last CTA: the complete histogram is in ghist.
-  __threadfence();
-  load_hist_to_smem(ghist, hist);
-  __syncthreads();
-  find_from_top<kBuckets>([&](int i) { return hist[i]; }, k, scratch, res);
+  for (int i = tid; i < kBinsA; i += kCsThreads)
+    if (s_hist[i]) atomicAdd(&hist_a[i], s_hist[i]);
   if (tid == 0) {
-    const uint32_t b = res[0], above = res[1];
-    const bool overflow = __ldcg(&st->list_overflow) != 0;
-    const bool inside = b >= blo && b <= bhi;
-    st->b1 = b;
-    st->k1 = k - above;
-    st->above = above;
-    st->mode = (!overflow && inside) ? 0u : 1u;
-    if (DT == 1) {
-      hdr->threshold_key = b;
+    if (s_tot[0]) atomicAdd(&st->above_total, s_tot[0]);
+    if (s_tot[1]) atomicAdd(&st->cand_total, s_tot[1]);
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&st->ticket_classify, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!s_last || warp != 0) return;
+
+  // ---- last CTA, one warp: where does the threshold lie? ----
+  __threadfence();
+  const uint32_t above_total = __ldcg(&st->above_total);
+  const uint32_t n_cand = __ldcg(&st->cand_total);
+  const bool overflow = __ldcg(&st->list_overflow) != 0;
+  const long long r = static_cast<long long>(k) - above_total;     // rank among the rest
+  const long long zeros = (lo_key == 1u) ? n - above_total - n_cand : 0;
+  uint32_t mode, tau = 0, n_greater = 0;
+  if (overflow || r < 1) {
+    mode = 1;
+  } else if (r <= n_cand) {
+    // level A from the top: lane L owns bins [kBinsA - 16(L+1), kBinsA - 16L)
+    constexpr int kPerLane = kBinsA / 32;
+    const int ltop = kBinsA - static_cast<int>(lane) * kPerLane;
+    uint32_t ls = 0;
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i) ls += __ldcg(hist_a + ltop - 1 - i);
+    const uint32_t excl = warp_excl_scan(ls);
+    const uint32_t want = static_cast<uint32_t>(r);
+    uint32_t bin = 0, aboveA = 0;
+    if (excl < want && want <= excl + ls) {
+      uint32_t a = excl;
+      int b = ltop - 1;
+      for (int i = 0; i < kPerLane - 1; ++i, --b) {
+        const uint32_t c = __ldcg(hist_a + b);
+        if (a + c >= want) break;
+        a += c;
+      }
+      bin = static_cast<uint32_t>(b);
+      aboveA = a;
+    }
+    const uint32_t owner = __ffs(__ballot_sync(kFull, excl < want && want <= excl + ls)) - 1;
+    bin = __shfl_sync(kFull, bin, owner);
+    aboveA = __shfl_sync(kFull, aboveA, owner);
+    if (lane == 0) {
+      st->binA = bin;
+      st->aboveA = aboveA;
+      st->rankA = want - aboveA;
+    }
+    mode = (DT == 0) ? 0u : 2u;
+    tau = lo_key + bin;                       // bf16: level A is exact
+    n_greater = above_total + aboveA;
+  } else if (lo_key == 1u && r <= n_cand + zeros) {
+    mode = 2;
+    tau = 0;
+    n_greater = above_total + n_cand;
+  } else {
+    mode = 1;
+  }
+  if (lane == 0) {
+    if (mode == 2) {
+      hdr->threshold_key = tau;
       hdr->status = __ldcg(&st->error);
       hdr->n_keep = k;
-      hdr->n_greater = above;
-      hdr->tie_quota = static_cast<long long>(k) - above;
-    } else if (b == 0) {
-      // exact zeros are never listed or re-read: they enter the refinement here
-      hist2[0] = __ldcg(&st->zero_count);
+      hdr->n_greater = n_greater;
+      hdr->tie_quota = static_cast<long long>(k) - n_greater;
     }
-    __threadfence();
-  }
-}
-
-// ---- fp32: low 16 key bits of the elements in bucket b1 ---------------------------------------
-__global__ void __launch_bounds__(kSelThreads)
-refine_kernel(const uint4* __restrict__ xq, long long n, uint32_t k, SelectState* __restrict__ st,
-              uint32_t* __restrict__ hist2, const unsigned long long* __restrict__ list,
-              uint32_t list_cap, surgeon_header* __restrict__ hdr) {
-  __shared__ uint32_t scratch[32];
-  __shared__ uint32_t res[2];
-  __shared__ bool s_last;
-  const int tid = threadIdx.x;
-  const uint32_t lane = lane_id();
-  const uint32_t b1 = st->b1;
-  const uint32_t mode = st->mode;
-  uint32_t round_cnt = 0;   // keys at the bottom of the bucket (low bits 0): round values tie a lot
-  auto add = [&](uint32_t key) {
-    if (key != 0 && (key >> 16) == b1) {
-      const uint32_t low = key & 0xFFFFu;
-      if (low == 0) ++round_cnt;
-      else atomicAdd(&hist2[low], 1u);
-    }
-  };
-  const long long gtid = static_cast<long long>(blockIdx.x) * kSelThreads + tid;
-  const long long gsz = static_cast<long long>(gridDim.x) * kSelThreads;
-  if (mode == 0) {
-    uint32_t cnt = st->list_count;
-    if (cnt > list_cap) cnt = list_cap;
-    for (long long i = gtid; i < cnt; i += gsz) add(static_cast<uint32_t>(__ldg(list + i)));
-  } else {
-    const long long nvec = n / 4;
-    for (long long v = gtid; v < nvec; v += gsz) {
-      const uint4 q = __ldg(xq + v);
-      add(q.x & 0x7FFFFFFFu); add(q.y & 0x7FFFFFFFu); add(q.z & 0x7FFFFFFFu); add(q.w & 0x7FFFFFFFu);
-    }
-    if (blockIdx.x == 0) {
-      const uint32_t* xe = reinterpret_cast<const uint32_t*>(xq);
-      for (long long j = nvec * 4 + tid; j < n; j += kSelThreads) add(xe[j] & 0x7FFFFFFFu);
-    }
-  }
-  round_cnt = warp_sum(round_cnt);
-  if (lane == 0 && round_cnt) atomicAdd(&hist2[0], round_cnt);
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(&st->ticket_refine, 1u) == gridDim.x - 1);
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  const uint32_t k1 = st->k1;
-  find_from_top<kLowBins>([&](int i) { return __ldcg(hist2 + i); }, k1, scratch, res);
-  if (tid == 0) {
-    const uint32_t ng = st->above + res[1];
-    hdr->threshold_key = (b1 << 16) | res[0];
-    hdr->status = __ldcg(&st->error);
-    hdr->n_keep = k;
-    hdr->n_greater = ng;
-    hdr->tie_quota = static_cast<long long>(k) - ng;
+    st->mode = mode;
     __threadfence();
   }
 }
@@ -466,140 +484,237 @@ __global__ void header_empty_kernel(surgeon_header* hdr, uint32_t sentinel) {
   hdr->tie_quota = 0;
 }
 
-// ---- per-tile counts -> exclusive scan over tiles -------------------------------------------
-// prefix[t] = (keys above the threshold before tile t) << 31 | (keys equal to it before tile t),
-// t = 0 .. tiles (the last entry holds the totals).
+// ---- threshold (where still open), per-chunk counts, exclusive scan ------------------------------
+// Launched cooperatively (all CTAs resident), so that the steps can be separated by grid-wide
+// barriers: a counter every CTA increments and then polls, with a bounded number of polls.
+__device__ __forceinline__ void grid_barrier(SelectState* st, uint32_t& epoch) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(&st->barrier_count, 1u);
+    ++epoch;
+    const uint32_t target = epoch * gridDim.x;
+    uint32_t spins = 0;
+    while (*reinterpret_cast<volatile uint32_t*>(&st->barrier_count) < target) {
+      if (++spins > (1u << 22)) { atomicMax(&st->error, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); break; }
+      __nanosleep(40);
+    }
+    __threadfence();
+  }
+  __syncthreads();
+}
+
+// prefix[c] = (elements kept for sure before chunk c) << 31 | (ties at the threshold before it),
+// c = 0 .. chunks (the last entry holds the totals).
 template <int DT>
-__global__ void __launch_bounds__(kSelThreads)
-count_kernel(const void* __restrict__ xv, long long n, SelectState* __restrict__ st,
-             surgeon_header* __restrict__ hdr, const unsigned long long* __restrict__ list,
-             uint32_t list_cap, uint32_t* __restrict__ cnt_gt, uint32_t* __restrict__ cnt_eq,
-             const uint32_t* __restrict__ cnt_zero, uint32_t* __restrict__ full_gt,
-             uint32_t* __restrict__ full_eq, unsigned long long* __restrict__ prefix, int tiles) {
+__global__ void __launch_bounds__(kSelThreads, 1)
+count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* __restrict__ st,
+             surgeon_header* __restrict__ hdr, uint32_t* __restrict__ hist_b,
+             uint32_t* __restrict__ hist_fb, const uint32_t* __restrict__ cnt_gt,
+             const uint32_t* __restrict__ cand_cnt, const void* __restrict__ slots_v,
+             unsigned long long* __restrict__ val, unsigned long long* __restrict__ prefix,
+             unsigned long long* __restrict__ partial, int tiles) {
   using E = typename Elem<DT>::type;
   constexpr uint32_t kMask = Elem<DT>::kKeyMask;
   constexpr int EPV = 16 / sizeof(E);
+  constexpr int kSlot = (DT == 0) ? 64 : 128;
+  constexpr long long kChunkElems = static_cast<long long>(kTileVecs) * EPV;
+  __shared__ uint32_t s_hist[kBinsB];          // level B / fall-back digit histogram
+  __shared__ uint32_t scratch[32];
+  __shared__ uint32_t res[2];
   __shared__ unsigned long long s_tot[32];
-  __shared__ bool s_last;
+  const E* __restrict__ x = reinterpret_cast<const E*>(xv);
+  const E* __restrict__ slots = reinterpret_cast<const E*>(slots_v);
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
   const uint32_t lane = lane_id();
-  const uint32_t tau = hdr->threshold_key;
-  const uint32_t mode = st->mode;
-  if (mode == 0) {
-    // listed keys: runs of entries share a tile, so a warp usually issues one atomic per count
-    uint32_t cnt = st->list_count;
-    if (cnt > list_cap) cnt = list_cap;
-    const long long rounded = (static_cast<long long>(cnt) + 31) & ~31LL;
-    for (long long i = static_cast<long long>(blockIdx.x) * kSelThreads + tid; i < rounded;
-         i += static_cast<long long>(gridDim.x) * kSelThreads) {
-      const bool valid = i < cnt;
-      const unsigned long long e = valid ? __ldg(list + i) : 0ull;
-      const uint32_t tile = static_cast<uint32_t>(e >> 32);
-      const uint32_t key = static_cast<uint32_t>(e);
-      const bool gt = valid && key > tau;
-      const bool eq = valid && key == tau;
-      const uint32_t t0 = __shfl_sync(kFull, tile, 0);
-      if (__all_sync(kFull, !valid || tile == t0)) {
-        const uint32_t g = __popc(__ballot_sync(kFull, gt));
-        const uint32_t q = __popc(__ballot_sync(kFull, eq));
-        if (lane == 0) {
-          if (g) atomicAdd(&cnt_gt[t0], g);
-          if (q) atomicAdd(&cnt_eq[t0], q);
+  const int gwarp = blockIdx.x * 32 + warp;
+  const int gwarps = gridDim.x * 32;
+  uint32_t epoch = 0;
+  const uint32_t mode = __ldcg(&st->mode);
+  uint32_t tau = 0, n_greater = 0;
+
+  if (mode == 1u) {
+    // ---- fall-back: exact radix select over the tensor itself, one digit per round ----
+    constexpr int kRounds = (DT == 0) ? 3 : 2;
+    const int shifts[3] = {DT == 0 ? 20 : 7, DT == 0 ? 10 : 0, 0};
+    const int bits[3] = {DT == 0 ? 11 : 8, DT == 0 ? 10 : 7, 10};
+    uint32_t fixed = 0, rank = k, above = 0;
+    const long long nvec = n / EPV;
+    const uint4* __restrict__ xq = reinterpret_cast<const uint4*>(xv);
+    for (int round = 0; round < kRounds; ++round) {
+      const int sh = shifts[round], nb = 1 << bits[round], hi = sh + bits[round];
+      for (int i = tid; i < kFbBins; i += kSelThreads) s_hist[i] = 0;
+      __syncthreads();
+      uint32_t zero_cnt = 0;     // digit 0 in a register (half of post-ReLU data)
+      auto add = [&](uint32_t key) {
+        const bool match = hi >= 31 || (key >> hi) == (fixed >> hi);
+        if (match) {
+          const uint32_t d = (key >> sh) & (nb - 1);
+          if (d == 0) ++zero_cnt;
+          else atomicAdd(&s_hist[d], 1u);
         }
-      } else {
-        if (gt) atomicAdd(&cnt_gt[tile], 1u);
-        if (eq) atomicAdd(&cnt_eq[tile], 1u);
+      };
+      for (long long v = static_cast<long long>(blockIdx.x) * kSelThreads + tid; v < nvec;
+           v += static_cast<long long>(gridDim.x) * kSelThreads) {
+        const uint4 q = __ldg(xq + v);
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < EPV; ++i)
+          add(((DT == 0) ? w[i % 4] : (w[i >> 1] >> (16 * (i & 1)))) & kMask);
+      }
+      if (blockIdx.x == 0)
+        for (long long j = nvec * EPV + tid; j < n; j += kSelThreads)
+          add(static_cast<uint32_t>(x[j]) & kMask);
+      zero_cnt = warp_sum(zero_cnt);
+      if (lane == 0 && zero_cnt) atomicAdd(&s_hist[0], zero_cnt);
+      __syncthreads();
+      uint32_t* gh = hist_fb + round * kFbBins;
+      for (int i = tid; i < kFbBins; i += kSelThreads)
+        if (s_hist[i]) atomicAdd(&gh[i], s_hist[i]);
+      grid_barrier(st, epoch);
+      for (int i = tid; i < kFbBins; i += kSelThreads) s_hist[i] = __ldcg(gh + i);
+      __syncthreads();
+      find_from_top<kFbBins>([&](int i) { return s_hist[i]; }, rank, scratch, res);
+      fixed |= res[0] << sh;
+      above += res[1];
+      rank -= res[1];
+      __syncthreads();
+    }
+    tau = fixed;
+    n_greater = above;
+  } else if (mode == 0u) {
+    // ---- fp32: level B over the candidates of level-A bin binA ----
+    const uint32_t lo_key = __ldcg(&st->lo_key), binA = __ldcg(&st->binA);
+    for (int c = gwarp; c < tiles; c += gwarps) {
+      const uint32_t cc = __ldg(cand_cnt + c);
+      for (uint32_t i = lane; i < cc; i += 32) {
+        const uint32_t rel = static_cast<uint32_t>(__ldg(slots + static_cast<long long>(c) * kSlot + i)) - lo_key;
+        if ((rel >> 12) == binA) atomicAdd(&hist_b[rel & (kBinsB - 1)], 1u);
       }
     }
+    grid_barrier(st, epoch);
+    for (int i = tid; i < kBinsB; i += kSelThreads) s_hist[i] = __ldcg(hist_b + i);
+    __syncthreads();
+    find_from_top<kBinsB>([&](int i) { return s_hist[i]; }, __ldcg(&st->rankA), scratch, res);
+    tau = lo_key + (binA << 12) + res[0];
+    n_greater = __ldcg(&st->above_total) + __ldcg(&st->aboveA) + res[1];
   } else {
-    // the list is unusable: count every tile from the tensor itself (one vector per thread,
-    // a warp's 32 vectors lie inside one tile)
-    const E* __restrict__ x = reinterpret_cast<const E*>(xv);
-    const long long n_steps = (static_cast<long long>(tiles) * kTileVecs + kSelThreads - 1) / kSelThreads;
-    for (long long s = blockIdx.x; s < n_steps; s += gridDim.x) {
-      const long long vec = s * kSelThreads + tid;
-      const long long t = vec / kTileVecs;
-      const long long base = vec * EPV;
-      uint32_t g = 0, q = 0;
-      if (base + EPV <= n) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + base));
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    tau = hdr->threshold_key;
+  }
+  if (mode != 2u && blockIdx.x == 0 && tid == 0) {
+    hdr->threshold_key = tau;
+    hdr->status = __ldcg(&st->error);
+    hdr->n_keep = k;
+    hdr->n_greater = n_greater;
+    hdr->tie_quota = static_cast<long long>(k) - n_greater;
+  }
+
+  // ---- per-chunk values; CTA b owns the chunks [b*per, (b+1)*per) ----
+  const int per = (tiles + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+  const int c_begin = blockIdx.x * per < tiles ? blockIdx.x * per : tiles;
+  const int c_end = c_begin + per < tiles ? c_begin + per : tiles;
+  unsigned long long acc = 0;
+  for (int c = c_begin + warp; c < c_end; c += 32) {
+    uint32_t g = 0, q = 0;
+    if (mode != 1u) {
+      const uint32_t cc = __ldg(cand_cnt + c), cg = __ldg(cnt_gt + c);
+      for (uint32_t i = lane; i < cc; i += 32) {
+        const uint32_t key = static_cast<uint32_t>(__ldg(slots + static_cast<long long>(c) * kSlot + i));
+        g += key > tau ? 1u : 0u;
+        q += key == tau ? 1u : 0u;
+      }
+      g = __reduce_add_sync(kFull, g) + cg;
+      q = __reduce_add_sync(kFull, q);
+      if (tau == 0) {         // lo_key == 1: whatever is neither above nor inside the bracket is 0
+        const long long left = n - static_cast<long long>(c) * kChunkElems;
+        q += static_cast<uint32_t>(left < kChunkElems ? left : kChunkElems) - cg - cc;
+      }
+    } else {
 #pragma unroll
-        for (int i = 0; i < EPV; ++i) {
-          const uint32_t key = ((DT == 0) ? w[i % 4] : (w[i >> 1] >> (16 * (i & 1)))) & kMask;
-          g += key > tau ? 1u : 0u;
-          q += key == tau ? 1u : 0u;
-        }
-      } else {
-        for (int i = 0; i < EPV; ++i) {
-          if (base + i < n) {
-            const uint32_t key = static_cast<uint32_t>(x[base + i]) & kMask;
+      for (int u = 0; u < kTileVecs / 32; ++u) {
+        const long long base = (static_cast<long long>(c) * kTileVecs + u * 32 + lane) * EPV;
+        if (base + EPV <= n) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + base));
+          const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int i = 0; i < EPV; ++i) {
+            const uint32_t key = ((DT == 0) ? w[i % 4] : (w[i >> 1] >> (16 * (i & 1)))) & kMask;
             g += key > tau ? 1u : 0u;
             q += key == tau ? 1u : 0u;
+          }
+        } else {
+          for (int i = 0; i < EPV; ++i) {
+            if (base + i < n) {
+              const uint32_t key = static_cast<uint32_t>(x[base + i]) & kMask;
+              g += key > tau ? 1u : 0u;
+              q += key == tau ? 1u : 0u;
+            }
           }
         }
       }
       g = __reduce_add_sync(kFull, g);
       q = __reduce_add_sync(kFull, q);
-      if (lane == 0 && t < tiles) {
-        if (g) atomicAdd(&full_gt[t], g);
-        if (q) atomicAdd(&full_eq[t], q);
-      }
     }
+    const unsigned long long v = (static_cast<unsigned long long>(g) << 31) | q;
+    if (lane == 0) val[c] = v;
+    acc += v;            // identical in every lane
   }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(&st->ticket_count, 1u) == gridDim.x - 1);
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-
-  // Last CTA: exclusive scan.  Warp w owns a contiguous range of tiles.
-  auto value = [&](int t) -> unsigned long long {
-    unsigned long long g, q;
-    if (mode == 0) {
-      g = __ldcg(cnt_gt + t);
-      q = __ldcg(cnt_eq + t) + (tau == 0 ? __ldcg(cnt_zero + t) : 0u);
-    } else {
-      g = __ldcg(full_gt + t);
-      q = __ldcg(full_eq + t);
-    }
-    return (g << 31) | q;
-  };
-  const int chunk = ((tiles + 31) / 32 + 31) & ~31;
-  const int begin = warp * chunk < tiles ? warp * chunk : tiles;
-  const int end = begin + chunk < tiles ? begin + chunk : tiles;
-  unsigned long long acc = 0;
-#pragma unroll 4
-  for (int t = begin + lane; t < end; t += 32) acc += value(t);
-  acc = warp_sum_u64(acc);
   if (lane == 0) s_tot[warp] = acc;
   __syncthreads();
-  unsigned long long carry = 0, total = 0;
-  for (int w = 0; w < 32; ++w) {
-    if (w < warp) carry += s_tot[w];
-    total += s_tot[w];
+  if (tid == 0) {
+    unsigned long long t = 0;
+    for (int w = 0; w < 32; ++w) t += s_tot[w];
+    partial[blockIdx.x] = t;
   }
-  for (int t0 = begin; t0 < end; t0 += 32) {
-    const int t = t0 + lane;
-    const unsigned long long v = t < end ? value(t) : 0ull;
+  grid_barrier(st, epoch);
+
+  // ---- exclusive scan: carry from the CTAs before, then warp w scans a sub-range ----
+  unsigned long long carry = 0;
+  {
+    unsigned long long p = 0;
+    for (int b = tid; b < static_cast<int>(blockIdx.x); b += kSelThreads) p += __ldcg(partial + b);
+    p = warp_sum_u64(p);
+    if (lane == 0) s_tot[warp] = p;
+    __syncthreads();
+    for (int w = 0; w < 32; ++w) carry += s_tot[w];
+    __syncthreads();
+  }
+  const int sub = ((per + 31) / 32 + 31) & ~31;
+  const int begin = c_begin + warp * sub < c_end ? c_begin + warp * sub : c_end;
+  const int end = begin + sub < c_end ? begin + sub : c_end;
+  unsigned long long wsum = 0;
+#pragma unroll 4
+  for (int c = begin + lane; c < end; c += 32) wsum += __ldcg(val + c);
+  wsum = warp_sum_u64(wsum);
+  if (lane == 0) s_tot[warp] = wsum;
+  __syncthreads();
+  for (int w = 0; w < warp; ++w) carry += s_tot[w];
+  for (int c0 = begin; c0 < end; c0 += 32) {
+    const int c = c0 + lane;
+    const unsigned long long v = c < end ? __ldcg(val + c) : 0ull;
     unsigned long long incl = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const unsigned long long up = __shfl_up_sync(kFull, incl, o);
       if (lane >= static_cast<uint32_t>(o)) incl += up;
     }
-    if (t < end) prefix[t] = carry + incl - v;
+    if (c < end) prefix[c] = carry + incl - v;
     carry += __shfl_sync(kFull, incl, 31);
   }
-  if (tid == 0) {
-    prefix[tiles] = total;
-    // self-check: the counts must add up to what the select found
-    const long long gt_all = static_cast<long long>(total >> 31);
-    const long long eq_all = static_cast<long long>(total & 0x7FFFFFFFull);
-    if (gt_all != hdr->n_greater || eq_all < hdr->tie_quota)
-      atomicMax(&hdr->status, static_cast<uint32_t>(SURGEON_ERR_INTERNAL));
+  if (c_end == tiles && c_begin < tiles) {
+    // the CTA that owns the last chunk also writes the totals and checks them
+    __syncthreads();
+    if (tid == 0) {
+      unsigned long long total = 0;
+      for (int b = 0; b <= static_cast<int>(blockIdx.x); ++b) total += __ldcg(partial + b);
+      prefix[tiles] = total;
+      const long long gt_all = static_cast<long long>(total >> 31);
+      const long long eq_all = static_cast<long long>(total & 0x7FFFFFFFull);
+      const long long ng = (mode == 2u) ? hdr->n_greater : static_cast<long long>(n_greater);
+      if (gt_all != ng || eq_all < static_cast<long long>(k) - gt_all)
+        atomicMax(&hdr->status, static_cast<uint32_t>(SURGEON_ERR_INTERNAL));
+    }
   }
 }
 
@@ -853,20 +968,9 @@ compact_boundary_kernel(const void* __restrict__ xv, long long n, surgeon_header
 }
 
 // ---- streaming compaction ---------------------------------------------------------------------
-// Persistent CTAs.  One producer thread keeps a ring of 32 KB stages full with 2-D TMA loads of
-// [256 rows x 128 bytes] (128-byte swizzle, so that 32 lanes can each read their own row without
-// bank conflicts).  Each of the 8 consumer warps owns one 4 KB chunk of a stage; each LANE owns
-// one 128-byte row of it, i.e. 32 (fp32) or 64 (bf16) consecutive elements, and builds their
-// bitmap word(s) with no cross-lane traffic.  One warp scan places the lanes' kept values; they
-// are gathered in the warp's part of the stage (in place) and leave as 16-byte vectors.
-constexpr int kCsWarps = 8;
-constexpr int kCsThreads = (kCsWarps + 1) * 32;
-constexpr int kCsStageRows = kCsWarps * 32;
-constexpr int kCsStageBytes = kCsStageRows * 128;
-constexpr int kCsStages = 3;
-constexpr size_t kCsSmem = static_cast<size_t>(kCsStages) * kCsStageBytes + 1024;
-static_assert(kCsStageRows * 128 / 16 == kCsWarps * kTileVecs, "a warp's 32 rows are one chunk");
-
+// Same ring and lane-per-row layout as classify_kernel.  A lane builds the bitmap word(s) of its
+// row with no cross-lane traffic; one warp scan places the lanes' kept values; they are gathered
+// in the warp's part of the stage (in place) and leave as 16-byte vectors.
 template <int DT>
 __global__ void __launch_bounds__(kCsThreads, 2)
 compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict__ xv,
@@ -1101,123 +1205,130 @@ decompress_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ 
   }
 }
 
+using TmaEncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                 const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                 const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The tensor as rows of 128 bytes (32 words), box = one ring stage, 128-byte swizzle.
+bool make_row_map(const void* x, long long n_rows_full, CUtensorMap* map) {
+  const TmaEncodeFn encode = reinterpret_cast<TmaEncodeFn>(tensor_map_encode_fn());
+  if (!encode) return false;
+  const cuuint64_t dims[2] = {32, static_cast<cuuint64_t>(n_rows_full)};
+  const cuuint64_t strides[1] = {128};
+  const cuuint32_t box[2] = {32, static_cast<cuuint32_t>(kCsStageRows)};
+  const cuuint32_t estr[2] = {1, 1};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(x), dims, strides, box,
+                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int DT>
 cudaError_t run_prune_compact(const void* x, long long n, long long k,
                               const surgeon_compressed& out, void* workspace,
                               cudaStream_t stream) {
-  constexpr int VEC = 16 / static_cast<int>(sizeof(typename Elem<DT>::type));
+  using E = typename Elem<DT>::type;
+  constexpr int VEC = 16 / static_cast<int>(sizeof(E));
   const PruneLayout L = prune_layout(n, DT);
   char* ws = static_cast<char*>(workspace);
   SelectState* st = reinterpret_cast<SelectState*>(ws);
-  uint32_t* hist1 = reinterpret_cast<uint32_t*>(ws + L.hist1);
   uint32_t* hist_s = reinterpret_cast<uint32_t*>(ws + L.hist_s);
-  uint32_t* hist2 = reinterpret_cast<uint32_t*>(ws + L.hist2);
+  uint32_t* hist_a = reinterpret_cast<uint32_t*>(ws + L.hist_a);
+  uint32_t* hist_b = reinterpret_cast<uint32_t*>(ws + L.hist_b);
+  uint32_t* hist_fb = reinterpret_cast<uint32_t*>(ws + L.hist_fb);
   uint32_t* cnt_gt = reinterpret_cast<uint32_t*>(ws + L.cnt_gt);
-  uint32_t* cnt_eq = reinterpret_cast<uint32_t*>(ws + L.cnt_eq);
-  uint32_t* cnt_zero = reinterpret_cast<uint32_t*>(ws + L.cnt_zero);
-  uint32_t* full_gt = reinterpret_cast<uint32_t*>(ws + L.full_gt);
-  uint32_t* full_eq = reinterpret_cast<uint32_t*>(ws + L.full_eq);
+  uint32_t* cand_cnt = reinterpret_cast<uint32_t*>(ws + L.cand_cnt);
+  unsigned long long* val = reinterpret_cast<unsigned long long*>(ws + L.val);
   unsigned long long* prefix = reinterpret_cast<unsigned long long*>(ws + L.prefix);
-  unsigned long long* list = reinterpret_cast<unsigned long long*>(ws + L.list);
-  const uint32_t list_cap = static_cast<uint32_t>(L.list_cap);
+  unsigned long long* partial = reinterpret_cast<unsigned long long*>(ws + L.partial);
+  void* slots = ws + L.slots;
   cudaError_t e = cudaMemsetAsync(workspace, 0, L.zero_bytes, stream);
   if (e != cudaSuccess) return e;
   const int sms = sm_count();
   static bool attrs_done_on[64] = {false};   // per device; a race only repeats idempotent calls
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
-  bool& attrs_done = attrs_done_on[dev];
-  if (!attrs_done) {
+  if (!attrs_done_on[dev]) {
     e = cudaFuncSetAttribute(sample_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kHistWords * 4);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(hist_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(kHistSmem));
+    e = cudaFuncSetAttribute(classify_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(kCsSmem));
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(compact_stream_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(kCsSmem));
     if (e != cudaSuccess) return e;
-    attrs_done = true;
+    attrs_done_on[dev] = true;
   }
+  const long long n_rows_full = n * static_cast<long long>(sizeof(E)) / 128;
+  const int n_chunks = static_cast<int>(L.tiles);
+  const int n_stage_tiles = (n_chunks + kCsWarps - 1) / kCsWarps;
+  const int stream_grid = n_stage_tiles < 2 * sms ? n_stage_tiles : 2 * sms;
+  CUtensorMap map;
+  const bool streamed = n > kSampleMinN && make_row_map(x, n_rows_full, &map);
 
   if (k == 0) {
     header_empty_kernel<<<1, 1, 0, stream>>>(out.header, Elem<DT>::kSentinel);
     note_launches(1);
+    if (n > 0) {   // nothing is kept: the scan is all zeros
+      e = cudaMemsetAsync(prefix, 0, static_cast<size_t>(L.tiles + 1) * 8, stream);
+      if (e != cudaSuccess) return e;
+    }
   } else {
-    const long long nvec = n / VEC;
-    int use_bracket = 0;
-    if (n > kSampleMinN) {
+    if (streamed) {
       // sample: segments of 32 vectors, about 1/32 of the tensor, at most 16384 segments
-      const long long n_seg_all = nvec / 32;
+      const long long n_seg_all = (n / VEC) / 32;
       long long n_seg = n_seg_all / 32;
       if (n_seg < 256) n_seg = 256;
       if (n_seg > 16384) n_seg = 16384;
       const long long seg_stride = n_seg_all / n_seg;   // >= 1 because n > 65536
-      const long long want = (n_seg + 63) / 64;
+      const long long want = (n_seg + 127) / 128;
       const int grid = static_cast<int>(want < sms ? want : sms);
       sample_kernel<DT><<<grid, kSelThreads, kHistWords * 4, stream>>>(
           reinterpret_cast<const uint4*>(x), n, static_cast<uint32_t>(k),
           static_cast<uint32_t>(n_seg), static_cast<uint32_t>(seg_stride), st, hist_s);
-      note_launches(1);
-      use_bracket = 1;
+      classify_kernel<DT><<<stream_grid, kCsThreads, kCsSmem, stream>>>(
+          map, x, n, n_rows_full, static_cast<uint32_t>(k), st, hist_a, cnt_gt, cand_cnt, slots,
+          out.header, n_chunks, n_stage_tiles);
+      note_launches(2);
+    } else {
+      // small tensor: straight to the fall-back select (mode = 1; the state is little-endian)
+      e = cudaMemsetAsync(&st->mode, 1, 1, stream);
+      if (e != cudaSuccess) return e;
     }
     {
-      const long long chunks = (nvec + kStageVecs - 1) / kStageVecs;
-      const int grid = static_cast<int>(chunks < 1 ? 1 : (chunks < sms ? chunks : sms));
-      hist_kernel<DT><<<grid, kSelThreads, kHistSmem, stream>>>(
-          x, n, static_cast<uint32_t>(k), use_bracket, st, hist1, hist2, cnt_gt, cnt_zero, list,
-          list_cap, out.header);
+      // cooperative launch: every CTA must be resident for the grid-wide barriers
+      long long want = (L.tiles + 31) / 32;
+      const int grid = static_cast<int>(want < 1 ? 1 : (want < sms ? want : sms));
+      const void* xa = x;
+      long long na = n;
+      uint32_t ka = static_cast<uint32_t>(k);
+      surgeon_header* hdr = out.header;
+      const uint32_t* cg = cnt_gt;
+      const uint32_t* cc = cand_cnt;
+      const void* sl = slots;
+      int tiles = n_chunks;
+      void* args[] = {&xa, &na, &ka, &st, &hdr, &hist_b, &hist_fb, &cg, &cc, &sl, &val, &prefix,
+                      &partial, &tiles};
+      e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(count_kernel<DT>), dim3(grid),
+                                      dim3(kSelThreads), args, 0, stream);
+      if (e != cudaSuccess) return e;
       note_launches(1);
     }
-    const long long want = (nvec + 4 * kSelThreads - 1) / (4 * kSelThreads);
-    const long long cap = 2LL * sms;
-    const int grid = static_cast<int>(want < 1 ? 1 : (want < cap ? want : cap));
-    if (DT == 0) {
-      refine_kernel<<<grid, kSelThreads, 0, stream>>>(
-          reinterpret_cast<const uint4*>(x), n, static_cast<uint32_t>(k), st, hist2, list, list_cap,
-          out.header);
-      note_launches(1);
-    }
-    count_kernel<DT><<<grid, kSelThreads, 0, stream>>>(
-        x, n, st, out.header, list, list_cap, cnt_gt, cnt_eq, cnt_zero, full_gt, full_eq, prefix,
-        static_cast<int>(L.tiles));
-    note_launches(1);
   }
   if (n == 0) {
     offsets_empty_kernel<<<1, 1, 0, stream>>>(out.block_offsets);
     note_launches(1);
   } else {
-    const long long n_rows_full = n * static_cast<long long>(sizeof(typename Elem<DT>::type)) / 128;
-    bool streamed = false;
-    if (n_rows_full >= kCsStageRows) {
-      using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                    const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                    const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-      const EncodeFn encode = reinterpret_cast<EncodeFn>(tensor_map_encode_fn());
-      CUtensorMap map;
-      const cuuint64_t dims[2] = {32, static_cast<cuuint64_t>(n_rows_full)};
-      const cuuint64_t strides[1] = {128};
-      const cuuint32_t box[2] = {32, static_cast<cuuint32_t>(kCsStageRows)};
-      const cuuint32_t estr[2] = {1, 1};
-      if (encode &&
-          encode(&map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(x), dims, strides, box,
-                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS) {
-        const int n_stage_tiles = static_cast<int>((L.tiles + kCsWarps - 1) / kCsWarps);
-        const int grid = n_stage_tiles < 2 * sms ? n_stage_tiles : 2 * sms;
-        compact_stream_kernel<DT><<<grid, kCsThreads, kCsSmem, stream>>>(
-            map, x, n, n_rows_full, out.header, out.bitmap, out.values, out.block_offsets, prefix,
-            static_cast<int>(L.tiles), n_stage_tiles);
-        streamed = true;
-      }
-    }
-    if (!streamed)
+    if (streamed)
+      compact_stream_kernel<DT><<<stream_grid, kCsThreads, kCsSmem, stream>>>(
+          map, x, n, n_rows_full, out.header, out.bitmap, out.values, out.block_offsets, prefix,
+          n_chunks, n_stage_tiles);
+    else
       compact_small_kernel<DT><<<static_cast<unsigned>(L.tiles), kCompactThreads, 0, stream>>>(
           x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix);
     compact_boundary_kernel<DT><<<1, kCompactThreads, 0, stream>>>(
-        x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix,
-        static_cast<int>(L.tiles));
+        x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix, n_chunks);
     note_launches(2);
   }
   return cudaGetLastError();

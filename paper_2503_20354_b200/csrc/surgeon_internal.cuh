@@ -33,53 +33,62 @@ static_assert((1 << kBlockShift) == SURGEON_BLOCK, "SURGEON_BLOCK must be 128");
 // the unit of the exclusive scan that places it.
 constexpr int kTileVecs = 256;
 constexpr int64_t compact_tile_elems(int dt) { return dt == 0 ? 1024 : 2048; }
-constexpr int kBuckets = 32768;        // histogram bins of the select pass (top 15 key bits)
-constexpr int kLowBins = 65536;        // bins of the fp32 refinement (low 16 key bits)
-constexpr int64_t kSampleMinN = 65536; // tensors up to this size list every non-zero element
+constexpr int kBuckets = 32768;        // bins of the sample histogram (top 15 key bits)
+constexpr int kMaxSpan = 32;           // widest bracket (in buckets) the candidate path handles
+constexpr int kBinsA = 16 * kMaxSpan;  // level A of the select among candidates
+constexpr int kBinsB = 4096;           // level B (fp32 only)
+constexpr int kFbBins = 2048;          // digit histogram of the fall-back radix select
+constexpr int64_t kSampleMinN = 65536; // smaller tensors go straight to the fall-back select
+// Candidate slots: per chunk, room for 1/16 of its elements (fp32: 32-bit keys, bf16: 16-bit).
+constexpr int slot_entries(int dt) { return dt == 0 ? 64 : 128; }
+constexpr int slot_entry_bytes(int dt) { return dt == 0 ? 4 : 2; }
 
 struct SelectState {
-  uint32_t ticket_sample, ticket_hist, ticket_refine, ticket_count;
+  uint32_t ticket_sample, ticket_classify, barrier_count, error;
   uint32_t blo, bhi;             // bucket bracket around the threshold, predicted from the sample
-  uint32_t list_count, list_overflow;
-  uint32_t b1, mode;             // bucket of the threshold; 0 = candidate list usable, 1 = re-read x
-  uint32_t k1, above;            // rank of the threshold inside bucket b1; keys in buckets above b1
-  uint32_t zero_count;           // elements whose key is exactly 0
-  uint32_t error;                // surgeon_status raised by a bounded wait of the select kernels
-  uint32_t pad[2];
+  uint32_t lo_key, hi_key;       // the same bracket as an inclusive key range (lo_key >= 1)
+  uint32_t mode;                 // 0 = threshold among the candidates, level B pending (fp32);
+                                 // 1 = bracket unusable, fall back to a radix select over x;
+                                 // 2 = threshold already final in the header
+  uint32_t list_overflow;
+  uint32_t above_total, cand_total;   // keys above hi_key / inside [lo_key, hi_key]
+  uint32_t binA, rankA, aboveA;  // level A: bin of the threshold, its rank inside, candidates above
+  uint32_t fb_prefix, fb_rank, fb_above;   // fall-back select: key bits fixed so far, rank, count above
+  uint32_t pad[14];
 };
-static_assert(sizeof(SelectState) == 64, "SelectState layout");
+static_assert(sizeof(SelectState) == 128, "SelectState layout");
 constexpr size_t kWsStateBytes = 256;
 
 // Byte offsets of the parts of the scratch buffer; everything in [0, zero_bytes) must be zero
-// when the first kernel starts.  Per compaction tile: cnt_gt / cnt_zero are filled by the
-// histogram pass (keys above the bracket, exact zeros), cnt_gt / cnt_eq are completed from the
-// candidate list once the threshold is known; full_gt / full_eq are used instead when the
-// tensor had to be re-read; prefix holds the exclusive scan the compaction kernel starts from.
+// when the first kernel starts.  Per chunk: cnt_gt = keys above the bracket, cand_cnt = keys
+// inside it (both written by the classify pass), val = (kept for sure << 31 | ties) once the
+// threshold is known, prefix = exclusive scan of val (chunks + 1 entries), slots = the keys
+// inside the bracket.  partial: one scan carry per CTA of the count kernel.
 struct PruneLayout {
-  size_t hist1, hist_s, hist2, cnt_gt, cnt_eq, cnt_zero, full_gt, full_eq, prefix, zero_bytes,
-      list, total;
-  int64_t tiles, list_cap;
+  size_t hist_s, hist_a, hist_b, hist_fb, zero_bytes, cnt_gt, cand_cnt, val, prefix, partial,
+      slots, total;
+  int64_t tiles;
 };
+constexpr size_t kMaxCountCtas = 1024;
 constexpr PruneLayout prune_layout(int64_t n, int dt) {
   PruneLayout L{};
   L.tiles = (n + compact_tile_elems(dt) - 1) / compact_tile_elems(dt);
-  const size_t per_tile = static_cast<size_t>(L.tiles) * 4;
+  const size_t t = static_cast<size_t>(L.tiles);
   size_t off = kWsStateBytes;
-  L.hist1 = off; off += static_cast<size_t>(kBuckets) * 4;
   L.hist_s = off; off += static_cast<size_t>(kBuckets) * 4;
-  L.hist2 = off; if (dt == 0) off += static_cast<size_t>(kLowBins) * 4;
-  L.cnt_gt = off; off += per_tile;
-  L.cnt_eq = off; off += per_tile;
-  L.cnt_zero = off; off += per_tile;
-  L.full_gt = off; off += per_tile;
-  L.full_eq = off; off += per_tile;
-  off = (off + 15) & ~static_cast<size_t>(15);
-  L.prefix = off; off += per_tile * 2 + 8;   // tiles + 1 entries
-  off = (off + 255) & ~static_cast<size_t>(255);
+  L.hist_a = off; off += static_cast<size_t>(kBinsA) * 4;
+  L.hist_b = off; off += static_cast<size_t>(kBinsB) * 4;
+  L.hist_fb = off; off += static_cast<size_t>(3 * kFbBins) * 4;
   L.zero_bytes = off;
-  L.list = off;
-  L.list_cap = n <= kSampleMinN ? n : n / 32 + kSampleMinN;
-  off += static_cast<size_t>(L.list_cap) * 8;
+  L.cnt_gt = off; off += t * 4;
+  L.cand_cnt = off; off += t * 4;
+  off = (off + 15) & ~static_cast<size_t>(15);
+  L.val = off; off += t * 8;
+  L.prefix = off; off += (t + 1) * 8;
+  L.partial = off; off += kMaxCountCtas * 8;
+  off = (off + 255) & ~static_cast<size_t>(255);
+  L.slots = off;
+  off += t * static_cast<size_t>(slot_entries(dt)) * slot_entry_bytes(dt);
   L.total = (off + 255) & ~static_cast<size_t>(255);
   return L;
 }
