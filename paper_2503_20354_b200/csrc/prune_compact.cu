@@ -197,8 +197,10 @@ sample_kernel(const uint4* __restrict__ xq, long long n, uint32_t k, uint32_t n_
     // the bracket as keys; key 0 (exact zeros) is never a candidate
     const uint32_t lo = (DT == 0) ? (blo << 16) : blo;
     st->lo_key = lo < 1u ? 1u : lo;
-    st->hi_key = (DT == 0) ? ((bhi << 16) | 0xFFFFu) : bhi;
-    st->mode = (bhi - blo + 1u > static_cast<uint32_t>(kMaxSpan)) ? 1u : 0u;
+    const uint32_t hi = (DT == 0) ? ((bhi << 16) | 0xFFFFu) : bhi;
+    st->hi_key = hi;
+    const int range_bits = 32 - __clz(hi - st->lo_key);       // bits of the widest relative key
+    st->shiftA = range_bits > 9 ? static_cast<uint32_t>(range_bits - 9) : 0u;
   }
 }
 
@@ -265,7 +267,6 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
   constexpr int EPR = 128 / sizeof(E);
   constexpr int WPL = EPR / 32;
   constexpr int kSlot = (DT == 0) ? 64 : 128;
-  constexpr int kShiftA = (DT == 0) ? 12 : 0;
   extern __shared__ __align__(1024) unsigned char cs_smem_raw[];
   unsigned char* ring = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(cs_smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -281,6 +282,7 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
   if (st->mode == 1u) return;          // the sample found no usable bracket
   const uint32_t lo_key = st->lo_key, hi_key = st->hi_key;
   const uint32_t range = hi_key - lo_key;
+  const uint32_t shiftA = st->shiftA;
   const uint32_t full_bar = smem_u32(bars);
   const uint32_t empty_bar = smem_u32(bars + kCsStages);
   if (tid == 0) {
@@ -387,7 +389,7 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
                           row + (((byte >> 4) ^ (lane & 7)) << 4) + (byte & 15))) & kMask;
               }
               slot[pos++] = static_cast<E>(key);
-              atomicAdd(&s_hist[(key - lo_key) >> kShiftA], 1u);
+              atomicAdd(&s_hist[(key - lo_key) >> shiftA], 1u);
             }
           }
         }
@@ -452,8 +454,8 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
       st->aboveA = aboveA;
       st->rankA = want - aboveA;
     }
-    mode = (DT == 0) ? 0u : 2u;
-    tau = lo_key + bin;                       // bf16: level A is exact
+    mode = shiftA ? 0u : 2u;
+    tau = lo_key + bin;                       // shiftA == 0: level A is exact
     n_greater = above_total + aboveA;
   } else if (lo_key == 1u && r <= n_cand + zeros) {
     mode = 2;
@@ -584,21 +586,33 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
     tau = fixed;
     n_greater = above;
   } else if (mode == 0u) {
-    // ---- fp32: level B over the candidates of level-A bin binA ----
-    const uint32_t lo_key = __ldcg(&st->lo_key), binA = __ldcg(&st->binA);
-    for (int c = gwarp; c < tiles; c += gwarps) {
-      const uint32_t cc = __ldg(cand_cnt + c);
-      for (uint32_t i = lane; i < cc; i += 32) {
-        const uint32_t rel = static_cast<uint32_t>(__ldg(slots + static_cast<long long>(c) * kSlot + i)) - lo_key;
-        if ((rel >> 12) == binA) atomicAdd(&hist_b[rel & (kBinsB - 1)], 1u);
+    // ---- further levels of at most 11 bits over the candidates that match so far ----
+    const uint32_t lo_key = __ldcg(&st->lo_key);
+    uint32_t shift = __ldcg(&st->shiftA), pre = __ldcg(&st->binA), rank = __ldcg(&st->rankA);
+    uint32_t above_c = __ldcg(&st->aboveA);
+    for (int level = 0; shift > 0; ++level) {
+      const uint32_t nb = shift < 11u ? shift : 11u, ns = shift - nb;
+      uint32_t* gh = hist_b + level * kFbBins;
+      for (int c = gwarp; c < tiles; c += gwarps) {
+        const uint32_t cc = __ldg(cand_cnt + c);
+        for (uint32_t i = lane; i < cc; i += 32) {
+          const uint32_t rel =
+              static_cast<uint32_t>(__ldg(slots + static_cast<long long>(c) * kSlot + i)) - lo_key;
+          if ((rel >> shift) == pre) atomicAdd(&gh[(rel >> ns) & ((1u << nb) - 1u)], 1u);
+        }
       }
+      grid_barrier(st, epoch);
+      for (int i = tid; i < kFbBins; i += kSelThreads) s_hist[i] = __ldcg(gh + i);
+      __syncthreads();
+      find_from_top<kFbBins>([&](int i) { return s_hist[i]; }, rank, scratch, res);
+      pre = (pre << nb) | res[0];
+      above_c += res[1];
+      rank -= res[1];
+      shift = ns;
+      __syncthreads();
     }
-    grid_barrier(st, epoch);
-    for (int i = tid; i < kBinsB; i += kSelThreads) s_hist[i] = __ldcg(hist_b + i);
-    __syncthreads();
-    find_from_top<kBinsB>([&](int i) { return s_hist[i]; }, __ldcg(&st->rankA), scratch, res);
-    tau = lo_key + (binA << 12) + res[0];
-    n_greater = __ldcg(&st->above_total) + __ldcg(&st->aboveA) + res[1];
+    tau = lo_key + pre;
+    n_greater = __ldcg(&st->above_total) + above_c;
   } else {
     tau = hdr->threshold_key;
   }

@@ -34,9 +34,9 @@ static_assert((1 << kBlockShift) == SURGEON_BLOCK, "SURGEON_BLOCK must be 128");
 constexpr int kTileVecs = 256;
 constexpr int64_t compact_tile_elems(int dt) { return dt == 0 ? 1024 : 2048; }
 constexpr int kBuckets = 32768;        // bins of the sample histogram (top 15 key bits)
-constexpr int kMaxSpan = 32;           // widest bracket (in buckets) the candidate path handles
-constexpr int kBinsA = 16 * kMaxSpan;  // level A of the select among candidates
-constexpr int kBinsB = 4096;           // level B (fp32 only)
+constexpr int kBinsA = 512;            // level A of the select among candidates: the top bits of
+                                       // (key - lo_key), shifted so that the bracket fits
+constexpr int kBinsB = 4096;           // up to two further levels of 2048 bins each
 constexpr int kFbBins = 2048;          // digit histogram of the fall-back radix select
 constexpr int64_t kSampleMinN = 65536; // smaller tensors go straight to the fall-back select
 // Candidate slots: per chunk, room for 1/16 of its elements (fp32: 32-bit keys, bf16: 16-bit).
@@ -52,9 +52,10 @@ struct SelectState {
                                  // 2 = threshold already final in the header
   uint32_t list_overflow;
   uint32_t above_total, cand_total;   // keys above hi_key / inside [lo_key, hi_key]
+  uint32_t shiftA;               // level A bin of a key = (key - lo_key) >> shiftA
   uint32_t binA, rankA, aboveA;  // level A: bin of the threshold, its rank inside, candidates above
   uint32_t fb_prefix, fb_rank, fb_above;   // fall-back select: key bits fixed so far, rank, count above
-  uint32_t pad[14];
+  uint32_t pad[13];
 };
 static_assert(sizeof(SelectState) == 128, "SelectState layout");
 constexpr size_t kWsStateBytes = 256;
