@@ -176,19 +176,26 @@ sample_kernel(const uint4* __restrict__ xq, long long n, uint32_t k, uint32_t n_
   load_hist_to_smem(shist, hist);
   __syncthreads();
   // rank of the threshold inside the sample, +- 5 standard deviations of a binomial count
-  const double S = static_cast<double>(32 * EPV) * n_seg;
-  const double q = static_cast<double>(k) / static_cast<double>(n);
-  const double r = q * S;
-  const double delta = 5.0 * sqrt(S * q * (1.0 - q)) + 8.0;
+  // (single precision, one thread: double-precision arithmetic is slow on this GPU)
+  __shared__ uint32_t s_rank[2];
+  if (tid == 0) {
+    const float S = static_cast<float>(32 * EPV) * static_cast<float>(n_seg);
+    const float q = static_cast<float>(static_cast<double>(k) / static_cast<double>(n));
+    const float r = q * S;
+    const float delta = 5.0f * sqrtf(S * q * (1.0f - q)) + 16.0f;
+    s_rank[0] = (r - delta >= 1.0f) ? static_cast<uint32_t>(r - delta) : 0u;           // 0: none
+    s_rank[1] = (r + delta <= S - 1.0f) ? static_cast<uint32_t>(r + delta) + 1u : 0u;  // 0: none
+  }
+  __syncthreads();
   uint32_t bhi = kBuckets - 1, blo = 0;
   auto ld = [&](int i) { return hist[i]; };
-  if (r - delta >= 1.0) {
-    find_from_top<kBuckets>(ld, static_cast<uint32_t>(r - delta), scratch, res);
+  if (s_rank[0]) {
+    find_from_top<kBuckets>(ld, s_rank[0], scratch, res);
     bhi = res[0];
     __syncthreads();
   }
-  if (r + delta <= S - 1.0) {
-    find_from_top<kBuckets>(ld, static_cast<uint32_t>(r + delta) + 1u, scratch, res);
+  if (s_rank[1]) {
+    find_from_top<kBuckets>(ld, s_rank[1], scratch, res);
     blo = res[0];
   }
   if (tid == 0) {
@@ -506,6 +513,31 @@ __device__ __forceinline__ void grid_barrier(SelectState* st, uint32_t& epoch) {
   __syncthreads();
 }
 
+// Calls f(key) for the first `cc` keys of chunk c's slot; one thread, 16-byte loads, four in flight.
+template <int DT, typename F>
+__device__ __forceinline__ void for_slot_keys(const typename Elem<DT>::type* __restrict__ slots,
+                                              int c, uint32_t cc, F f) {
+  constexpr int kSlot = (DT == 0) ? 64 : 128;
+  constexpr int EPV = (DT == 0) ? 4 : 8;
+  const uint4* __restrict__ p = reinterpret_cast<const uint4*>(slots + static_cast<long long>(c) * kSlot);
+  const int nv = static_cast<int>((cc + EPV - 1) / EPV);
+  for (int v0 = 0; v0 < nv; v0 += 4) {
+    uint4 q[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) q[u] = (v0 + u < nv) ? __ldg(p + v0 + u) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+      for (int e = 0; e < EPV; ++e) {
+        const uint32_t idx = static_cast<uint32_t>((v0 + u) * EPV + e);
+        const uint32_t key = (DT == 0) ? w[e % 4] : ((w[e >> 1] >> (16 * (e & 1))) & 0xFFFFu);
+        if (idx < cc) f(key);
+      }
+    }
+  }
+}
+
 // prefix[c] = (elements kept for sure before chunk c) << 31 | (ties at the threshold before it),
 // c = 0 .. chunks (the last entry holds the totals).
 template <int DT>
@@ -519,7 +551,6 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
   using E = typename Elem<DT>::type;
   constexpr uint32_t kMask = Elem<DT>::kKeyMask;
   constexpr int EPV = 16 / sizeof(E);
-  constexpr int kSlot = (DT == 0) ? 64 : 128;
   constexpr long long kChunkElems = static_cast<long long>(kTileVecs) * EPV;
   __shared__ uint32_t s_hist[kBinsB];          // level B / fall-back digit histogram
   __shared__ uint32_t scratch[32];
@@ -530,8 +561,6 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
   const uint32_t lane = lane_id();
-  const int gwarp = blockIdx.x * 32 + warp;
-  const int gwarps = gridDim.x * 32;
   uint32_t epoch = 0;
   const uint32_t mode = __ldcg(&st->mode);
   uint32_t tau = 0, n_greater = 0;
@@ -593,13 +622,11 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
     for (int level = 0; shift > 0; ++level) {
       const uint32_t nb = shift < 11u ? shift : 11u, ns = shift - nb;
       uint32_t* gh = hist_b + level * kFbBins;
-      for (int c = gwarp; c < tiles; c += gwarps) {
-        const uint32_t cc = __ldg(cand_cnt + c);
-        for (uint32_t i = lane; i < cc; i += 32) {
-          const uint32_t rel =
-              static_cast<uint32_t>(__ldg(slots + static_cast<long long>(c) * kSlot + i)) - lo_key;
+      for (int c = blockIdx.x * kSelThreads + tid; c < tiles; c += gridDim.x * kSelThreads) {
+        for_slot_keys<DT>(slots, c, __ldg(cand_cnt + c), [&](uint32_t key) {
+          const uint32_t rel = key - lo_key;
           if ((rel >> shift) == pre) atomicAdd(&gh[(rel >> ns) & ((1u << nb) - 1u)], 1u);
-        }
+        });
       }
       grid_barrier(st, epoch);
       for (int i = tid; i < kFbBins; i += kSelThreads) s_hist[i] = __ldcg(gh + i);
@@ -624,27 +651,34 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
     hdr->tie_quota = static_cast<long long>(k) - n_greater;
   }
 
+  const long long quota = (mode == 2u) ? hdr->tie_quota : static_cast<long long>(k) - n_greater;
+
   // ---- per-chunk values; CTA b owns the chunks [b*per, (b+1)*per) ----
   const int per = (tiles + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
   const int c_begin = blockIdx.x * per < tiles ? blockIdx.x * per : tiles;
   const int c_end = c_begin + per < tiles ? c_begin + per : tiles;
   unsigned long long acc = 0;
-  for (int c = c_begin + warp; c < c_end; c += 32) {
-    uint32_t g = 0, q = 0;
-    if (mode != 1u) {
+  if (mode != 1u) {
+    // one thread per chunk: the listed keys above / equal to the threshold complete the counts
+    for (int c = c_begin + tid; c < c_end; c += kSelThreads) {
       const uint32_t cc = __ldg(cand_cnt + c), cg = __ldg(cnt_gt + c);
-      for (uint32_t i = lane; i < cc; i += 32) {
-        const uint32_t key = static_cast<uint32_t>(__ldg(slots + static_cast<long long>(c) * kSlot + i));
+      uint32_t g = cg, q = 0;
+      for_slot_keys<DT>(slots, c, cc, [&](uint32_t key) {
         g += key > tau ? 1u : 0u;
         q += key == tau ? 1u : 0u;
-      }
-      g = __reduce_add_sync(kFull, g) + cg;
-      q = __reduce_add_sync(kFull, q);
+      });
       if (tau == 0) {         // lo_key == 1: whatever is neither above nor inside the bracket is 0
         const long long left = n - static_cast<long long>(c) * kChunkElems;
         q += static_cast<uint32_t>(left < kChunkElems ? left : kChunkElems) - cg - cc;
       }
-    } else {
+      const unsigned long long v = (static_cast<unsigned long long>(g) << 31) | q;
+      val[c] = v;
+      acc += v;
+    }
+  } else {
+   for (int c = c_begin + warp; c < c_end; c += 32) {
+    uint32_t g = 0, q = 0;
+    {
 #pragma unroll
       for (int u = 0; u < kTileVecs / 32; ++u) {
         const long long base = (static_cast<long long>(c) * kTileVecs + u * 32 + lane) * EPV;
@@ -671,9 +705,10 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
       q = __reduce_add_sync(kFull, q);
     }
     const unsigned long long v = (static_cast<unsigned long long>(g) << 31) | q;
-    if (lane == 0) val[c] = v;
-    acc += v;            // identical in every lane
+    if (lane == 0) { val[c] = v; acc += v; }
+   }
   }
+  acc = warp_sum_u64(acc);
   if (lane == 0) s_tot[warp] = acc;
   __syncthreads();
   if (tid == 0) {
@@ -713,7 +748,13 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
       const unsigned long long up = __shfl_up_sync(kFull, incl, o);
       if (lane >= static_cast<uint32_t>(o)) incl += up;
     }
-    if (c < end) prefix[c] = carry + incl - v;
+    if (c < end) {
+      const unsigned long long ex = carry + incl - v;
+      prefix[c] = ex;
+      const long long eq_b = static_cast<long long>(ex & 0x7FFFFFFFull);
+      const long long eq_e = static_cast<long long>((ex + v) & 0x7FFFFFFFull);
+      if (eq_b < quota && eq_e > quota) st->boundary_plus1 = static_cast<uint32_t>(c) + 1u;
+    }
     carry += __shfl_sync(kFull, incl, 31);
   }
   if (c_end == tiles && c_begin < tiles) {
@@ -957,20 +998,15 @@ __global__ void __launch_bounds__(kCompactThreads)
 compact_boundary_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restrict__ hdr,
                         uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
                         uint32_t* __restrict__ offsets,
-                        const unsigned long long* __restrict__ prefix, int tiles) {
+                        const unsigned long long* __restrict__ prefix,
+                        const SelectState* __restrict__ st, int tiles) {
   using E = typename Elem<DT>::type;
   const E* __restrict__ x = reinterpret_cast<const E*>(xv);
   const long long quota = hdr->tie_quota;
   if (threadIdx.x == 0)   // the sentinel entry of the block offsets
     offsets[(n + SURGEON_BLOCK - 1) >> kBlockShift] = static_cast<uint32_t>(hdr->n_keep);
-  // first tile whose inclusive tie count exceeds the quota (the counts never decrease)
-  int lo = 0, hi = tiles;
-  while (lo < hi) {
-    const int mid = (lo + hi) >> 1;
-    if (static_cast<long long>(prefix[mid + 1] & kCountMask) > quota) hi = mid;
-    else lo = mid + 1;
-  }
-  if (lo >= tiles) return;
+  const int lo = static_cast<int>(st->boundary_plus1) - 1;   // found by the count kernel's scan
+  if (lo < 0 || lo >= tiles) return;
   const unsigned long long pb = prefix[lo];
   const long long eq_b = static_cast<long long>(pb & kCountMask);
   if (eq_b >= quota) return;                            // the quota ends exactly between tiles
@@ -1312,7 +1348,8 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
     }
     {
       // cooperative launch: every CTA must be resident for the grid-wide barriers
-      long long want = (L.tiles + 31) / 32;
+      // list path: one thread per chunk; fall-back (known for small tensors): all SMs read x
+      const long long want = streamed ? (L.tiles + kSelThreads - 1) / kSelThreads : (L.tiles + 31) / 32;
       const int grid = static_cast<int>(want < 1 ? 1 : (want < sms ? want : sms));
       const void* xa = x;
       long long na = n;
@@ -1342,7 +1379,7 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
       compact_small_kernel<DT><<<static_cast<unsigned>(L.tiles), kCompactThreads, 0, stream>>>(
           x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix);
     compact_boundary_kernel<DT><<<1, kCompactThreads, 0, stream>>>(
-        x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix, n_chunks);
+        x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix, st, n_chunks);
     note_launches(2);
   }
   return cudaGetLastError();
