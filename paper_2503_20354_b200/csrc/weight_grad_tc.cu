@@ -449,7 +449,14 @@ static size_t fast_partial_bytes(const FastParams& f) {
   return (b + 255) & ~static_cast<size_t>(255);
 }
 
+static size_t direct_partial_bytes(const DirectParams& p) {
+  const size_t b = static_cast<size_t>(p.splits) * p.O * p.C * sizeof(float);
+  return (b + 255) & ~static_cast<size_t>(255);
+}
+
 size_t weight_grad_tc_workspace(const surgeon_layer_desc& d) {
+  DirectParams dp;
+  if (plan_direct(d, &dp)) return kStatusBytes + direct_partial_bytes(dp) + direct_grad_bf16_bytes(dp);
   FastParams f;
   if (plan_conv_fast(d, &f))
     return kStatusBytes + fast_partial_bytes(f) + conv_fast_grad_bf16_bytes(f);
@@ -465,6 +472,17 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
   float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes);
   cudaError_t e = cudaMemsetAsync(status, 0, kStatusBytes, stream);
   if (e != cudaSuccess) return e;
+  DirectParams dp;
+  if (plan_direct(d, &dp)) {
+    void* grad_bf16 = reinterpret_cast<char*>(partial) + direct_partial_bytes(dp);
+    e = launch_direct(act, dp, grad_out, grad_bf16, partial, status, stream);
+    if (e != cudaSuccess) return e;
+    const long long mn = static_cast<long long>(dp.O) * dp.C;
+    reduce_splits_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
+        partial, mn, dp.splits, dw, accumulate, status, act.header);
+    note_launches(1);
+    return cudaGetLastError();
+  }
   FastParams f;
   if (plan_conv_fast(d, &f)) {
     void* grad_bf16 = reinterpret_cast<char*>(partial) + fast_partial_bytes(f);

@@ -508,6 +508,15 @@ bool plan_conv_fast(const surgeon_layer_desc& d, FastParams* out) {
   return true;
 }
 
+cudaError_t launch_grad_to_bf16(const float* g, long long n, void* out_bf16, cudaStream_t stream) {
+  const long long want = (n / 8 + 255) / 256;
+  const long long cap = 16LL * sm_count();
+  const int grid = static_cast<int>(want < 1 ? 1 : (want > cap ? cap : want));
+  grad_to_bf16_kernel<<<grid, 256, 0, stream>>>(g, n, static_cast<unsigned short*>(out_bf16));
+  note_launches(1);
+  return cudaGetLastError();
+}
+
 size_t conv_fast_grad_bf16_bytes(const FastParams& p) {
   const size_t b = static_cast<size_t>(p.B) * p.O * p.P * 2;
   return (b + 255) & ~static_cast<size_t>(255);

@@ -29,4 +29,26 @@ cudaError_t launch_conv_fast(const surgeon_compressed& act, const FastParams& p,
                              const float* grad_out, void* grad_bf16, float* partial,
                              uint32_t* status, cudaStream_t stream);
 
+// fp32 -> bf16 (round to nearest even) copy of n elements, as one streaming kernel.
+cudaError_t launch_grad_to_bf16(const float* g, long long n, void* out_bf16, cudaStream_t stream);
+
+// ---- layers whose im2col operand is the activation itself (weight_grad_tc_direct.cu) ----------
+struct DirectParams {
+  int mode;                 // 0 = linear [T, C] (MN-major operands), 1 = conv 1x1 stride 1 (K-major)
+  int C, O;                 // input / output channels
+  int T;                    // linear: rows; conv: positions per image
+  int imgs;                 // conv: batch; linear: 1
+  int acc_n, n_acc, n_cols; // columns per accumulator, accumulators per CTA, their product
+  int m_tiles, n_tiles, splits;
+  int tiles_per_img, total_ktiles, ktiles_per_split;
+  int stages, tmem_cols, smem_bytes;
+  long long n_words;        // words of the bitmap (filled by the launcher)
+};
+bool plan_direct(const surgeon_layer_desc& d, DirectParams* out);
+size_t direct_grad_bf16_bytes(const DirectParams& p);
+// partial = [splits][O][C] fp32, status = one zeroed word.
+cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& p,
+                          const float* grad_out, void* grad_bf16, float* partial,
+                          uint32_t* status, cudaStream_t stream);
+
 }  // namespace surgeon
