@@ -340,15 +340,17 @@ dw_tc_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ value
   }
 
   // ================= epilogue: TMEM -> scratch partial tile =================
-  if (warp >= 1 && warp <= 4) {
-    const bool done = mbar_wait(acc_bar, 0, 256);
+  if (warp >= 1) {
+    // 8 warps: a warp may read the 32 TMEM lanes of its quarter (warp % 4); the two warps of a
+    // quarter take alternate groups of 16 columns
+    const bool done = mbar_wait(acc_bar, 0, 64);
     tc_fence_after();
     if (done && !*fail) {
       const int lane_grp = warp & 3;              // TMEM lanes this warp may read
       const int row = lane_grp * 32 + static_cast<int>(lane);
       const int nn = nn0 + row;
       float* out = partial + static_cast<long long>(split) * p.O * p.n_gemm;
-      for (int col = 0; col < p.tile_n; col += 16) {
+      for (int col = 16 * ((warp - 1) >> 2); col < p.tile_n; col += 32) {
         uint32_t r[16];
         tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_grp * 32) << 16) + col, r);
         if (nn < p.n_gemm) {

@@ -378,15 +378,17 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
   }
 
   // ================= epilogue: TMEM -> scratch partial tile =================
-  if (warp >= 1 && warp <= 4) {
-    const bool done = mbar_wait(acc_bar, 0, 256);
+  if (warp >= 1) {
+    // 16 warps: a warp may read the 32 TMEM lanes of its quarter (warp % 4); the four warps of a
+    // quarter take every fourth group of 16 columns
+    const bool done = mbar_wait(acc_bar, 0, 64);
     tc_fence_after();
     if (done && !*fail) {
       const int lane_grp = warp & 3;
       const int row = lane_grp * 32 + static_cast<int>(lane);
       const int nn = nn0 + row;
       float* out = partial + static_cast<long long>(split) * p.O * p.n_gemm;
-      for (int col = 0; col < n_cols; col += 16) {
+      for (int col = 16 * ((warp - 1) >> 2); col < n_cols; col += 64) {
         uint32_t r[16];
         tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_grp * 32) << 16) + col, r);
         if (nn < p.n_gemm) {
@@ -423,6 +425,28 @@ grad_to_bf16_kernel(const float* __restrict__ g, long long n, unsigned short* __
   if (blockIdx.x == 0)
     for (long long j = (n8 << 3) + threadIdx.x; j < n; j += blockDim.x)
       out[j] = static_cast<unsigned short>(pack_bf16x2(g[j], 0.0f) & 0xFFFFu);
+}
+
+// rows of `len` floats -> rows of `pitch` bf16 (pitch a multiple of 8, padding zero)
+__global__ void __launch_bounds__(256)
+grad_to_bf16_rows_kernel(const float* __restrict__ g, long long rows, int len, int pitch,
+                         unsigned short* __restrict__ out) {
+  const int per_row = pitch >> 3;
+  const long long total = rows * per_row;
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+       i += stride) {
+    const long long r = i / per_row;
+    const int c0 = static_cast<int>(i - r * per_row) * 8;
+    const float* src = g + r * len + c0;
+    float v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = (c0 + e < len) ? __ldg(src + e) : 0.0f;
+    uint4 o;
+    o.x = pack_bf16x2(v[0], v[1]); o.y = pack_bf16x2(v[2], v[3]);
+    o.z = pack_bf16x2(v[4], v[5]); o.w = pack_bf16x2(v[6], v[7]);
+    reinterpret_cast<uint4*>(out)[i] = o;
+  }
 }
 
 using TensorMapEncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -513,6 +537,17 @@ cudaError_t launch_grad_to_bf16(const float* g, long long n, void* out_bf16, cud
   const long long cap = 16LL * sm_count();
   const int grid = static_cast<int>(want < 1 ? 1 : (want > cap ? cap : want));
   grad_to_bf16_kernel<<<grid, 256, 0, stream>>>(g, n, static_cast<unsigned short*>(out_bf16));
+  note_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_grad_to_bf16_rows(const float* g, long long rows, int len, int pitch,
+                                     void* out_bf16, cudaStream_t stream) {
+  const long long want = (rows * (pitch >> 3) + 255) / 256;
+  const long long cap = 16LL * sm_count();
+  const int grid = static_cast<int>(want < 1 ? 1 : (want > cap ? cap : want));
+  grad_to_bf16_rows_kernel<<<grid, 256, 0, stream>>>(g, rows, len, pitch,
+                                                     static_cast<unsigned short*>(out_bf16));
   note_launches(1);
   return cudaGetLastError();
 }

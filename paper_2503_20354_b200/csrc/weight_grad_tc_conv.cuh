@@ -31,18 +31,24 @@ cudaError_t launch_conv_fast(const surgeon_compressed& act, const FastParams& p,
 
 // fp32 -> bf16 (round to nearest even) copy of n elements, as one streaming kernel.
 cudaError_t launch_grad_to_bf16(const float* g, long long n, void* out_bf16, cudaStream_t stream);
+// The same for `rows` rows of `len` elements, written with a row pitch of `pitch` >= len
+// elements (a multiple of 8); the padding is zero.
+cudaError_t launch_grad_to_bf16_rows(const float* g, long long rows, int len, int pitch,
+                                     void* out_bf16, cudaStream_t stream);
 
 // ---- layers whose im2col operand is the activation itself (weight_grad_tc_direct.cu) ----------
 struct DirectParams {
   int mode;                 // 0 = linear [T, C] (MN-major operands), 1 = conv 1x1 stride 1 (K-major)
   int C, O;                 // input / output channels
   int T;                    // linear: rows; conv: positions per image
+  int pitch;                // elements per row of the bf16 gradient copy
   int imgs;                 // conv: batch; linear: 1
   int acc_n, n_acc, n_cols; // columns per accumulator, accumulators per CTA, their product
   int m_tiles, n_tiles, splits;
   int tiles_per_img, total_ktiles, ktiles_per_split;
   int stages, tmem_cols, smem_bytes;
   long long n_words;        // words of the bitmap (filled by the launcher)
+  unsigned partial_blk;     // index of the bitmap's last block if it is partial, else 0xFFFFFFFF
 };
 bool plan_direct(const surgeon_layer_desc& d, DirectParams* out);
 size_t direct_grad_bf16_bytes(const DirectParams& p);

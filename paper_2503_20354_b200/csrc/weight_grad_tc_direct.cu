@@ -11,11 +11,12 @@
 //            (rows of 64 channels = 128 bytes, one row per k, 128-byte swizzle);
 //   conv   : A[b, c, p] and G[b, o, p] are contiguous along p -> both operands K-major.
 // The output gradient is converted to bf16 once by a streaming pre-pass and arrives by TMA.
-// The activation operand is rebuilt from the compressed store by 16 producer warps: a thread
-// owns units of 8 consecutive elements, finds their rank in the packed vector from the block
-// offset and the 128 bitmap bits of their block, gathers the kept values and writes one 16-byte
-// piece of the swizzled tile.  The loads of a unit are issued two units ahead of its store
-// (metadata) and one unit ahead (values), so their latency overlaps the work on earlier units.
+// The activation operand is rebuilt from the compressed store by 16 producer warps, 8 per K-tile,
+// two tiles in flight: a lane owns a run of 32 consecutive elements (64 bytes of the swizzled
+// tile), finds the rank of its first kept element from the block offset and the block's bitmap
+// words, zero-fills its 64 bytes and scatters the kept values into them, so the work is
+// proportional to the number of kept elements.  The metadata of a lane's next run is fetched
+// while the current one is rebuilt.
 // One thread issues the MMAs, one the TMA loads; split-K partial tiles are reduced in a fixed
 // order by the caller.  Every wait is bounded and ends in SURGEON_ERR_TIMEOUT.
 #include <cuda.h>
@@ -36,8 +37,6 @@ constexpr int kProdWarps = 16;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kThreads = 64 + kProdThreads;     // warp 0: MMA, warp 1: TMA, warps 2..17: producers
 constexpr int kMaxStages = 4;
-constexpr int kUnitsPerTile = kTileM * kTileK / 8;            // 1024
-constexpr int kUnitsPerThread = kUnitsPerTile / kProdThreads; // 2
 constexpr int kATileBytes = kTileM * kTileK * 2;              // 16 KB
 
 // Shared-memory matrix descriptor of an MN-major operand with 128-byte swizzle: rows of 64
@@ -53,48 +52,30 @@ __device__ __forceinline__ uint64_t make_desc_mn(uint32_t saddr) {
   return d;
 }
 
-// What a thread needs to decompress one unit: where it goes, and the raw metadata loads.
-struct UnitMeta {
-  uint32_t dst;        // byte offset inside the A tile; 0xFFFFFFFF = write zeros at `zdst`
-  uint32_t zdst;
-  uint32_t bitpos;     // position of the unit's first bit inside its 128-bit block
-  uint32_t base;       // kept elements before the block
-  uint4 words;         // the block's 128 bitmap bits
+// What a lane fetches for the 32 consecutive elements ("word") it rebuilds: the kept count before
+// their 128-element block, the block's bitmap words, and the bitmap word after the one the run
+// starts in (the run need not start on a word boundary).
+struct WordRaw {
+  uint32_t base;
+  uint32_t next;
+  uint4 words;
+  uint32_t j;          // flat index of the run's first element
+  uint32_t nvalid;     // elements of the run that exist (0: nothing to do)
 };
 
+// Predicated load of packed value `idx` (zero when !on); no branch.
 template <int DT>
-__device__ __forceinline__ void gather_unit(const UnitMeta& m, const void* __restrict__ values,
-                                            uint32_t (&v)[8]) {
-  const uint32_t w[4] = {m.words.x, m.words.y, m.words.z, m.words.w};
-  const uint32_t wi = m.bitpos >> 5, sh = m.bitpos & 31;
-  uint32_t rank = m.base;
-#pragma unroll
-  for (int j = 0; j < 3; ++j) rank += (static_cast<uint32_t>(j) < wi) ? __popc(w[j]) : 0u;
-  const uint32_t word = wi == 0 ? w[0] : (wi == 1 ? w[1] : (wi == 2 ? w[2] : w[3]));
-  rank += __popc(word & ((1u << sh) - 1u));
-  const uint32_t bits = (m.dst == 0xFFFFFFFFu) ? 0u : ((word >> sh) & 0xFFu);
-#pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    const bool on = (bits >> e) & 1u;
-    const uint32_t idx = rank + __popc(bits & ((1u << e) - 1u));
-    if (DT == 0) v[e] = on ? __ldg(reinterpret_cast<const uint32_t*>(values) + idx) : 0u;
-    else v[e] = on ? static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(values) + idx)) : 0u;
-  }
-}
-
-template <int DT>
-__device__ __forceinline__ uint4 pack_unit(const uint32_t (&v)[8]) {
-  uint4 o;
-  if (DT == 0) {
-    o.x = pack_bf16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
-    o.y = pack_bf16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
-    o.z = pack_bf16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
-    o.w = pack_bf16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
-  } else {
-    o.x = v[0] | (v[1] << 16); o.y = v[2] | (v[3] << 16);
-    o.z = v[4] | (v[5] << 16); o.w = v[6] | (v[7] << 16);
-  }
-  return o;
+__device__ __forceinline__ uint32_t ld_packed(const void* __restrict__ values, uint32_t idx, bool on) {
+  uint32_t r = 0;
+  const unsigned char* src =
+      reinterpret_cast<const unsigned char*>(values) + static_cast<size_t>(idx) * (DT == 0 ? 4 : 2);
+  if (DT == 0)
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q ld.global.nc.u32 %0, [%1];\n\t}"
+                 : "+r"(r) : "l"(src), "r"(static_cast<uint32_t>(on)));
+  else
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q ld.global.nc.u16 %0, [%1];\n\t}"
+                 : "+r"(r) : "l"(src), "r"(static_cast<uint32_t>(on)));
+  return r;
 }
 
 template <int DT, int MODE>
@@ -126,7 +107,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   if (tid == 0) {
     tma_prefetch_desc(&grad_map);
     for (int s = 0; s < p.stages; ++s) {
-      mbar_init(full_bar + 8 * s, kProdWarps + 1);   // 16 producer warps + the TMA thread
+      mbar_init(full_bar + 8 * s, kProdWarps / 2 + 1);   // the 8 warps of a tile + the TMA thread
       mbar_init(empty_bar + 8 * s, 1);
     }
     mbar_init(acc_bar, 1);
@@ -202,96 +183,122 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
     __syncwarp();
   } else {
     // ================= producers =================
-    const int ptid = tid - 64;
-    const int n_units = n_kt * kUnitsPerThread;
-    // unit i of this thread: K-tile kt_begin + i/2, unit index (i&1)*512 + ptid inside the tile
-    auto load_meta = [&](int i) {
-      UnitMeta m;
-      const int kt = kt_begin + (i >> 1);
-      const int u = (i & 1) * kProdThreads + ptid;
+    // Warps 2..9 rebuild the even K-tiles of this CTA's range, warps 10..17 the odd ones.  A lane
+    // owns one run of 32 consecutive elements per tile (linear: 32 channels of one row t; conv: 32
+    // positions of one channel) = 64 bytes of the operand tile: it zero-fills them and then
+    // scatters the kept values, whose count is what the work is proportional to.
+    const int pw = warp - 2;
+    const int wg = pw >> 3, w8 = pw & 7;
+    int row, part;                       // tile row and which run of the row
+    if (MODE == 0) { row = 8 * w8 + static_cast<int>(lane >> 2); part = lane & 3; }   // k-row, 32-ch quarter
+    else { row = 16 * w8 + static_cast<int>(lane >> 1); part = lane & 1; }            // channel, 32-pos half
+    const uint32_t xr = row & 7;
+    const uint32_t y = (MODE == 0) ? (part & 1) * 4 : part * 4;     // first 16-byte chunk of the run
+    const uint32_t rowbase = (MODE == 0) ? (part >> 1) * (kTileK * 128) + row * 128 : row * 128;
+    auto fetch = [&](int it) {
+      WordRaw r;
+      r.base = 0; r.next = 0; r.words = make_uint4(0, 0, 0, 0); r.j = 0; r.nvalid = 0;
+      const int kt = kt_begin + it;
       long long j;
-      bool valid;
+      int nvalid;
       if (MODE == 0) {
-        const int k = u >> 4, h = u & 15;                   // k-row, 8-channel unit of the row
-        const long long t = static_cast<long long>(kt) * kTileK + k;
-        const int c = c0 + 8 * h;
-        valid = t < p.T && c < p.C;
+        const long long t = static_cast<long long>(kt) * kTileK + row;
+        const int c = c0 + 32 * part;
+        nvalid = (t < p.T) ? min(32, p.C - c) : 0;
         j = t * p.C + c;
-        m.zdst = static_cast<uint32_t>((h >> 3) * (kTileK * 128) + k * 128 + (((h & 7) ^ (k & 7)) << 4));
       } else {
-        const int row = u >> 3, chunk = u & 7;              // channel row, 8-position unit
         const int img = kt / p.tiles_per_img;
-        const int pp = (kt - img * p.tiles_per_img) * kTileK + 8 * chunk;
+        const int pp = (kt - img * p.tiles_per_img) * kTileK + 32 * part;
         const int c = c0 + row;
-        valid = c < p.C && pp < p.T;
+        nvalid = (c < p.C) ? min(32, p.T - pp) : 0;
         j = (static_cast<long long>(img) * p.C + c) * p.T + pp;
-        m.zdst = tile_off(row, chunk);
       }
-      m.dst = valid ? m.zdst : 0xFFFFFFFFu;
-      m.bitpos = 0; m.base = 0; m.words = make_uint4(0, 0, 0, 0);
-      if (valid) {
-        const long long blk = j >> kBlockShift;
-        m.bitpos = static_cast<uint32_t>(j) & (SURGEON_BLOCK - 1);
-        m.base = __ldg(offsets + blk);
-        if (blk * kBlockWords + kBlockWords <= p.n_words) {
-          m.words = __ldg(reinterpret_cast<const uint4*>(bitmap) + blk);
+      if (nvalid > 0) {
+        r.nvalid = static_cast<uint32_t>(nvalid);
+        r.j = static_cast<uint32_t>(j);
+        const uint32_t blk = r.j >> kBlockShift;
+        const long long wi = r.j >> 5;
+        r.base = __ldg(offsets + blk);
+        if (blk != p.partial_blk) {
+          r.words = __ldg(reinterpret_cast<const uint4*>(bitmap) + blk);
         } else {                                   // the last, partial block of the bitmap
-          const long long w0 = blk * kBlockWords;
-          m.words.x = __ldg(bitmap + w0);
-          m.words.y = (w0 + 1 < p.n_words) ? __ldg(bitmap + w0 + 1) : 0u;
-          m.words.z = (w0 + 2 < p.n_words) ? __ldg(bitmap + w0 + 2) : 0u;
-          m.words.w = 0u;
+          const long long w0 = static_cast<long long>(blk) * kBlockWords;
+          r.words.x = __ldg(bitmap + w0);
+          r.words.y = (w0 + 1 < p.n_words) ? __ldg(bitmap + w0 + 1) : 0u;
+          r.words.z = (w0 + 2 < p.n_words) ? __ldg(bitmap + w0 + 2) : 0u;
         }
+        if ((r.j & 31u) && wi + 1 < p.n_words) r.next = __ldg(bitmap + wi + 1);
       }
-      return m;
+      return r;
     };
-    UnitMeta m_next = {};      // metadata of unit i+1
-    uint32_t v_cur[8];         // values of unit i
-    UnitMeta m_cur = {};
-    if (n_units > 0) {
-      m_cur = load_meta(0);
-      m_next = (n_units > 1) ? load_meta(1) : m_cur;
-      gather_unit<DT>(m_cur, values, v_cur);
-    }
-    bool ok = true;
-    for (int i = 0; i < n_units; ++i) {
-      UnitMeta m_after = {};
-      if (i + 2 < n_units) m_after = load_meta(i + 2);
-      uint32_t v_next[8];
-      if (i + 1 < n_units) gather_unit<DT>(m_next, values, v_next);
-      const int it = i >> 1;
+    const int first_it = wg;
+    WordRaw cur = {};
+    if (first_it < n_kt) cur = fetch(first_it);
+    for (int it = first_it; it < n_kt; it += 2) {
+      WordRaw nxt = {};
+      if (it + 2 < n_kt) nxt = fetch(it + 2);       // in flight while this tile is rebuilt
+      // bits of the run and rank of its first kept element
+      const uint32_t wq = (cur.j >> 5) & 3, sh = cur.j & 31;
+      uint32_t rank = cur.base;
+      rank += wq > 0 ? __popc(cur.words.x) : 0u;
+      rank += wq > 1 ? __popc(cur.words.y) : 0u;
+      rank += wq > 2 ? __popc(cur.words.z) : 0u;
+      const uint32_t w0 = wq == 0 ? cur.words.x : (wq == 1 ? cur.words.y : (wq == 2 ? cur.words.z : cur.words.w));
+      const uint32_t w1 = wq == 3 ? cur.next : (wq == 0 ? cur.words.y : (wq == 1 ? cur.words.z : cur.words.w));
+      rank += __popc(w0 & ((1u << sh) - 1u));
+      uint32_t bits = __funnelshift_r(w0, w1, sh);
+      bits = cur.nvalid >= 32 ? bits : (bits & ((1u << cur.nvalid) - 1u));
+      const uint32_t count = __popc(bits);
+      const uint32_t max_count = __reduce_max_sync(0xFFFFFFFFu, count);
+      uint32_t v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = ld_packed<DT>(values, rank + i, static_cast<uint32_t>(i) < count);
+
       const int s = it % p.stages;
-      if ((i & 1) == 0 && it >= p.stages) {
-        if (!mbar_wait(empty_bar + 8 * s, ((it / p.stages) - 1) & 1)) {
-          fail = 1;
-          atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+      if (it >= p.stages && !mbar_wait(empty_bar + 8 * s, ((it / p.stages) - 1) & 1, 32)) {
+        fail = 1;
+        atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+      }
+      if (fail) break;
+      unsigned char* dst_row = smem + s * stage_bytes + rowbase;
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<uint4*>(dst_row + (((y + q) ^ xr) << 4)) = make_uint4(0, 0, 0, 0);
+      uint32_t left = bits;
+      for (uint32_t g = 0; g < max_count; g += 8) {
+        if (g > 0) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) v[i] = ld_packed<DT>(values, rank + g + i, g + i < count);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (g + i < count) {
+            const uint32_t b = __ffs(left) - 1;
+            left &= left - 1;
+            const unsigned short h = (DT == 0) ? to_bf16_bits(__uint_as_float(v[i]))
+                                               : static_cast<unsigned short>(v[i]);
+            *reinterpret_cast<unsigned short*>(dst_row + (((y + (b >> 3)) ^ xr) << 4) + ((b & 7) << 1)) = h;
+          }
         }
       }
-      if (fail) { ok = false; break; }
-      unsigned char* a_tile = smem + s * stage_bytes;
-      *reinterpret_cast<uint4*>(a_tile + m_cur.zdst) = pack_unit<DT>(v_cur);
-      if (i & 1) {
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(full_bar + 8 * s);
-      }
-      m_cur = m_next;
-      m_next = m_after;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) v_cur[e] = v_next[e];
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full_bar + 8 * s);
+      cur = nxt;
     }
-    (void)ok;
   }
 
   // ================= epilogue: TMEM -> scratch partial tile =================
-  if (warp >= 2 && warp <= 5) {
-    const bool done = mbar_wait(acc_bar, 0, 256);
+  if (warp >= 2) {
+    // 16 warps: a warp may read the 32 TMEM lanes of its quarter (warp % 4); the four warps of a
+    // quarter take every fourth group of 16 columns
+    const bool done = mbar_wait(acc_bar, 0, 64);
     tc_fence_after();
     if (done && !fail) {
-      const int lane_grp = warp & 3;              // TMEM lanes this warp may read
+      const int lane_grp = warp & 3;
       const int c = c0 + lane_grp * 32 + static_cast<int>(lane);
       float* out = partial + static_cast<long long>(split) * p.O * p.C;
-      for (int col = 0; col < p.n_cols; col += 16) {
+      for (int col = 16 * ((warp - 2) >> 2); col < p.n_cols; col += 64) {
         uint32_t r[16];
         tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_grp * 32) << 16) + col, r);
         if (c < p.C) {
@@ -327,11 +334,11 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   } else if (d.kind == 1 && d.kh == 1 && d.kw == 1 && d.stride == 1 && d.pad == 0) {
     p.mode = 1;
     p.T = d.h * d.w; p.imgs = d.batch;
-    if (p.T % 8 != 0) return false;                          // units never straddle a plane
   } else {
     return false;
   }
   p.C = d.c_in; p.O = d.c_out;
+  p.pitch = (p.mode == 0) ? p.O : (p.T + 7) / 8 * 8;   // row pitch of the bf16 gradient copy
   if (p.mode == 0) {
     // columns come in slabs of 64; per CTA two accumulators of 192 or 128 columns, or one small one
     const int g = (p.O + 63) / 64;
@@ -383,7 +390,8 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
 }
 
 size_t direct_grad_bf16_bytes(const DirectParams& p) {
-  const size_t b = static_cast<size_t>(p.imgs) * p.O * p.T * 2;
+  const size_t b = (p.mode == 0) ? static_cast<size_t>(p.T) * p.O * 2
+                                 : static_cast<size_t>(p.imgs) * p.O * p.pitch * 2;
   return (b + 255) & ~static_cast<size_t>(255);
 }
 
@@ -392,8 +400,13 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
                           uint32_t* status, cudaStream_t stream) {
   DirectParams p = plan;
   p.n_words = (act.n + 31) / 32;
-  const long long gn = static_cast<long long>(p.imgs) * p.O * p.T;
-  cudaError_t e = launch_grad_to_bf16(grad_out, gn, grad_bf16, stream);
+  p.partial_blk = (act.n % SURGEON_BLOCK) ? static_cast<unsigned>(act.n / SURGEON_BLOCK) : 0xFFFFFFFFu;
+  cudaError_t e;
+  if (p.mode == 1 && p.pitch != p.T)     // rows padded to a 16-byte pitch for the tensor map
+    e = launch_grad_to_bf16_rows(grad_out, static_cast<long long>(p.imgs) * p.O, p.T, p.pitch,
+                                 grad_bf16, stream);
+  else
+    e = launch_grad_to_bf16(grad_out, static_cast<long long>(p.imgs) * p.O * p.T, grad_bf16, stream);
   if (e != cudaSuccess) return e;
   const EncodeFn encode = reinterpret_cast<EncodeFn>(tensor_map_encode_fn());
   if (!encode) return cudaErrorNotSupported;
@@ -410,8 +423,8 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
   } else {
     const cuuint64_t dims[3] = {static_cast<cuuint64_t>(p.T), static_cast<cuuint64_t>(p.O),
                                 static_cast<cuuint64_t>(p.imgs)};
-    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(p.T) * 2,
-                                   static_cast<cuuint64_t>(p.T) * p.O * 2};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(p.pitch) * 2,
+                                   static_cast<cuuint64_t>(p.pitch) * p.O * 2};
     const cuuint32_t box[3] = {static_cast<cuuint32_t>(kTileK), static_cast<cuuint32_t>(p.acc_n), 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, grad_bf16, dims, strides, box, estr,

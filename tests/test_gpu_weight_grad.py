@@ -72,6 +72,13 @@ SHAPES = [
     W.linear("fc", 64, 2048, 1000, dist="abs_normal", dt=W.F32),
     W.linear("tokens", 2 * 197, 768, 256, dist="normal", dt=W.F32),
     W.linear("tiny", 5, 7, 3, dist="normal", dt=W.F32),
+    # layers whose im2col operand is the activation itself (the direct kernel): linear layers
+    # with two 192-column accumulators, ragged channel / row counts; 1x1 convs on 14x14 and 7x7
+    # maps (the bf16 gradient copy gets a padded row pitch)
+    W.linear("lin_two_acc192", 3 * 64 + 17, 256, 768, dist="normal", dt=W.F32),
+    W.linear("lin_c40_o520", 200, 40, 520, dist="gelu_normal", dt=W.F32),
+    W.conv("d1x1_hw14", 3, 136, 14, 264, 1, 1, 0),
+    W.conv("d1x1_hw7", 5, 72, 7, 48, 1, 1, 0),
 ]
 
 
