@@ -226,6 +226,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
           r.words.x = __ldg(bitmap + w0);
           r.words.y = (w0 + 1 < p.n_words) ? __ldg(bitmap + w0 + 1) : 0u;
           r.words.z = (w0 + 2 < p.n_words) ? __ldg(bitmap + w0 + 2) : 0u;
+          r.words.w = (w0 + 3 < p.n_words) ? __ldg(bitmap + w0 + 3) : 0u;
         }
         if ((r.j & 31u) && wi + 1 < p.n_words) r.next = __ldg(bitmap + wi + 1);
       }
