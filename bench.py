@@ -7,7 +7,7 @@ saved activation (Algorithm 1: prune and decompose steps), and the weight gradie
 compressed store (its Reshape and gradient steps).  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                  [--workload wrn28|tiny|resnet50|vit] [--batch B] [--path tc|fp32]
+                  [--workload wrn28|tiny|resnet50|vit|sweep] [--batch B] [--path tc|fp32]
 
 N > 1 (launched with torch.distributed.run): every rank runs an independent replica of the
 step on its own GPU (the path has no exchange step); time is the max over ranks.
@@ -66,7 +66,7 @@ def prune_alg_bytes(layer, n_keep: int) -> int:
     one to emit), the bitmap, the packed values and the block offsets."""
     es = 4 if layer.dt == 0 else 2
     n = layer.n_act
-    return 2 * n * es + (n + 7) // 8 + n_keep * es + 8 * ((n + 1023) // 1024 + 1)
+    return 2 * n * es + (n + 7) // 8 + n_keep * es + 4 * ((n + 127) // 128 + 1)
 
 
 class ClockSampler:
@@ -189,12 +189,69 @@ class Stack:
         if ev: ev[2].record()
 
 
+def run_sweep(args, device):
+    """Prune+compact bandwidth sweep: single tensors of 2^20 .. 2^max elements, fp32 and bf16, four
+    value distributions, four ratios; L2 flushed (256 MB written) before every timed call."""
+    from paper_2503_20354_b200 import binding as B
+    from paper_2503_20354_b200 import workloads as W
+    peaks = load_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    sizes = [20, 22, 24, 26, 28, 30][: args.sweep_sizes]
+    cases = []
+    launches0 = B.surgeon_launch_count()
+    for bf16 in (False, True):
+        for lg in sizes:
+            n = 1 << lg
+            es = 2 if bf16 else 4
+            for dist in ("relu_normal", "normal", "student_t2", "ties16"):
+                x = W.draw(dist, n, args.seed, device=device)
+                if bf16:
+                    x = x.to(torch.bfloat16)
+                out = B.CompressedActivation(n, B.dtype_code(x.dtype), 0.0, device)
+                ws = torch.empty(out.sizes.workspace_bytes, dtype=torch.uint8, device=device)
+                for ratio in (0.1, 0.5, 0.9, 0.99):
+                    ts = []
+                    for it in range(args.warmup + args.steps):
+                        flush.zero_()
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                        B.surgeon_prune_compact(x, ratio, out=out, workspace=ws)
+                        e1.record()
+                        e1.synchronize()
+                        if it >= args.warmup:
+                            ts.append(e0.elapsed_time(e1))
+                    ms = float(np.median(ts))
+                    k = out.sizes.n_keep
+                    balg = 2 * n * es + n // 8 + k * es + 4 * (n // 128 + 1)
+                    if out.read_header().status != 0:
+                        raise SystemExit("device status in sweep case")
+                    cases.append({"dtype": "bf16" if bf16 else "f32", "log2_n": lg, "dist": dist, "ratio": ratio,
+                                  "us": round(ms * 1e3, 1), "GB/s": round(balg / ms / 1e6, 1)})
+                del x, out, ws
+    big = [c["GB/s"] for c in cases if c["log2_n"] == sizes[-1]]
+    val = float(np.median(big))
+    print(json.dumps({
+        "metric": METRIC, "value": round(val, 1), "unit": "GB/s (algorithmic bytes / call time, median at the largest size)",
+        "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+        "config": {"workload": "prune+compact sweep, 2^20..2^%d elements, fp32 and bf16" % sizes[-1],
+                   "l2": "flushed before every call"},
+        "roofline": {"kernel": "surgeon_prune_compact (all kernels of a call)", "bound": "hbm", "achieved": round(val, 1),
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(val / float(peaks["hbm_gbs"]), 4),
+                     "traffic": None, "peak_source": peaks["_source"] + " copy bandwidth"},
+        "gpu_launches": int(B.surgeon_launch_count() - launches0), "cases": cases}))
+
+
 def run_ours(args, rank, world, local):
     from paper_2503_20354_b200 import binding as B
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     B.lib()
     device = torch.device("cuda", local if world > 1 else 0)
+    if args.workload == "sweep":
+        if rank == 0:
+            run_sweep(args, device)
+        return
     layers, desc_text = get_layers(args.workload, args.batch)
     path = B.PATH_FP32 if args.path == "fp32" else B.PATH_TENSOR_CORE
     stack = Stack(layers, path, args.seed + rank, device)
@@ -399,7 +456,8 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="wrn28", choices=["wrn28", "tiny", "resnet50", "vit"])
+    ap.add_argument("--workload", default="wrn28", choices=["wrn28", "tiny", "resnet50", "vit", "sweep"])
+    ap.add_argument("--sweep-sizes", type=int, default=5, help="how many of 2^20,22,24,26,28,30 the sweep covers")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--path", default="tc", choices=["tc", "fp32"])
     ap.add_argument("--seed", type=int, default=0)
