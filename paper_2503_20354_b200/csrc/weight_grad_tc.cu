@@ -192,9 +192,9 @@ dw_tc_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ value
     bool ok = true;
     for (int it = 0; it < n_kt; ++it) {
       const int s = it % p.stages;
-      if (it >= p.stages) {
+      if (it >= p.stages && ptid == 0) {     // one thread polls; the rest wait at the barrier below
         const uint32_t parity = ((it / p.stages) - 1) & 1;
-        if (!mbar_wait(empty_bar + 8 * s, parity)) {
+        if (!mbar_wait(empty_bar + 8 * s, parity, 32)) {
           *fail = 1;
           atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
         }

@@ -263,8 +263,8 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
     if (g < n_kt) stage_meta(tile_of(g));
     for (int it = g; it < n_kt; it += kGroups) {
       const int s = it % p.stages;
-      if (it >= p.stages) {
-        if (!mbar_wait(empty_bar + 8 * s, ((it / p.stages) - 1) & 1)) {
+      if (it >= p.stages && gtid == 0) {     // one thread polls; the rest wait at the barrier below
+        if (!mbar_wait(empty_bar + 8 * s, ((it / p.stages) - 1) & 1, 32)) {
           *fail = 1;
           atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
         }

@@ -256,10 +256,11 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
       for (int i = 0; i < 8; ++i) v[i] = ld_packed<DT>(values, rank + i, static_cast<uint32_t>(i) < count);
 
       const int s = it % p.stages;
-      if (it >= p.stages && !mbar_wait(empty_bar + 8 * s, ((it / p.stages) - 1) & 1, 32)) {
-        fail = 1;
+      if (it >= p.stages && lane == 0 && !mbar_wait(empty_bar + 8 * s, ((it / p.stages) - 1) & 1, 32)) {
+        fail = 1;                                  // one lane polls; the warp follows
         atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
       }
+      __syncwarp();
       if (fail) break;
       unsigned char* dst_row = smem + s * stage_bytes + rowbase;
 #pragma unroll
