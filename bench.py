@@ -253,6 +253,12 @@ def run_ours(args, rank, world, local):
             run_sweep(args, device)
         return
     layers, desc_text = get_layers(args.workload, args.batch)
+    if args.layers:      # profiling aid: keep only the named layers of the stack
+        keep = set(args.layers.split(","))
+        layers = [l for l in layers if l.name in keep]
+        desc_text += " (layers %s only)" % args.layers
+        if len(layers) < 2:
+            raise SystemExit("--layers must name at least two layers of the stack (the ratio rule needs two)")
     path = B.PATH_FP32 if args.path == "fp32" else B.PATH_TENSOR_CORE
     stack = Stack(layers, path, args.seed + rank, device)
     torch.cuda.synchronize()
@@ -459,6 +465,7 @@ def main():
     ap.add_argument("--workload", default="wrn28", choices=["wrn28", "tiny", "resnet50", "vit", "sweep"])
     ap.add_argument("--sweep-sizes", type=int, default=5, help="how many of 2^20,22,24,26,28,30 the sweep covers")
     ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--layers", default=None, help="comma-separated layer names: run only these (profiling)")
     ap.add_argument("--path", default="tc", choices=["tc", "fp32"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=2)

@@ -131,7 +131,7 @@ surgeon_status surgeon_prune_compact(const void* x, int64_t n, surgeon_dtype dt,
  * plug-in behind an interface that forbids cudaMalloc, or a process that gave away its whole
  * memory budget at start-up still owns x and the four output buffers of *out, but has no scratch
  * to pass as `workspace`.  This variant takes none: the scratch is a fixed array inside the
- * library (about 2.5 MB of global data on every GPU that loads the library, held until the
+ * library (about 1.3 MB of global data on every GPU that loads the library, held until the
  * process exits), so neither the caller nor the library allocates or frees anything.
  * Same arguments, results, ordering on cuda_stream and error codes as surgeon_prune_compact,
  * except:

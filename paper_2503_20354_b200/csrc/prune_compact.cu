@@ -205,8 +205,8 @@ sample_kernel(const uint4* __restrict__ xq, long long n, uint32_t k, uint32_t n_
     const uint32_t lo = (DT == 0) ? (blo << 16) : blo;
     st->lo_key = lo < 1u ? 1u : lo;
     const uint32_t hi = (DT == 0) ? ((bhi << 16) | 0xFFFFu) : bhi;
-    st->hi_key = hi;
-    const int range_bits = 32 - __clz(hi - st->lo_key);       // bits of the widest relative key
+    st->hi_key = hi;                                            // hi < lo_key: the bracket is {0}
+    const int range_bits = hi >= st->lo_key ? 32 - __clz(hi - st->lo_key) : 0;   // widest relative key
     st->shiftA = range_bits > 9 ? static_cast<uint32_t>(range_bits - 9) : 0u;
   }
 }
@@ -288,7 +288,9 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
   const uint32_t lane = lane_id();
   if (st->mode == 1u) return;          // the sample found no usable bracket
   const uint32_t lo_key = st->lo_key, hi_key = st->hi_key;
-  const uint32_t range = hi_key - lo_key;
+  // keys inside the bracket: key - cand_lo <= range (nothing when the bracket holds only key 0)
+  const uint32_t cand_lo = hi_key >= lo_key ? lo_key : 0xFFFFFFFFu;
+  const uint32_t range = hi_key >= lo_key ? hi_key - lo_key : 0u;
   const uint32_t shiftA = st->shiftA;
   const uint32_t full_bar = smem_u32(bars);
   const uint32_t empty_bar = smem_u32(bars + kCsStages);
@@ -348,14 +350,14 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
             if (DT == 0) {
               const uint32_t key = c[i] & kMask;
               aw[0] |= (key > hi_key ? 1u : 0u) << (4 * j + i);
-              cw[0] |= (key - lo_key <= range ? 1u : 0u) << (4 * j + i);
+              cw[0] |= (key - cand_lo <= range ? 1u : 0u) << (4 * j + i);
             } else {
               const int e = 8 * j + 2 * i;
               const uint32_t k0 = c[i] & kMask, k1 = (c[i] >> 16) & kMask;
               aw[e >> 5] |= (k0 > hi_key ? 1u : 0u) << (e & 31);
               aw[e >> 5] |= (k1 > hi_key ? 1u : 0u) << ((e + 1) & 31);
-              cw[e >> 5] |= (k0 - lo_key <= range ? 1u : 0u) << (e & 31);
-              cw[e >> 5] |= (k1 - lo_key <= range ? 1u : 0u) << ((e + 1) & 31);
+              cw[e >> 5] |= (k0 - cand_lo <= range ? 1u : 0u) << (e & 31);
+              cw[e >> 5] |= (k1 - cand_lo <= range ? 1u : 0u) << ((e + 1) & 31);
             }
           }
         }

@@ -6,7 +6,7 @@
 // (for instance while a stream is being captured), a plug-in behind a host API that forbids
 // cudaMalloc, or a process whose memory budget was handed out in full at start-up.  Such a
 // caller already owns the input and the output buffers of the store, but the select and the
-// compaction also need a couple of megabytes of scratch.  This entry point keeps that
+// compaction also need a bit over a megabyte of scratch.  This entry point keeps that
 // scratch inside the library image, so nothing is allocated by anybody.
 #include <mutex>
 
