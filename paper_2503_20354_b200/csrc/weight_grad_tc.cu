@@ -74,19 +74,30 @@ __device__ __forceinline__ void decompress_range(const uint32_t* __restrict__ bi
   const long long blk_word0 = blk * kBlockWords;
   uint32_t w = 0;
   if (blk_word0 + lane < first_word) w = __ldg(bitmap + blk_word0 + lane);
-  long long rank = static_cast<long long>(__ldg(offsets + blk)) + warp_sum(__popc(w));
-  for (long long wi = first_word; wi <= last_word; ++wi) {
-    const uint32_t word = __ldg(bitmap + wi);
-    const long long j = (wi << 5) + lane;
-    const bool in_range = (j >= start) && (j < start + len);
-    unsigned short v = 0;
-    if (in_range && ((word >> lane) & 1u)) {
-      const long long r = rank + __popc(word & lt);
-      if (DT == 0) v = to_bf16_bits(__ldg(reinterpret_cast<const float*>(values) + r));
-      else v = __ldg(reinterpret_cast<const unsigned short*>(values) + r);
+  uint32_t rank0 = __ldg(offsets + blk) + warp_sum(__popc(w));    // kept before first_word
+  // 32 bitmap words per round: every lane fetches one word, a warp scan ranks them, and the
+  // value loads of the round do not depend on one another
+  for (long long w0 = first_word; w0 <= last_word; w0 += 32) {
+    const long long mine = w0 + lane;
+    const uint32_t my_word = (mine <= last_word) ? __ldg(bitmap + mine) : 0u;
+    const uint32_t my_cnt = __popc(my_word);
+    const uint32_t my_excl = warp_excl_scan(my_cnt);
+    const int n_here = static_cast<int>(last_word - w0 < 31 ? last_word - w0 + 1 : 32);
+#pragma unroll 4
+    for (int i = 0; i < n_here; ++i) {
+      const uint32_t word = __shfl_sync(0xFFFFFFFFu, my_word, i);
+      const uint32_t before = __shfl_sync(0xFFFFFFFFu, my_excl, i);
+      const long long j = ((w0 + i) << 5) + lane;
+      const bool in_range = (j >= start) && (j < start + len);
+      unsigned short v = 0;
+      if (in_range && ((word >> lane) & 1u)) {
+        const uint32_t r = rank0 + before + __popc(word & lt);
+        if (DT == 0) v = to_bf16_bits(__ldg(reinterpret_cast<const float*>(values) + r));
+        else v = __ldg(reinterpret_cast<const unsigned short*>(values) + r);
+      }
+      if (in_range) dst[j - start] = v;
     }
-    if (in_range) dst[j - start] = v;
-    rank += __popc(word);
+    rank0 += __shfl_sync(0xFFFFFFFFu, my_excl + my_cnt, 31);
   }
 }
 

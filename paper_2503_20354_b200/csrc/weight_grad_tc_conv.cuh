@@ -38,7 +38,9 @@ cudaError_t launch_grad_to_bf16_rows(const float* g, long long rows, int len, in
 
 // ---- layers whose im2col operand is the activation itself (weight_grad_tc_direct.cu) ----------
 struct DirectParams {
-  int mode;                 // 0 = linear [T, C] (MN-major operands), 1 = conv 1x1 stride 1 (K-major)
+  int mode;                 // 0 = linear [T, C] (MN-major operands), 1 = conv 1x1 stride 1 (K-major),
+                            // 2 = conv 1x1 stride 2 (K-major, sampled input)
+  int ow, in_w, in_hw;      // mode 2: output row length, input row length, input plane size
   int C, O;                 // input / output channels
   int T;                    // linear: rows; conv: positions per image
   int pitch;                // elements per row of the bf16 gradient copy

@@ -1,5 +1,5 @@
 // Tensor-core weight gradient for layers whose im2col operand is the activation itself: linear
-// layers ([T, C] activations) and 1x1 / stride 1 / pad 0 convolutions (NCHW).  Algorithm 1,
+// layers ([T, C] activations) and 1x1 / pad 0 convolutions of stride 1 or 2 (NCHW).  Algorithm 1,
 // Reshape and gradient steps with Eq. 2:  D[c, o] = sum_k A[k, c] * G[k, o].
 //
 //   c (input channel)  -> MMA M, 128 per CTA (TMEM lanes)
@@ -195,6 +195,72 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
     const uint32_t xr = row & 7;
     const uint32_t y = (MODE == 0) ? (part & 1) * 4 : part * 4;     // first 16-byte chunk of the run
     const uint32_t rowbase = (MODE == 0) ? (part >> 1) * (kTileK * 128) + row * 128 : row * 128;
+    if (MODE == 2) {
+      // 1x1 stride-2 conv: the run's 32 output positions sample every other element of every
+      // other input row.  Per output-row segment: 64 bitmap bits from the segment's first input
+      // element, the even ones are the segment's bits; a kept element's place in the packed
+      // vector counts the odd (skipped) bits before it as well.
+      for (int it = wg; it < n_kt; it += 2) {
+        const int kt = kt_begin + it;
+        const int img = kt / p.tiles_per_img;
+        const int q0 = (kt - img * p.tiles_per_img) * kTileK + 32 * part;     // first output position
+        const int c = c0 + row;
+        int left = (c < p.C) ? min(32, p.T - q0) : 0;
+        const int s = it % p.stages;
+        if (it >= p.stages && lane == 0 && !mbar_wait(empty_bar + 8 * s, ((it / p.stages) - 1) & 1, 32)) {
+          fail = 1;
+          atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+        }
+        __syncwarp();
+        if (fail) break;
+        unsigned char* dst_row = smem + s * stage_bytes + rowbase;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          *reinterpret_cast<uint4*>(dst_row + (((y + q) ^ xr) << 4)) = make_uint4(0, 0, 0, 0);
+        const long long plane = (static_cast<long long>(img) * p.C + c) * p.in_hw;
+        int oy = q0 / p.ow, ox = q0 - oy * p.ow;
+        int b0 = 0;                                    // position of the segment inside the run
+        while (left > 0) {
+          const int seg = min(left, p.ow - ox);
+          const long long j = plane + static_cast<long long>(2 * oy) * p.in_w + 2 * ox;
+          const long long blk = j >> kBlockShift;
+          const long long wi = j >> 5;
+          uint32_t rank = __ldg(offsets + blk);
+          for (long long w = blk * kBlockWords; w < wi; ++w) rank += __popc(__ldg(bitmap + w));
+          const uint32_t w0 = __ldg(bitmap + wi);
+          const uint32_t w1 = (wi + 1 < p.n_words) ? __ldg(bitmap + wi + 1) : 0u;
+          const uint32_t w2 = (wi + 2 < p.n_words) ? __ldg(bitmap + wi + 2) : 0u;
+          const uint32_t sh = static_cast<uint32_t>(j & 31);
+          rank += __popc(w0 & ((1u << sh) - 1u));
+          unsigned long long win = (static_cast<unsigned long long>(__funnelshift_r(w1, w2, sh)) << 32) |
+                                   __funnelshift_r(w0, w1, sh);
+          // even bits of the window -> the segment's bits
+          unsigned long long e = win & 0x5555555555555555ull;
+          e = (e | (e >> 1)) & 0x3333333333333333ull;
+          e = (e | (e >> 2)) & 0x0F0F0F0F0F0F0F0Full;
+          e = (e | (e >> 4)) & 0x00FF00FF00FF00FFull;
+          e = (e | (e >> 8)) & 0x0000FFFF0000FFFFull;
+          e = (e | (e >> 16)) & 0x00000000FFFFFFFFull;
+          uint32_t ev = static_cast<uint32_t>(e);
+          ev = seg >= 32 ? ev : (ev & ((1u << seg) - 1u));
+          while (ev) {
+            const int i = __ffs(ev) - 1;
+            ev &= ev - 1;
+            const uint32_t idx = rank + __popcll(win & ((1ull << (2 * i)) - 1ull));
+            uint32_t v;
+            if (DT == 0) v = to_bf16_bits(__ldg(reinterpret_cast<const float*>(values) + idx));
+            else v = __ldg(reinterpret_cast<const unsigned short*>(values) + idx);
+            const int b = b0 + i;
+            *reinterpret_cast<unsigned short*>(dst_row + (((y + (b >> 3)) ^ xr) << 4) + ((b & 7) << 1)) =
+                static_cast<unsigned short>(v);
+          }
+          b0 += seg; left -= seg; ox = 0; ++oy;
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full_bar + 8 * s);
+      }
+    } else {
     auto fetch = [&](int it) {
       WordRaw r;
       r.base = 0; r.next = 0; r.words = make_uint4(0, 0, 0, 0); r.j = 0; r.nvalid = 0;
@@ -288,6 +354,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
       if (lane == 0) mbar_arrive(full_bar + 8 * s);
       cur = nxt;
     }
+    }  // MODE != 2
   }
 
   // ================= epilogue: TMEM -> scratch partial tile =================
@@ -336,6 +403,11 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   } else if (d.kind == 1 && d.kh == 1 && d.kw == 1 && d.stride == 1 && d.pad == 0) {
     p.mode = 1;
     p.T = d.h * d.w; p.imgs = d.batch;
+  } else if (d.kind == 1 && d.kh == 1 && d.kw == 1 && d.stride == 2 && d.pad == 0) {
+    p.mode = 2;                                    // output positions; the input is sampled
+    p.ow = (d.w - 1) / 2 + 1;
+    p.T = ((d.h - 1) / 2 + 1) * p.ow; p.imgs = d.batch;
+    p.in_w = d.w; p.in_hw = d.h * d.w;
   } else {
     return false;
   }
@@ -404,7 +476,7 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
   p.n_words = (act.n + 31) / 32;
   p.partial_blk = (act.n % SURGEON_BLOCK) ? static_cast<unsigned>(act.n / SURGEON_BLOCK) : 0xFFFFFFFFu;
   cudaError_t e;
-  if (p.mode == 1 && p.pitch != p.T)     // rows padded to a 16-byte pitch for the tensor map
+  if (p.mode != 0 && p.pitch != p.T)     // rows padded to a 16-byte pitch for the tensor map
     e = launch_grad_to_bf16_rows(grad_out, static_cast<long long>(p.imgs) * p.O, p.T, p.pitch,
                                  grad_bf16, stream);
   else
@@ -444,6 +516,7 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
     return cudaGetLastError();
   };
   if (p.mode == 0) e = act.dt == 0 ? launch(dw_direct_kernel<0, 0>) : launch(dw_direct_kernel<1, 0>);
+  else if (p.mode == 2) e = act.dt == 0 ? launch(dw_direct_kernel<0, 2>) : launch(dw_direct_kernel<1, 2>);
   else e = act.dt == 0 ? launch(dw_direct_kernel<0, 1>) : launch(dw_direct_kernel<1, 1>);
   note_launches(1);
   return e;

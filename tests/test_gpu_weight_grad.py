@@ -79,6 +79,12 @@ SHAPES = [
     W.linear("lin_c40_o520", 200, 40, 520, dist="gelu_normal", dt=W.F32),
     W.conv("d1x1_hw14", 3, 136, 14, 264, 1, 1, 0),
     W.conv("d1x1_hw7", 5, 72, 7, 48, 1, 1, 0),
+    # 1x1 stride 2 (the residual downsample shortcut): even and odd map sizes, output rows
+    # shorter and longer than one 32-position run, channels past one tile
+    W.conv("d1x1s2_hw56", 2, 72, 56, 136, 1, 2, 0),
+    W.conv("d1x1s2_hw28", 3, 264, 28, 520, 1, 2, 0),
+    W.conv("d1x1s2_hw15", 3, 40, 15, 48, 1, 2, 0),
+    W.conv("d1x1s2_hw70", 1, 16, 70, 32, 1, 2, 0),
 ]
 
 
