@@ -52,6 +52,8 @@ struct TcParams {
   int max_rows;     // input rows one K-tile can touch (conv)
   int dt;           // activation dtype
   int g_vec_ok;     // gradient rows can be read with 16-byte loads
+  int ch_pitch;     // elements between the channels of the patch (conv), a multiple of 32
+  long long n_words;  // words of the bitmap (filled by the launcher)
 };
 
 __device__ __forceinline__ void producer_sync() {
@@ -98,6 +100,39 @@ __device__ __forceinline__ void decompress_range(const uint32_t* __restrict__ bi
       if (in_range) dst[j - start] = v;
     }
     rank0 += __shfl_sync(0xFFFFFFFFu, my_excl + my_cnt, 31);
+  }
+}
+
+// One thread rebuilds up to 32 consecutive elements: dst[0..31] (64 bytes, 16-byte aligned) =
+// bf16 of the pruned activation at flat indices start .. start + len - 1, zeros after them.
+// The work after the fixed part is one load and one store per kept element.
+template <int DT>
+__device__ __forceinline__ void decompress_run(const uint32_t* __restrict__ bitmap,
+                                               const void* __restrict__ values,
+                                               const uint32_t* __restrict__ offsets,
+                                               long long n_words, long long start, int len,
+                                               unsigned short* __restrict__ dst) {
+  uint4* d4 = reinterpret_cast<uint4*>(dst);
+  d4[0] = make_uint4(0, 0, 0, 0); d4[1] = make_uint4(0, 0, 0, 0);
+  d4[2] = make_uint4(0, 0, 0, 0); d4[3] = make_uint4(0, 0, 0, 0);
+  const long long blk = start >> kBlockShift;
+  const long long wi = start >> 5;
+  uint32_t rank = __ldg(offsets + blk);
+  for (long long w = blk * kBlockWords; w < wi; ++w) rank += __popc(__ldg(bitmap + w));
+  const uint32_t w0 = __ldg(bitmap + wi);
+  const uint32_t w1 = (wi + 1 < n_words) ? __ldg(bitmap + wi + 1) : 0u;
+  const uint32_t sh = static_cast<uint32_t>(start & 31);
+  rank += __popc(w0 & ((1u << sh) - 1u));
+  uint32_t bits = __funnelshift_r(w0, w1, sh);
+  if (len < 32) bits &= (1u << len) - 1u;
+  while (bits) {
+    const int i = __ffs(bits) - 1;
+    bits &= bits - 1;
+    unsigned short v;
+    if (DT == 0) v = static_cast<unsigned short>(to_bf16_bits(__ldg(reinterpret_cast<const float*>(values) + rank)));
+    else v = __ldg(reinterpret_cast<const unsigned short*>(values) + rank);
+    ++rank;
+    dst[i] = v;
   }
 }
 
@@ -274,11 +309,15 @@ dw_tc_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ value
         const int range_len = (iy_hi - iy_lo + 1) * p.W;
         for (int cg = first_c; cg <= last_c; cg += p.group_ch) {
           const int cg_end = min(cg + p.group_ch, last_c + 1);
-          for (int c = cg + pwarp; c < cg_end; c += kProducerWarps) {
+          // one task = 32 consecutive elements of one channel's rows
+          const int runs = (range_len + 31) >> 5;
+          const int n_tasks = (cg_end - cg) * runs;
+          for (int t = ptid; t < n_tasks; t += kProducerThreads) {
+            const int ci = t / runs, run = t - ci * runs;
             const long long start =
-                ((static_cast<long long>(img) * p.C + c) * p.H + iy_lo) * p.W;
-            decompress_range<DT>(bitmap, values, offsets, start, range_len,
-                                 patch + (c - cg) * range_len);
+                ((static_cast<long long>(img) * p.C + cg + ci) * p.H + iy_lo) * p.W + 32 * run;
+            decompress_run<DT>(bitmap, values, offsets, p.n_words, start,
+                               min(32, range_len - 32 * run), patch + ci * p.ch_pitch + 32 * run);
           }
           producer_sync();
           // rows of this channel group: nn in [cg*RS, cg_end*RS)
@@ -295,7 +334,7 @@ dw_tc_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ value
 #pragma unroll
               for (int e = 0; e < 8; ++e) h[e] = 0;
             } else {
-              const unsigned short* src = patch + (ri.c - cg) * range_len;
+              const unsigned short* src = patch + (ri.c - cg) * p.ch_pitch;
               int pp = p0 + chunk * 8;
               int y = pp / p.OW;
               int x = pp - y * p.OW;
@@ -431,8 +470,9 @@ bool plan(const surgeon_layer_desc& d, int dt, TcParams* out) {
     int in_rows = (out_rows - 1) * p.stride + p.KH;
     if (in_rows > p.H) in_rows = p.H;
     p.max_rows = in_rows;
-    const long long per_ch = static_cast<long long>(in_rows) * p.W;
+    const long long per_ch = (static_cast<long long>(in_rows) * p.W + 31) / 32 * 32;
     if (per_ch > kPatchElems) return false;
+    p.ch_pitch = static_cast<int>(per_ch);
     p.group_ch = static_cast<int>(kPatchElems / per_ch);
   } else {
     p.max_rows = 1;
@@ -509,6 +549,7 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
   }
   TcParams p;
   if (!plan(d, act.dt, &p)) return cudaErrorNotSupported;
+  p.n_words = (act.n + 31) / 32;
   const size_t smem = smem_bytes(p);
   const uint32_t* offs = act.block_offsets;
   dim3 grid(p.m_tiles, p.n_tiles, p.splits);
