@@ -153,5 +153,38 @@ __device__ __forceinline__ unsigned short to_bf16_bits(float v) {
 }
 
 
+// The MMAs of one K-tile of 64: four K-steps into each of N_ACC accumulators of `acc_n` columns.
+// `da` / `db` are the descriptors of the stage's operands; a K-step advances the start-address
+// field by KSTEP (16-byte units: 2 for K-major rows, 128 for MN-major slabs), an accumulator's B
+// rows lie `acc_inc` units further.  The issuing thread's own instructions are the bound of
+// the tensor pipe when they are many (each MMA of 128 columns lasts only 64 clocks), so
+// nothing here is computed per MMA beyond two additions.
+template <int N_ACC, int KSTEP>
+__device__ __forceinline__ void umma_ktile(uint32_t tmem_base, uint32_t acc_n, uint64_t da, uint64_t db,
+                                           uint64_t acc_inc, uint32_t idesc, uint32_t accum) {
+#pragma unroll
+  for (int a = 0; a < N_ACC; ++a) {
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk)
+      umma_bf16(tmem_base + a * acc_n, da + static_cast<uint64_t>(kk * KSTEP),
+                db + a * acc_inc + static_cast<uint64_t>(kk * KSTEP), idesc, kk > 0 ? 1u : accum);
+  }
+}
+
+// Predicated load of packed value `idx` (zero when !on); no branch.
+template <int DT>
+__device__ __forceinline__ uint32_t ld_packed(const void* __restrict__ values, uint32_t idx, bool on) {
+  uint32_t r = 0;
+  const unsigned char* src =
+      reinterpret_cast<const unsigned char*>(values) + static_cast<size_t>(idx) * (DT == 0 ? 4 : 2);
+  if (DT == 0)
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q ld.global.nc.u32 %0, [%1];\n\t}"
+                 : "+r"(r) : "l"(src), "r"(static_cast<uint32_t>(on)));
+  else
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q ld.global.nc.u16 %0, [%1];\n\t}"
+                 : "+r"(r) : "l"(src), "r"(static_cast<uint32_t>(on)));
+  return r;
+}
+
 }  // namespace tc
 }  // namespace surgeon

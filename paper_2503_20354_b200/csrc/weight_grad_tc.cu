@@ -125,14 +125,19 @@ __device__ __forceinline__ void decompress_run(const uint32_t* __restrict__ bitm
   rank += __popc(w0 & ((1u << sh) - 1u));
   uint32_t bits = __funnelshift_r(w0, w1, sh);
   if (len < 32) bits &= (1u << len) - 1u;
-  while (bits) {
-    const int i = __ffs(bits) - 1;
-    bits &= bits - 1;
-    unsigned short v;
-    if (DT == 0) v = static_cast<unsigned short>(to_bf16_bits(__ldg(reinterpret_cast<const float*>(values) + rank)));
-    else v = __ldg(reinterpret_cast<const unsigned short*>(values) + rank);
-    ++rank;
-    dst[i] = v;
+  const uint32_t count = __popc(bits);
+  for (uint32_t g = 0; g < count; g += 8) {      // eight independent loads in flight per round
+    uint32_t v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = ld_packed<DT>(values, rank + g + i, g + i < count);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (g + i < count) {
+        const int b = __ffs(bits) - 1;
+        bits &= bits - 1;
+        dst[b] = (DT == 0) ? to_bf16_bits(__uint_as_float(v[i])) : static_cast<unsigned short>(v[i]);
+      }
+    }
   }
 }
 
@@ -206,21 +211,23 @@ dw_tc_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ value
     // ================= MMA issuer =================
     if (lane == 0) {
       const uint32_t idesc = make_idesc(kTileM, p.tile_n);
+      const uint32_t smem0 = smem_u32(smem);
+      const uint64_t a_base = make_desc(smem0);
+      const uint64_t b_base = make_desc(smem0 + kTileM * 128);
+      const uint64_t stage_inc = static_cast<uint64_t>(stage_bytes >> 4);
+      uint64_t da = a_base, db = b_base;
+      uint32_t parity = 0, accum = 0;
+      int s = 0;
       bool ok = true;
-      for (int it = 0; it < n_kt && ok; ++it) {
-        const int s = it % p.stages;
-        const uint32_t parity = (it / p.stages) & 1;
+      for (int it = 0; it < n_kt; ++it) {
         ok = mbar_wait(full_bar + 8 * s, parity);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
-        const uint32_t b_addr = a_addr + kTileM * 128;
-#pragma unroll
-        for (int kk = 0; kk < kTileK / 16; ++kk) {
-          umma_bf16(tmem_base, make_desc(a_addr + kk * 32), make_desc(b_addr + kk * 32), idesc,
-                    (it > 0 || kk > 0) ? 1u : 0u);
-        }
+        umma_ktile<1, 2>(tmem_base, p.tile_n, da, db, 0, idesc, accum);
         umma_commit(empty_bar + 8 * s);   // stage is free once these MMAs have read it
+        accum = 1;
+        if (++s == p.stages) { s = 0; parity ^= 1; da = a_base; db = b_base; }
+        else { da += stage_inc; db += stage_inc; }
       }
       if (!ok) { *fail = 1; atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); }
       umma_commit(acc_bar);               // accumulator complete (or abandoned)
@@ -434,6 +441,25 @@ reduce_splits_kernel(const float* __restrict__ partial, long long mn, int splits
   dw[i] = accumulate ? dw[i] + s : s;
 }
 
+// The same for a tap-stacked partial [splits][taps * O][C]: dw[o][c][tap] gets row tap * O + o.
+__global__ void __launch_bounds__(256)
+reduce_splits_taps_kernel(const float* __restrict__ partial, int o_real, int c_in, int taps,
+                          int splits, float* __restrict__ dw, int accumulate,
+                          const uint32_t* __restrict__ status, surgeon_header* __restrict__ hdr) {
+  const long long mn = static_cast<long long>(o_real) * c_in * taps;
+  const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i == 0 && *status != 0 && hdr) atomicMax(&hdr->status, *status);
+  if (i >= mn) return;
+  const long long oc = i / taps;
+  const int tap = static_cast<int>(i - oc * taps);
+  const long long o = oc / c_in;
+  const long long c = oc - o * c_in;
+  const long long src = (static_cast<long long>(tap) * o_real + o) * c_in + c;
+  float s = partial[src];
+  for (int z = 1; z < splits; ++z) s += partial[z * mn + src];
+  dw[i] = accumulate ? dw[i] + s : s;
+}
+
 bool plan(const surgeon_layer_desc& d, int dt, TcParams* out) {
   TcParams p{};
   p.kind = d.kind; p.B = d.batch; p.C = d.c_in; p.H = d.h; p.W = d.w; p.O = d.c_out;
@@ -531,8 +557,12 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
     e = launch_direct(act, dp, grad_out, grad_bf16, partial, status, stream);
     if (e != cudaSuccess) return e;
     const long long mn = static_cast<long long>(dp.O) * dp.C;
-    reduce_splits_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
-        partial, mn, dp.splits, dw, accumulate, status, act.header);
+    if (dp.taps > 1)
+      reduce_splits_taps_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
+          partial, dp.o_real, dp.C, dp.taps, dp.splits, dw, accumulate, status, act.header);
+    else
+      reduce_splits_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
+          partial, mn, dp.splits, dw, accumulate, status, act.header);
     note_launches(1);
     return cudaGetLastError();
   }

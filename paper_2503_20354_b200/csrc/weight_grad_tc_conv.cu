@@ -138,22 +138,25 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
     // ================= MMA issuer =================
     if (lane == 0) {
       const uint32_t idesc = make_idesc(kTileM, p.acc_n);
+      const uint32_t smem0 = smem_u32(smem);
+      const uint64_t a_base = make_desc(smem0);
+      const uint64_t b_base = make_desc(smem0 + kTileM * 128);
+      const uint64_t stage_inc = static_cast<uint64_t>(stage_bytes >> 4);
+      const uint64_t acc_inc = static_cast<uint64_t>((p.acc_n * 128) >> 4);
+      uint64_t da = a_base, db = b_base;
+      uint32_t parity = 0, accum = 0;
+      int s = 0;
       bool ok = true;
       for (int it = 0; it < n_kt; ++it) {
-        const int s = it % p.stages;
-        ok = mbar_wait(full_bar + 8 * s, (it / p.stages) & 1);
+        ok = mbar_wait(full_bar + 8 * s, parity);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
-        const uint32_t b_addr = a_addr + kTileM * 128;
-#pragma unroll
-        for (int kk = 0; kk < kTileK / 16; ++kk) {
-          const uint64_t da = make_desc(a_addr + kk * 32);
-          for (int a = 0; a < p.n_acc; ++a)
-            umma_bf16(tmem_base + a * p.acc_n, da, make_desc(b_addr + a * p.acc_n * 128 + kk * 32),
-                      idesc, (it > 0 || kk > 0) ? 1u : 0u);
-        }
+        if (p.n_acc == 1) umma_ktile<1, 2>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
+        else umma_ktile<2, 2>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
         umma_commit(empty_bar + 8 * s);
+        accum = 1;
+        if (++s == p.stages) { s = 0; parity ^= 1; da = a_base; db = b_base; }
+        else { da += stage_inc; db += stage_inc; }
       }
       if (!ok) { *fail = 1; atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); }
       umma_commit(acc_bar);

@@ -41,7 +41,10 @@ struct DirectParams {
   int mode;                 // 0 = linear [T, C] (MN-major operands), 1 = conv 1x1 stride 1 (K-major),
                             // 2 = conv 1x1 stride 2 (K-major, sampled input)
   int ow, in_w, in_hw;      // mode 2: output row length, input row length, input plane size
-  int C, O;                 // input / output channels
+  int taps;                 // 1, or kh*kw for a k x k stride-1 conv (mode 1 over shifted gradients)
+  int kh, kw, pad, in_h, oh;  // taps > 1: kernel and map sizes (with ow, in_w)
+  int o_real;               // output channels of the layer; O = taps * o_real
+  int C, O;                 // input channels / gradient channels (taps * output channels)
   int T;                    // linear: rows; conv: positions per image
   int pitch;                // elements per row of the bf16 gradient copy
   int imgs;                 // conv: batch; linear: 1
@@ -54,7 +57,7 @@ struct DirectParams {
 };
 bool plan_direct(const surgeon_layer_desc& d, DirectParams* out);
 size_t direct_grad_bf16_bytes(const DirectParams& p);
-// partial = [splits][O][C] fp32, status = one zeroed word.
+// partial = [splits][O][C] fp32 (O counts the stacked taps), status = one zeroed word.
 cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& p,
                           const float* grad_out, void* grad_bf16, float* partial,
                           uint32_t* status, cudaStream_t stream);

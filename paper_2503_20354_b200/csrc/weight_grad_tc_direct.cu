@@ -1,5 +1,6 @@
 // Tensor-core weight gradient for layers whose im2col operand is the activation itself: linear
-// layers ([T, C] activations) and 1x1 / pad 0 convolutions of stride 1 or 2 (NCHW).  Algorithm 1,
+// layers ([T, C] activations), 1x1 / pad 0 convolutions of stride 1 or 2, and k x k stride-1
+// convolutions through shifted copies of the output gradient (NCHW).  Algorithm 1,
 // Reshape and gradient steps with Eq. 2:  D[c, o] = sum_k A[k, c] * G[k, o].
 //
 //   c (input channel)  -> MMA M, 128 per CTA (TMEM lanes)
@@ -63,21 +64,6 @@ struct WordRaw {
   uint32_t nvalid;     // elements of the run that exist (0: nothing to do)
 };
 
-// Predicated load of packed value `idx` (zero when !on); no branch.
-template <int DT>
-__device__ __forceinline__ uint32_t ld_packed(const void* __restrict__ values, uint32_t idx, bool on) {
-  uint32_t r = 0;
-  const unsigned char* src =
-      reinterpret_cast<const unsigned char*>(values) + static_cast<size_t>(idx) * (DT == 0 ? 4 : 2);
-  if (DT == 0)
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q ld.global.nc.u32 %0, [%1];\n\t}"
-                 : "+r"(r) : "l"(src), "r"(static_cast<uint32_t>(on)));
-  else
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q ld.global.nc.u16 %0, [%1];\n\t}"
-                 : "+r"(r) : "l"(src), "r"(static_cast<uint32_t>(on)));
-  return r;
-}
-
 template <int DT, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ values,
@@ -124,31 +110,26 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
     // ================= MMA issuer =================
     if (lane == 0) {
       const uint32_t idesc = make_idesc(kTileM, p.acc_n) | (MODE == 0 ? ((1u << 15) | (1u << 16)) : 0u);
+      const uint32_t smem0 = smem_u32(smem);
+      const uint64_t a_base = (MODE == 0) ? make_desc_mn(smem0) : make_desc(smem0);
+      const uint64_t b_base = (MODE == 0) ? make_desc_mn(smem0 + kATileBytes) : make_desc(smem0 + kATileBytes);
+      const uint64_t stage_inc = static_cast<uint64_t>(stage_bytes >> 4);
+      const uint64_t acc_inc = static_cast<uint64_t>((p.acc_n * 128) >> 4);
+      constexpr int kStep = (MODE == 0) ? 128 : 2;
+      uint64_t da = a_base, db = b_base;
+      uint32_t parity = 0, accum = 0;
+      int s = 0;
       bool ok = true;
       for (int it = 0; it < n_kt; ++it) {
-        const int s = it % p.stages;
-        ok = mbar_wait(full_bar + 8 * s, (it / p.stages) & 1);
+        ok = mbar_wait(full_bar + 8 * s, parity);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
-        const uint32_t b_addr = a_addr + kATileBytes;
-#pragma unroll
-        for (int kk = 0; kk < kTileK / 16; ++kk) {
-          if (MODE == 0) {
-            const uint64_t da = make_desc_mn(a_addr + kk * 2048);
-            for (int a = 0; a < p.n_acc; ++a)
-              umma_bf16(tmem_base + a * p.acc_n, da,
-                        make_desc_mn(b_addr + a * p.acc_n * 128 + kk * 2048), idesc,
-                        (it > 0 || kk > 0) ? 1u : 0u);
-          } else {
-            const uint64_t da = make_desc(a_addr + kk * 32);
-            for (int a = 0; a < p.n_acc; ++a)
-              umma_bf16(tmem_base + a * p.acc_n, da,
-                        make_desc(b_addr + a * p.acc_n * 128 + kk * 32), idesc,
-                        (it > 0 || kk > 0) ? 1u : 0u);
-          }
-        }
+        if (p.n_acc == 1) umma_ktile<1, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
+        else umma_ktile<2, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
         umma_commit(empty_bar + 8 * s);
+        accum = 1;
+        if (++s == p.stages) { s = 0; parity ^= 1; da = a_base; db = b_base; }
+        else { da += stage_inc; db += stage_inc; }
       }
       if (!ok) { fail = 1; atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); }
       umma_commit(acc_bar);
@@ -243,16 +224,28 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
           e = (e | (e >> 16)) & 0x00000000FFFFFFFFull;
           uint32_t ev = static_cast<uint32_t>(e);
           ev = seg >= 32 ? ev : (ev & ((1u << seg) - 1u));
+          // packed places of the kept samples are not contiguous (skipped odd elements lie
+          // between them): eight loads in flight per round
           while (ev) {
-            const int i = __ffs(ev) - 1;
-            ev &= ev - 1;
-            const uint32_t idx = rank + __popcll(win & ((1ull << (2 * i)) - 1ull));
-            uint32_t v;
-            if (DT == 0) v = to_bf16_bits(__ldg(reinterpret_cast<const float*>(values) + idx));
-            else v = __ldg(reinterpret_cast<const unsigned short*>(values) + idx);
-            const int b = b0 + i;
-            *reinterpret_cast<unsigned short*>(dst_row + (((y + (b >> 3)) ^ xr) << 4) + ((b & 7) << 1)) =
-                static_cast<unsigned short>(v);
+            uint32_t idx[8], vv[8];
+            uint32_t e2 = ev;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int i = e2 ? __ffs(e2) - 1 : 0;
+              idx[u] = rank + __popcll(win & ((1ull << (2 * i)) - 1ull));
+              vv[u] = ld_packed<DT>(values, idx[u], e2 != 0);
+              e2 &= e2 - 1;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              if (ev) {
+                const int b = b0 + __ffs(ev) - 1;
+                ev &= ev - 1;
+                const unsigned short h = (DT == 0) ? to_bf16_bits(__uint_as_float(vv[u]))
+                                                   : static_cast<unsigned short>(vv[u]);
+                *reinterpret_cast<unsigned short*>(dst_row + (((y + (b >> 3)) ^ xr) << 4) + ((b & 7) << 1)) = h;
+              }
+            }
           }
           b0 += seg; left -= seg; ox = 0; ++oy;
         }
@@ -387,6 +380,39 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
 }
 
+// Shifted bf16 copies of the output gradient of a k x k stride-1 convolution (Eq. 2 summed over
+// input positions): out[img][tap * O + o][y' * W + x'] = g[img][o][y' + pad - r][x' + pad - s],
+// zero where that lies outside the output map; tap = r * kw + s.  One thread writes 8 positions.
+__global__ void __launch_bounds__(256)
+grad_taps_bf16_kernel(const float* __restrict__ g, unsigned short* __restrict__ out,
+                      long long chunks, DirectParams p) {
+  const int per_row = p.pitch >> 3;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < chunks;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const long long rowi = i / per_row;              // img * taps * O + tap * O + o
+    const int chunk = static_cast<int>(i - rowi * per_row);
+    const int v = static_cast<int>(rowi % p.O);
+    const long long img = rowi / p.O;
+    const int tap = v / p.o_real, o = v - tap * p.o_real;
+    const int r = tap / p.kw, sft = tap - r * p.kw;
+    const float* src = g + (img * p.o_real + o) * static_cast<long long>(p.oh) * p.ow;
+    int pos = chunk * 8;
+    int yy = pos / p.in_w, xx = pos - yy * p.in_w;   // input position
+    float f[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int y = yy + p.pad - r, x = xx + p.pad - sft;
+      f[e] = (pos < p.T && y >= 0 && y < p.oh && x >= 0 && x < p.ow) ? __ldg(src + y * p.ow + x) : 0.0f;
+      ++pos; ++xx;
+      if (xx == p.in_w) { xx = 0; ++yy; }
+    }
+    uint4 w;
+    w.x = pack_bf16x2(f[0], f[1]); w.y = pack_bf16x2(f[2], f[3]);
+    w.z = pack_bf16x2(f[4], f[5]); w.w = pack_bf16x2(f[6], f[7]);
+    *reinterpret_cast<uint4*>(out + rowi * p.pitch + chunk * 8) = w;
+  }
+}
+
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                               CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -408,10 +434,25 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
     p.ow = (d.w - 1) / 2 + 1;
     p.T = ((d.h - 1) / 2 + 1) * p.ow; p.imgs = d.batch;
     p.in_w = d.w; p.in_hw = d.h * d.w;
+  } else if (d.kind == 1 && d.stride == 1 && d.kh * d.kw > 1 && d.kh <= 7 && d.kw <= 7 &&
+             d.pad < d.kh && d.pad < d.kw) {
+    // k x k, stride 1: the sum runs over INPUT positions, and tap (r, s) multiplies the
+    // activation with the output gradient shifted by (pad - r, pad - s).  The shifted copies
+    // (zero outside the map) are stacked as kh*kw*O gradient channels, which makes this the 1x1
+    // problem with that many output channels; the activation operand is never expanded.
+    p.mode = 1;
+    p.taps = d.kh * d.kw;
+    p.kh = d.kh; p.kw = d.kw; p.pad = d.pad; p.in_h = d.h; p.in_w = d.w;
+    p.oh = d.h + 2 * d.pad - d.kh + 1; p.ow = d.w + 2 * d.pad - d.kw + 1;
+    if (p.oh < 1 || p.ow < 1) return false;
+    p.T = d.h * d.w; p.imgs = d.batch;
   } else {
     return false;
   }
-  p.C = d.c_in; p.O = d.c_out;
+  if (p.taps == 0) p.taps = 1;
+  p.o_real = d.c_out;
+  if (static_cast<long long>(p.taps) * d.c_out > 2147483647LL / 256) return false;
+  p.C = d.c_in; p.O = p.taps * d.c_out;
   p.pitch = (p.mode == 0) ? p.O : (p.T + 7) / 8 * 8;   // row pitch of the bf16 gradient copy
   if (p.mode == 0) {
     // columns come in slabs of 64; per CTA two accumulators of 192 or 128 columns, or one small one
@@ -423,12 +464,19 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
       p.acc_n = (t6 <= t4) ? 192 : 128;
     }
   } else {
-    int acc_n = 0;
-    for (int c = 256; c >= 128; c -= 16)
-      if (p.O % c == 0) { acc_n = c; break; }
-    if (acc_n == 0) acc_n = (p.O <= 256) ? (p.O + 15) / 16 * 16 : 256;
-    p.acc_n = acc_n;
-    p.n_acc = (p.O + acc_n - 1) / acc_n >= 2 ? 2 : 1;
+    // one or two accumulators of a multiple of 16 columns: the fewest padded columns overall,
+    // then the widest CTA tile
+    long long best_waste = -1;
+    for (int na = 2; na >= 1; --na)
+      for (int c = 256; c >= 16; c -= 16) {
+        const int cols = c * na;
+        const long long padded = static_cast<long long>((p.O + cols - 1) / cols) * cols;
+        const long long waste = padded - p.O;
+        if (best_waste < 0 || waste < best_waste ||
+            (waste == best_waste && cols > p.acc_n * p.n_acc)) {
+          best_waste = waste; p.acc_n = c; p.n_acc = na;
+        }
+      }
   }
   p.n_cols = p.acc_n * p.n_acc;
   p.n_tiles = (p.O + p.n_cols - 1) / p.n_cols;
@@ -476,7 +524,16 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
   p.n_words = (act.n + 31) / 32;
   p.partial_blk = (act.n % SURGEON_BLOCK) ? static_cast<unsigned>(act.n / SURGEON_BLOCK) : 0xFFFFFFFFu;
   cudaError_t e;
-  if (p.mode != 0 && p.pitch != p.T)     // rows padded to a 16-byte pitch for the tensor map
+  if (p.taps > 1) {
+    const long long chunks = static_cast<long long>(p.imgs) * p.O * (p.pitch >> 3);
+    const long long want = (chunks + 255) / 256;
+    const long long cap = 32LL * sm_count();
+    const int grid = static_cast<int>(want < 1 ? 1 : (want > cap ? cap : want));
+    grad_taps_bf16_kernel<<<grid, 256, 0, stream>>>(grad_out, static_cast<unsigned short*>(grad_bf16),
+                                                    chunks, p);
+    note_launches(1);
+    e = cudaGetLastError();
+  } else if (p.mode != 0 && p.pitch != p.T)     // rows padded to a 16-byte pitch for the tensor map
     e = launch_grad_to_bf16_rows(grad_out, static_cast<long long>(p.imgs) * p.O, p.T, p.pitch,
                                  grad_bf16, stream);
   else

@@ -85,6 +85,11 @@ SHAPES = [
     W.conv("d1x1s2_hw28", 3, 264, 28, 520, 1, 2, 0),
     W.conv("d1x1s2_hw15", 3, 40, 15, 48, 1, 2, 0),
     W.conv("d1x1s2_hw70", 1, 16, 70, 32, 1, 2, 0),
+    # k x k stride 1 through shifted gradient copies: 5x5, a 2x3 kernel with less padding than
+    # "same", channels past one tile on a 14x14 map
+    W.conv("t5x5_hw12", 2, 24, 12, 40, 5, 1, 2),
+    W.Layer("t2x3_pad1", 1, 3, 16, 9, 11, 24, 2, 3, 1, 1),
+    W.conv("t3x3_hw14_c136", 2, 136, 14, 72, 3),
 ]
 
 
