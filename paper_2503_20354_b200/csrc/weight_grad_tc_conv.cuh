@@ -44,6 +44,10 @@ struct DirectParams {
   int taps;                 // 1, or kh*kw for a k x k stride-1 conv (mode 1 over shifted gradients)
   int kh, kw, pad, in_h, oh;  // taps > 1: kernel and map sizes (with ow, in_w)
   int o_real;               // output channels of the layer; O = taps * o_real
+  int row_shift;            // taps > 1: only the kw column shifts are stored; rows shift by TMA offset
+  int copies;               // stacked gradient copies: taps, or kw with row_shift
+  int g_len;                // conv: elements per row of the gradient copy (T, or oh * in_w)
+  int upt, n_units;         // conv: accumulator units per tap (of acc_n columns), units in all
   int C, O;                 // input channels / gradient channels (taps * output channels)
   int T;                    // linear: rows; conv: positions per image
   int pitch;                // elements per row of the bf16 gradient copy

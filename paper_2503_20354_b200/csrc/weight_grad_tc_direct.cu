@@ -82,7 +82,9 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   const uint32_t lane = lane_id();
   const int m_tile = blockIdx.x, n_tile = blockIdx.y, split = blockIdx.z;
   const int c0 = m_tile * kTileM;
-  const int o0 = n_tile * p.n_cols;
+  const int o0 = n_tile * p.n_cols;                  // linear: first gradient column of the CTA
+  const int u0 = n_tile * p.n_acc;                   // conv: first column unit of the CTA
+  const int n_acc_here = (MODE == 0) ? p.n_acc : min(p.n_acc, p.n_units - u0);
   const int kt_begin = split * p.ktiles_per_split;
   const int kt_end = min(kt_begin + p.ktiles_per_split, p.total_ktiles);
   const int n_kt = kt_end - kt_begin;
@@ -124,8 +126,9 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         ok = mbar_wait(full_bar + 8 * s, parity);
         if (!ok) break;
         tc_fence_after();
-        if (p.n_acc == 1) umma_ktile<1, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
-        else umma_ktile<2, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
+        if (n_acc_here == 1) umma_ktile<1, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
+        else if (n_acc_here == 2) umma_ktile<2, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
+        else umma_ktile<3, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
         umma_commit(empty_bar + 8 * s);
         accum = 1;
         if (++s == p.stages) { s = 0; parity ^= 1; da = a_base; db = b_base; }
@@ -147,7 +150,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         }
         const int kt = kt_begin + it;
         const uint32_t b_addr = smem_u32(smem + s * stage_bytes) + kATileBytes;
-        mbar_arrive_expect_tx(full_bar + 8 * s, static_cast<uint32_t>(p.n_cols) * 128u);
+        mbar_arrive_expect_tx(full_bar + 8 * s, static_cast<uint32_t>(n_acc_here * p.acc_n) * 128u);
         if (MODE == 0) {
           for (int g = 0; g < p.n_cols / 64; ++g)
             tma_load_2d(b_addr + g * (kTileK * 128), &grad_map, o0 + g * 64, kt * kTileK,
@@ -155,9 +158,21 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         } else {
           const int img = kt / p.tiles_per_img;
           const int p0 = (kt - img * p.tiles_per_img) * kTileK;
-          for (int a = 0; a < p.n_acc; ++a)
-            tma_load_3d(b_addr + a * p.acc_n * 128, &grad_map, p0, o0 + a * p.acc_n, img,
+          for (int a = 0; a < n_acc_here; ++a) {
+            // unit -> tap and channel range; the copy holding the tap's column shift, and the
+            // tap's row shift as an offset along the flattened map
+            const int u = u0 + a;
+            const int tap = u / p.upt;
+            const int o_lo = (u - tap * p.upt) * p.acc_n;
+            int copy = tap, x = p0;
+            if (p.row_shift) {
+              const int r = tap / p.kw;
+              copy = tap - r * p.kw;
+              x = p0 + (p.pad - r) * p.in_w;
+            }
+            tma_load_3d(b_addr + a * p.acc_n * 128, &grad_map, x, copy * p.o_real + o_lo, img,
                         full_bar + 8 * s);
+          }
         }
       }
     }
@@ -360,15 +375,24 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
       const int lane_grp = warp & 3;
       const int c = c0 + lane_grp * 32 + static_cast<int>(lane);
       float* out = partial + static_cast<long long>(split) * p.O * p.C;
-      for (int col = 16 * ((warp - 2) >> 2); col < p.n_cols; col += 64) {
+      const int cols_here = n_acc_here * p.acc_n;
+      for (int col = 16 * ((warp - 2) >> 2); col < cols_here; col += 64) {
         uint32_t r[16];
         tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_grp * 32) << 16) + col, r);
+        int row0, n_ok;                   // first partial row of the 16 columns, how many exist
+        if (MODE == 0) {
+          row0 = o0 + col; n_ok = p.O - row0;
+        } else {
+          const int a = col / p.acc_n;
+          const int u = u0 + a;
+          const int tap = u / p.upt;
+          const int o_lo = (u - tap * p.upt) * p.acc_n + (col - a * p.acc_n);
+          row0 = tap * p.o_real + o_lo; n_ok = p.o_real - o_lo;
+        }
         if (c < p.C) {
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const int o = o0 + col + e;
-            if (o < p.O) out[static_cast<long long>(o) * p.C + c] = __uint_as_float(r[e]);
-          }
+          for (int e = 0; e < 16; ++e)
+            if (e < n_ok) out[static_cast<long long>(row0 + e) * p.C + c] = __uint_as_float(r[e]);
         }
       }
     } else if (!done && lane == 0) {
@@ -413,6 +437,44 @@ grad_taps_bf16_kernel(const float* __restrict__ g, unsigned short* __restrict__ 
   }
 }
 
+// The same for rows a multiple of 8 wide, where only the KW column shifts are materialised:
+// out[img][s * O + o][y * W + x'] = g[img][o][y][x' + pad - s] for the OH gradient rows y (zero
+// where the column lies outside the output map).  One thread reads a window of 8 + KW - 1
+// gradient values and writes 8 positions of every shift.
+template <int KW>
+__global__ void __launch_bounds__(256)
+grad_cols_bf16_kernel(const float* __restrict__ g, unsigned short* __restrict__ out,
+                      long long chunks, DirectParams p) {
+  const int per_row = p.in_w >> 3;                     // chunks per map row
+  const int per_plane = p.pitch >> 3;                  // pitch = OH * W
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < chunks;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const long long plane = i / per_plane;             // img * O + o
+    const int chunk = static_cast<int>(i - plane * per_plane);
+    const int y = chunk / per_row;
+    const int x0 = (chunk - y * per_row) * 8;
+    const long long img = plane / p.o_real;
+    const int o = static_cast<int>(plane - img * p.o_real);
+    const float* src = g + (plane * p.oh + y) * static_cast<long long>(p.ow);
+    float f[8 + KW - 1];                               // f[j] = g[y][x0 + pad - (KW - 1) + j]
+#pragma unroll
+    for (int j = 0; j < 8 + KW - 1; ++j) {
+      const int x = x0 + p.pad - (KW - 1) + j;
+      f[j] = (x >= 0 && x < p.ow) ? __ldg(src + x) : 0.0f;
+    }
+#pragma unroll
+    for (int sft = 0; sft < KW; ++sft) {
+      const int b = KW - 1 - sft;                      // element e of shift sft is f[e + b]
+      uint4 w;
+      w.x = pack_bf16x2(f[b], f[b + 1]); w.y = pack_bf16x2(f[b + 2], f[b + 3]);
+      w.z = pack_bf16x2(f[b + 4], f[b + 5]); w.w = pack_bf16x2(f[b + 6], f[b + 7]);
+      unsigned short* dst = out + ((img * KW + sft) * p.o_real + o) * static_cast<long long>(p.pitch) +
+                            static_cast<long long>(chunk) * 8;
+      *reinterpret_cast<uint4*>(dst) = w;
+    }
+  }
+}
+
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                               CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -446,6 +508,9 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
     p.oh = d.h + 2 * d.pad - d.kh + 1; p.ow = d.w + 2 * d.pad - d.kw + 1;
     if (p.oh < 1 || p.ow < 1) return false;
     p.T = d.h * d.w; p.imgs = d.batch;
+    // Rows a multiple of 8 wide: only the kw column shifts need copies; a row shift is a
+    // 16-byte-aligned offset of the TMA coordinate along the flattened map (zero fill outside).
+    p.row_shift = (d.w % 8 == 0 && (d.kw == 2 || d.kw == 3 || d.kw == 5 || d.kw == 7)) ? 1 : 0;
   } else {
     return false;
   }
@@ -453,7 +518,9 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   p.o_real = d.c_out;
   if (static_cast<long long>(p.taps) * d.c_out > 2147483647LL / 256) return false;
   p.C = d.c_in; p.O = p.taps * d.c_out;
-  p.pitch = (p.mode == 0) ? p.O : (p.T + 7) / 8 * 8;   // row pitch of the bf16 gradient copy
+  p.copies = p.row_shift ? p.kw : p.taps;
+  p.g_len = p.row_shift ? p.oh * p.in_w : p.T;         // elements per row of the bf16 gradient copy
+  p.pitch = (p.mode == 0) ? p.O : (p.g_len + 7) / 8 * 8;
   if (p.mode == 0) {
     // columns come in slabs of 64; per CTA two accumulators of 192 or 128 columns, or one small one
     const int g = (p.O + 63) / 64;
@@ -464,22 +531,23 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
       p.acc_n = (t6 <= t4) ? 192 : 128;
     }
   } else {
-    // one or two accumulators of a multiple of 16 columns: the fewest padded columns overall,
-    // then the widest CTA tile
-    long long best_waste = -1;
-    for (int na = 2; na >= 1; --na)
-      for (int c = 256; c >= 16; c -= 16) {
-        const int cols = c * na;
-        const long long padded = static_cast<long long>((p.O + cols - 1) / cols) * cols;
-        const long long waste = padded - p.O;
-        if (best_waste < 0 || waste < best_waste ||
-            (waste == best_waste && cols > p.acc_n * p.n_acc)) {
-          best_waste = waste; p.acc_n = c; p.n_acc = na;
-        }
-      }
+    // Columns come in units: one tap's output channels are cut into `upt` accumulators of acc_n
+    // columns (a multiple of 16 with the fewest padded columns, then the widest); a CTA holds up
+    // to three units (<= 512 TMEM columns) and keeps at least three pipeline stages when it has
+    // several column tiles to choose from.
+    int best_waste = -1;
+    for (int c = 256; c >= 16; c -= 16) {
+      const int upt = (p.o_real + c - 1) / c;
+      const int waste = upt * c - p.o_real;
+      if (best_waste < 0 || waste < best_waste) { best_waste = waste; p.acc_n = c; p.upt = upt; }
+    }
+    p.n_units = p.taps * p.upt;
+    const int col_cap = (p.taps > 1) ? 384 : 512;
+    p.n_acc = 1;
+    while (p.n_acc < 3 && p.n_acc < p.n_units && (p.n_acc + 1) * p.acc_n <= col_cap) ++p.n_acc;
   }
   p.n_cols = p.acc_n * p.n_acc;
-  p.n_tiles = (p.O + p.n_cols - 1) / p.n_cols;
+  p.n_tiles = (p.mode == 0) ? (p.O + p.n_cols - 1) / p.n_cols : (p.n_units + p.n_acc - 1) / p.n_acc;
   p.m_tiles = (p.C + kTileM - 1) / kTileM;
   p.tiles_per_img = (p.T + kTileK - 1) / kTileK;
   const long long total = static_cast<long long>(p.imgs) * p.tiles_per_img;
@@ -513,7 +581,7 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
 
 size_t direct_grad_bf16_bytes(const DirectParams& p) {
   const size_t b = (p.mode == 0) ? static_cast<size_t>(p.T) * p.O * 2
-                                 : static_cast<size_t>(p.imgs) * p.O * p.pitch * 2;
+                                 : static_cast<size_t>(p.imgs) * p.copies * p.o_real * p.pitch * 2;
   return (b + 255) & ~static_cast<size_t>(255);
 }
 
@@ -524,7 +592,21 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
   p.n_words = (act.n + 31) / 32;
   p.partial_blk = (act.n % SURGEON_BLOCK) ? static_cast<unsigned>(act.n / SURGEON_BLOCK) : 0xFFFFFFFFu;
   cudaError_t e;
-  if (p.taps > 1) {
+  if (p.row_shift) {
+    const long long chunks = static_cast<long long>(p.imgs) * p.o_real * (p.pitch >> 3);
+    const long long want = (chunks + 255) / 256;
+    const long long cap = 32LL * sm_count();
+    const int grid = static_cast<int>(want < 1 ? 1 : (want > cap ? cap : want));
+    unsigned short* ob = static_cast<unsigned short*>(grad_bf16);
+    switch (p.kw) {
+      case 2: grad_cols_bf16_kernel<2><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p); break;
+      case 3: grad_cols_bf16_kernel<3><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p); break;
+      case 5: grad_cols_bf16_kernel<5><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p); break;
+      default: grad_cols_bf16_kernel<7><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p); break;
+    }
+    note_launches(1);
+    e = cudaGetLastError();
+  } else if (p.taps > 1) {
     const long long chunks = static_cast<long long>(p.imgs) * p.O * (p.pitch >> 3);
     const long long want = (chunks + 255) / 256;
     const long long cap = 32LL * sm_count();
@@ -552,10 +634,10 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else {
-    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(p.T), static_cast<cuuint64_t>(p.O),
-                                static_cast<cuuint64_t>(p.imgs)};
+    const cuuint64_t rows = static_cast<cuuint64_t>(p.copies) * p.o_real;
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(p.g_len), rows, static_cast<cuuint64_t>(p.imgs)};
     const cuuint64_t strides[2] = {static_cast<cuuint64_t>(p.pitch) * 2,
-                                   static_cast<cuuint64_t>(p.pitch) * p.O * 2};
+                                   static_cast<cuuint64_t>(p.pitch) * rows * 2};
     const cuuint32_t box[3] = {static_cast<cuuint32_t>(kTileK), static_cast<cuuint32_t>(p.acc_n), 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, grad_bf16, dims, strides, box, estr,
