@@ -15,9 +15,8 @@
 // The activation operand is rebuilt from the compressed store by 16 producer warps, 8 per K-tile,
 // two tiles in flight: a lane owns a run of 32 consecutive elements (64 bytes of the swizzled
 // tile), finds the rank of its first kept element from the block offset and the block's bitmap
-// words, zero-fills its 64 bytes and scatters the kept values into them, so the work is
-// proportional to the number of kept elements.  The metadata of a lane's next run is fetched
-// while the current one is rebuilt.
+// words, and rebuilds the run as four 16-byte chunks with one predicated load per element (all
+// independent).  The metadata of a lane's next run is fetched while the current one is rebuilt.
 // One thread issues the MMAs, one the TMA loads; split-K partial tiles are reduced in a fixed
 // order by the caller.  Every wait is bounded and ends in SURGEON_ERR_TIMEOUT.
 #include <cuda.h>
@@ -323,11 +322,31 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
       rank += __popc(w0 & ((1u << sh) - 1u));
       uint32_t bits = __funnelshift_r(w0, w1, sh);
       bits = cur.nvalid >= 32 ? bits : (bits & ((1u << cur.nvalid) - 1u));
-      const uint32_t count = __popc(bits);
-      const uint32_t max_count = __reduce_max_sync(0xFFFFFFFFu, count);
-      uint32_t v[8];
+      // The run as four 16-byte chunks of 8 elements: every element is one predicated load (its
+      // place in the packed vector advances with each kept element before it), so the 32 loads
+      // of a lane are independent and nothing is stored twice.
+      uint4 chunk[4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) v[i] = ld_packed<DT>(values, rank + i, static_cast<uint32_t>(i) < count);
+      for (int q = 0; q < 4; ++q) {
+        const uint32_t byte = (bits >> (8 * q)) & 0xFFu;
+        uint32_t idx = rank + (q == 0 ? 0u : __popc(bits & ((1u << (8 * q)) - 1u)));
+        uint32_t v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const uint32_t on = (byte >> e) & 1u;
+          v[e] = ld_packed<DT>(values, idx, on != 0);
+          idx += on;
+        }
+        if (DT == 0) {
+          chunk[q].x = pack_bf16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
+          chunk[q].y = pack_bf16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
+          chunk[q].z = pack_bf16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
+          chunk[q].w = pack_bf16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
+        } else {
+          chunk[q].x = v[0] | (v[1] << 16); chunk[q].y = v[2] | (v[3] << 16);
+          chunk[q].z = v[4] | (v[5] << 16); chunk[q].w = v[6] | (v[7] << 16);
+        }
+      }
 
       const int s = it % p.stages;
       if (it >= p.stages && lane == 0 && !mbar_wait(empty_bar + 8 * s, ((it / p.stages) - 1) & 1, 32)) {
@@ -339,24 +358,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
       unsigned char* dst_row = smem + s * stage_bytes + rowbase;
 #pragma unroll
       for (int q = 0; q < 4; ++q)
-        *reinterpret_cast<uint4*>(dst_row + (((y + q) ^ xr) << 4)) = make_uint4(0, 0, 0, 0);
-      uint32_t left = bits;
-      for (uint32_t g = 0; g < max_count; g += 8) {
-        if (g > 0) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) v[i] = ld_packed<DT>(values, rank + g + i, g + i < count);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          if (g + i < count) {
-            const uint32_t b = __ffs(left) - 1;
-            left &= left - 1;
-            const unsigned short h = (DT == 0) ? to_bf16_bits(__uint_as_float(v[i]))
-                                               : static_cast<unsigned short>(v[i]);
-            *reinterpret_cast<unsigned short*>(dst_row + (((y + (b >> 3)) ^ xr) << 4) + ((b & 7) << 1)) = h;
-          }
-        }
-      }
+        *reinterpret_cast<uint4*>(dst_row + (((y + q) ^ xr) << 4)) = chunk[q];
       fence_proxy_async();
       __syncwarp();
       if (lane == 0) mbar_arrive(full_bar + 8 * s);
