@@ -55,7 +55,8 @@ struct DirectParams {
   int acc_n, n_acc, n_cols; // columns per accumulator, accumulators per CTA, their product
   int m_tiles, n_tiles, splits;
   int tiles_per_img, total_ktiles, ktiles_per_split;
-  int stages, tmem_cols, smem_bytes;
+  int a_stages, b_stages;   // depth of the activation-tile and gradient-tile rings
+  int tmem_cols, smem_bytes;
   long long n_words;        // words of the bitmap (filled by the launcher)
   unsigned partial_blk;     // index of the bitmap's last block if it is partial, else 0xFFFFFFFF
 };

@@ -36,7 +36,8 @@ constexpr int kTileK = 64;
 constexpr int kProdWarps = 16;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kThreads = 64 + kProdThreads;     // warp 0: MMA, warp 1: TMA, warps 2..17: producers
-constexpr int kMaxStages = 4;
+constexpr int kMaxAStages = 8;
+constexpr int kMaxBStages = 4;
 constexpr int kATileBytes = kTileM * kTileK * 2;              // 16 KB
 
 // Shared-memory matrix descriptor of an MN-major operand with 128-byte swizzle: rows of 64
@@ -71,8 +72,12 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  const int stage_bytes = kATileBytes + p.n_cols * 128;
-  __shared__ __align__(8) unsigned long long bars[2 * kMaxStages + 1];
+  // Two rings: activation tiles (16 KB each, many) and gradient tiles (n_cols rows each, few).
+  // The activation ring is deep because rebuilding a tile takes longer than its MMAs; the
+  // gradient tiles arrive by TMA well ahead and need only be double- or triple-buffered.
+  const int b_stage_bytes = p.n_cols * 128;
+  unsigned char* b_ring = smem + p.a_stages * kATileBytes;
+  __shared__ __align__(8) unsigned long long bars[2 * kMaxAStages + 2 * kMaxBStages + 1];
   __shared__ uint32_t tmem_slot;
   __shared__ volatile uint32_t fail;
 
@@ -88,14 +93,20 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   const int kt_end = min(kt_begin + p.ktiles_per_split, p.total_ktiles);
   const int n_kt = kt_end - kt_begin;
 
-  const uint32_t full_bar = smem_u32(bars);
-  const uint32_t empty_bar = smem_u32(bars + kMaxStages);
-  const uint32_t acc_bar = smem_u32(bars + 2 * kMaxStages);
+  const uint32_t full_a = smem_u32(bars);
+  const uint32_t empty_a = smem_u32(bars + kMaxAStages);
+  const uint32_t full_b = smem_u32(bars + 2 * kMaxAStages);
+  const uint32_t empty_b = smem_u32(bars + 2 * kMaxAStages + kMaxBStages);
+  const uint32_t acc_bar = smem_u32(bars + 2 * kMaxAStages + 2 * kMaxBStages);
   if (tid == 0) {
     tma_prefetch_desc(&grad_map);
-    for (int s = 0; s < p.stages; ++s) {
-      mbar_init(full_bar + 8 * s, kProdWarps / 2 + 1);   // the 8 warps of a tile + the TMA thread
-      mbar_init(empty_bar + 8 * s, 1);
+    for (int s = 0; s < p.a_stages; ++s) {
+      mbar_init(full_a + 8 * s, kProdWarps / 2);       // the 8 warps that rebuild a tile
+      mbar_init(empty_a + 8 * s, 1);
+    }
+    for (int s = 0; s < p.b_stages; ++s) {
+      mbar_init(full_b + 8 * s, 1);                    // the TMA thread (+ the bytes it expects)
+      mbar_init(empty_b + 8 * s, 1);
     }
     mbar_init(acc_bar, 1);
     fail = 0;
@@ -111,27 +122,28 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
     // ================= MMA issuer =================
     if (lane == 0) {
       const uint32_t idesc = make_idesc(kTileM, p.acc_n) | (MODE == 0 ? ((1u << 15) | (1u << 16)) : 0u);
-      const uint32_t smem0 = smem_u32(smem);
-      const uint64_t a_base = (MODE == 0) ? make_desc_mn(smem0) : make_desc(smem0);
-      const uint64_t b_base = (MODE == 0) ? make_desc_mn(smem0 + kATileBytes) : make_desc(smem0 + kATileBytes);
-      const uint64_t stage_inc = static_cast<uint64_t>(stage_bytes >> 4);
+      const uint64_t a_base = (MODE == 0) ? make_desc_mn(smem_u32(smem)) : make_desc(smem_u32(smem));
+      const uint64_t b_base = (MODE == 0) ? make_desc_mn(smem_u32(b_ring)) : make_desc(smem_u32(b_ring));
+      const uint64_t a_inc = static_cast<uint64_t>(kATileBytes >> 4);
+      const uint64_t b_inc = static_cast<uint64_t>(b_stage_bytes >> 4);
       const uint64_t acc_inc = static_cast<uint64_t>((p.acc_n * 128) >> 4);
       constexpr int kStep = (MODE == 0) ? 128 : 2;
       uint64_t da = a_base, db = b_base;
-      uint32_t parity = 0, accum = 0;
-      int s = 0;
+      uint32_t pa = 0, pb = 0, accum = 0;
+      int sa = 0, sb = 0;
       bool ok = true;
       for (int it = 0; it < n_kt; ++it) {
-        ok = mbar_wait(full_bar + 8 * s, parity);
+        ok = mbar_wait_suspend(full_b + 8 * sb, pb) && mbar_wait_suspend(full_a + 8 * sa, pa);
         if (!ok) break;
         tc_fence_after();
         if (n_acc_here == 1) umma_ktile<1, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
         else if (n_acc_here == 2) umma_ktile<2, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
         else umma_ktile<3, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
-        umma_commit(empty_bar + 8 * s);
+        umma_commit(empty_a + 8 * sa);
+        umma_commit(empty_b + 8 * sb);
         accum = 1;
-        if (++s == p.stages) { s = 0; parity ^= 1; da = a_base; db = b_base; }
-        else { da += stage_inc; db += stage_inc; }
+        if (++sa == p.a_stages) { sa = 0; pa ^= 1; da = a_base; } else { da += a_inc; }
+        if (++sb == p.b_stages) { sb = 0; pb ^= 1; db = b_base; } else { db += b_inc; }
       }
       if (!ok) { fail = 1; atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); }
       umma_commit(acc_bar);
@@ -140,23 +152,24 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   } else if (warp == 1) {
     // ================= gradient tiles by TMA =================
     if (lane == 0) {
+      int sb = 0;
+      uint32_t round = 0;
+      int img = 0, kin = 0;                            // conv: image and K-tile within it
+      if (MODE != 0) { img = kt_begin / p.tiles_per_img; kin = kt_begin - img * p.tiles_per_img; }
       for (int it = 0; it < n_kt; ++it) {
-        const int s = it % p.stages;
-        if (it >= p.stages && !mbar_wait(empty_bar + 8 * s, ((it / p.stages) - 1) & 1)) {
+        if (round > 0 && !mbar_wait_suspend(empty_b + 8 * sb, (round - 1) & 1)) {
           fail = 1;
           atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
           break;
         }
-        const int kt = kt_begin + it;
-        const uint32_t b_addr = smem_u32(smem + s * stage_bytes) + kATileBytes;
-        mbar_arrive_expect_tx(full_bar + 8 * s, static_cast<uint32_t>(n_acc_here * p.acc_n) * 128u);
+        const uint32_t b_addr = smem_u32(b_ring + sb * b_stage_bytes);
+        mbar_arrive_expect_tx(full_b + 8 * sb, static_cast<uint32_t>(n_acc_here * p.acc_n) * 128u);
         if (MODE == 0) {
           for (int g = 0; g < p.n_cols / 64; ++g)
-            tma_load_2d(b_addr + g * (kTileK * 128), &grad_map, o0 + g * 64, kt * kTileK,
-                        full_bar + 8 * s);
+            tma_load_2d(b_addr + g * (kTileK * 128), &grad_map, o0 + g * 64, (kt_begin + it) * kTileK,
+                        full_b + 8 * sb);
         } else {
-          const int img = kt / p.tiles_per_img;
-          const int p0 = (kt - img * p.tiles_per_img) * kTileK;
+          const int p0 = kin * kTileK;
           for (int a = 0; a < n_acc_here; ++a) {
             // unit -> tap and channel range; the copy holding the tap's column shift, and the
             // tap's row shift as an offset along the flattened map
@@ -170,9 +183,11 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
               x = p0 + (p.pad - r) * p.in_w;
             }
             tma_load_3d(b_addr + a * p.acc_n * 128, &grad_map, x, copy * p.o_real + o_lo, img,
-                        full_bar + 8 * s);
+                        full_b + 8 * sb);
           }
+          if (++kin == p.tiles_per_img) { kin = 0; ++img; }
         }
+        if (++sb == p.b_stages) { sb = 0; ++round; }
       }
     }
     __syncwarp();
@@ -180,8 +195,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
     // ================= producers =================
     // Warps 2..9 rebuild the even K-tiles of this CTA's range, warps 10..17 the odd ones.  A lane
     // owns one run of 32 consecutive elements per tile (linear: 32 channels of one row t; conv: 32
-    // positions of one channel) = 64 bytes of the operand tile: it zero-fills them and then
-    // scatters the kept values, whose count is what the work is proportional to.
+    // positions of one channel) = 64 bytes of the operand tile.
     const int pw = warp - 2;
     const int wg = pw >> 3, w8 = pw & 7;
     int row, part;                       // tile row and which run of the row
@@ -190,6 +204,21 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
     const uint32_t xr = row & 7;
     const uint32_t y = (MODE == 0) ? (part & 1) * 4 : part * 4;     // first 16-byte chunk of the run
     const uint32_t rowbase = (MODE == 0) ? (part >> 1) * (kTileK * 128) + row * 128 : row * 128;
+    // ring position of this group's tile `it` (= it % a_stages) and how often it has wrapped
+    int sa = wg % p.a_stages;
+    uint32_t round = 0;
+    auto wait_stage = [&]() -> bool {
+      if (round > 0 && lane == 0 && !mbar_wait_suspend(empty_a + 8 * sa, (round - 1) & 1)) {
+        fail = 1;                                  // one lane polls; the warp follows
+        atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+      }
+      __syncwarp();
+      return fail == 0;
+    };
+    auto next_stage = [&]() {
+      sa += 2;
+      if (sa >= p.a_stages) { sa -= p.a_stages; ++round; }
+    };
     if (MODE == 2) {
       // 1x1 stride-2 conv: the run's 32 output positions sample every other element of every
       // other input row.  Per output-row segment: 64 bitmap bits from the segment's first input
@@ -201,14 +230,8 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         const int q0 = (kt - img * p.tiles_per_img) * kTileK + 32 * part;     // first output position
         const int c = c0 + row;
         int left = (c < p.C) ? min(32, p.T - q0) : 0;
-        const int s = it % p.stages;
-        if (it >= p.stages && lane == 0 && !mbar_wait(empty_bar + 8 * s, ((it / p.stages) - 1) & 1, 32)) {
-          fail = 1;
-          atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
-        }
-        __syncwarp();
-        if (fail) break;
-        unsigned char* dst_row = smem + s * stage_bytes + rowbase;
+        if (!wait_stage()) break;
+        unsigned char* dst_row = smem + sa * kATileBytes + rowbase;
 #pragma unroll
         for (int q = 0; q < 4; ++q)
           *reinterpret_cast<uint4*>(dst_row + (((y + q) ^ xr) << 4)) = make_uint4(0, 0, 0, 0);
@@ -241,13 +264,12 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
           // packed places of the kept samples are not contiguous (skipped odd elements lie
           // between them): eight loads in flight per round
           while (ev) {
-            uint32_t idx[8], vv[8];
+            uint32_t vv[8];
             uint32_t e2 = ev;
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
               const int i = e2 ? __ffs(e2) - 1 : 0;
-              idx[u] = rank + __popcll(win & ((1ull << (2 * i)) - 1ull));
-              vv[u] = ld_packed<DT>(values, idx[u], e2 != 0);
+              vv[u] = ld_packed<DT>(values, rank + __popcll(win & ((1ull << (2 * i)) - 1ull)), e2 != 0);
               e2 &= e2 - 1;
             }
 #pragma unroll
@@ -265,106 +287,122 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         }
         fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(full_bar + 8 * s);
+        if (lane == 0) mbar_arrive(full_a + 8 * sa);
+        next_stage();
       }
     } else {
-    auto fetch = [&](int it) {
-      WordRaw r;
-      r.base = 0; r.next = 0; r.words = make_uint4(0, 0, 0, 0); r.j = 0; r.nvalid = 0;
-      const int kt = kt_begin + it;
-      long long j;
-      int nvalid;
+      // Flat index of the lane's run in the group's first tile, advanced by two tiles per round
+      // without multiplications: linear j = t * C + c; conv j = (img * C + c) * T + position.
+      const int kt_first = kt_begin + wg;
+      long long j_run;                     // linear: flat index; conv: flat index of the row's image plane
+      long long t_row = 0;                 // linear: row t of the run
+      int kin = 0;                         // conv: K-tile within the image
+      int n_run;                           // linear: channels of the run that exist (constant)
       if (MODE == 0) {
-        const long long t = static_cast<long long>(kt) * kTileK + row;
         const int c = c0 + 32 * part;
-        nvalid = (t < p.T) ? min(32, p.C - c) : 0;
-        j = t * p.C + c;
+        n_run = max(0, min(32, p.C - c));
+        t_row = static_cast<long long>(kt_first) * kTileK + row;
+        j_run = t_row * p.C + c;
       } else {
-        const int img = kt / p.tiles_per_img;
-        const int pp = (kt - img * p.tiles_per_img) * kTileK + 32 * part;
-        const int c = c0 + row;
-        nvalid = (c < p.C) ? min(32, p.T - pp) : 0;
-        j = (static_cast<long long>(img) * p.C + c) * p.T + pp;
+        const int img = kt_first / p.tiles_per_img;
+        kin = kt_first - img * p.tiles_per_img;
+        n_run = (c0 + row < p.C) ? 1 : 0;
+        j_run = (static_cast<long long>(img) * p.C + (c0 + row)) * p.T;
       }
-      if (nvalid > 0) {
-        r.nvalid = static_cast<uint32_t>(nvalid);
-        r.j = static_cast<uint32_t>(j);
-        const uint32_t blk = r.j >> kBlockShift;
-        const long long wi = r.j >> 5;
-        r.base = __ldg(offsets + blk);
-        if (blk != p.partial_blk) {
-          r.words = __ldg(reinterpret_cast<const uint4*>(bitmap) + blk);
-        } else {                                   // the last, partial block of the bitmap
-          const long long w0 = static_cast<long long>(blk) * kBlockWords;
-          r.words.x = __ldg(bitmap + w0);
-          r.words.y = (w0 + 1 < p.n_words) ? __ldg(bitmap + w0 + 1) : 0u;
-          r.words.z = (w0 + 2 < p.n_words) ? __ldg(bitmap + w0 + 2) : 0u;
-          r.words.w = (w0 + 3 < p.n_words) ? __ldg(bitmap + w0 + 3) : 0u;
-        }
-        if ((r.j & 31u) && wi + 1 < p.n_words) r.next = __ldg(bitmap + wi + 1);
-      }
-      return r;
-    };
-    const int first_it = wg;
-    WordRaw cur = {};
-    if (first_it < n_kt) cur = fetch(first_it);
-    for (int it = first_it; it < n_kt; it += 2) {
-      WordRaw nxt = {};
-      if (it + 2 < n_kt) nxt = fetch(it + 2);       // in flight while this tile is rebuilt
-      // bits of the run and rank of its first kept element
-      const uint32_t wq = (cur.j >> 5) & 3, sh = cur.j & 31;
-      uint32_t rank = cur.base;
-      rank += wq > 0 ? __popc(cur.words.x) : 0u;
-      rank += wq > 1 ? __popc(cur.words.y) : 0u;
-      rank += wq > 2 ? __popc(cur.words.z) : 0u;
-      const uint32_t w0 = wq == 0 ? cur.words.x : (wq == 1 ? cur.words.y : (wq == 2 ? cur.words.z : cur.words.w));
-      const uint32_t w1 = wq == 3 ? cur.next : (wq == 0 ? cur.words.y : (wq == 1 ? cur.words.z : cur.words.w));
-      rank += __popc(w0 & ((1u << sh) - 1u));
-      uint32_t bits = __funnelshift_r(w0, w1, sh);
-      bits = cur.nvalid >= 32 ? bits : (bits & ((1u << cur.nvalid) - 1u));
-      // The run as four 16-byte chunks of 8 elements: every element is one predicated load (its
-      // place in the packed vector advances with each kept element before it), so the 32 loads
-      // of a lane are independent and nothing is stored twice.
-      uint4 chunk[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const uint32_t byte = (bits >> (8 * q)) & 0xFFu;
-        uint32_t idx = rank + (q == 0 ? 0u : __popc(bits & ((1u << (8 * q)) - 1u)));
-        uint32_t v[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const uint32_t on = (byte >> e) & 1u;
-          v[e] = ld_packed<DT>(values, idx, on != 0);
-          idx += on;
-        }
-        if (DT == 0) {
-          chunk[q].x = pack_bf16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
-          chunk[q].y = pack_bf16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
-          chunk[q].z = pack_bf16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
-          chunk[q].w = pack_bf16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
+      const long long j_step = (MODE == 0) ? 2LL * kTileK * p.C : static_cast<long long>(p.C) * p.T;
+      auto fetch = [&]() {                 // metadata of the run at the current position
+        WordRaw r;
+        r.base = 0; r.next = 0; r.words = make_uint4(0, 0, 0, 0); r.j = 0; r.nvalid = 0;
+        long long j;
+        int nvalid;
+        if (MODE == 0) {
+          nvalid = (t_row < p.T) ? n_run : 0;
+          j = j_run;
         } else {
-          chunk[q].x = v[0] | (v[1] << 16); chunk[q].y = v[2] | (v[3] << 16);
-          chunk[q].z = v[4] | (v[5] << 16); chunk[q].w = v[6] | (v[7] << 16);
+          const int pp = kin * kTileK + 32 * part;
+          nvalid = n_run ? max(0, min(32, p.T - pp)) : 0;
+          j = j_run + pp;
         }
-      }
-
-      const int s = it % p.stages;
-      if (it >= p.stages && lane == 0 && !mbar_wait(empty_bar + 8 * s, ((it / p.stages) - 1) & 1, 32)) {
-        fail = 1;                                  // one lane polls; the warp follows
-        atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
-      }
-      __syncwarp();
-      if (fail) break;
-      unsigned char* dst_row = smem + s * stage_bytes + rowbase;
+        if (nvalid > 0) {
+          r.nvalid = static_cast<uint32_t>(nvalid);
+          r.j = static_cast<uint32_t>(j);
+          const long long blk = j >> kBlockShift;
+          const long long wi = j >> 5;
+          r.base = __ldg(offsets + blk);
+          if (static_cast<unsigned long long>(blk) != p.partial_blk) {
+            r.words = __ldg(reinterpret_cast<const uint4*>(bitmap) + blk);
+          } else {                                   // the last, partial block of the bitmap
+            const long long w0 = blk * kBlockWords;
+            r.words.x = __ldg(bitmap + w0);
+            r.words.y = (w0 + 1 < p.n_words) ? __ldg(bitmap + w0 + 1) : 0u;
+            r.words.z = (w0 + 2 < p.n_words) ? __ldg(bitmap + w0 + 2) : 0u;
+            r.words.w = (w0 + 3 < p.n_words) ? __ldg(bitmap + w0 + 3) : 0u;
+          }
+          if ((r.j & 31u) && wi + 1 < p.n_words) r.next = __ldg(bitmap + wi + 1);
+        }
+        return r;
+      };
+      auto advance = [&]() {               // two K-tiles on
+        if (MODE == 0) { t_row += 2 * kTileK; j_run += j_step; }
+        else {
+          kin += 2;
+          while (kin >= p.tiles_per_img) { kin -= p.tiles_per_img; j_run += j_step; }
+        }
+      };
+      WordRaw cur = {};
+      if (wg < n_kt) cur = fetch();
+      for (int it = wg; it < n_kt; it += 2) {
+        WordRaw nxt = {};
+        advance();
+        if (it + 2 < n_kt) nxt = fetch();             // in flight while this tile is rebuilt
+        // bits of the run and rank of its first kept element
+        const uint32_t wq = (cur.j >> 5) & 3, sh = cur.j & 31;
+        uint32_t rank = cur.base;
+        rank += wq > 0 ? __popc(cur.words.x) : 0u;
+        rank += wq > 1 ? __popc(cur.words.y) : 0u;
+        rank += wq > 2 ? __popc(cur.words.z) : 0u;
+        const uint32_t w0 = wq == 0 ? cur.words.x : (wq == 1 ? cur.words.y : (wq == 2 ? cur.words.z : cur.words.w));
+        const uint32_t w1 = wq == 3 ? cur.next : (wq == 0 ? cur.words.y : (wq == 1 ? cur.words.z : cur.words.w));
+        rank += __popc(w0 & ((1u << sh) - 1u));
+        uint32_t bits = __funnelshift_r(w0, w1, sh);
+        bits = cur.nvalid >= 32 ? bits : (bits & ((1u << cur.nvalid) - 1u));
+        // The run as four 16-byte chunks of 8 elements: every element is one predicated load (its
+        // place in the packed vector advances with each kept element before it), so the 32 loads
+        // of a lane are independent and nothing is stored twice.
+        uint4 chunk[4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q)
-        *reinterpret_cast<uint4*>(dst_row + (((y + q) ^ xr) << 4)) = chunk[q];
-      fence_proxy_async();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(full_bar + 8 * s);
-      cur = nxt;
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t byte = (bits >> (8 * q)) & 0xFFu;
+          uint32_t idx = rank + (q == 0 ? 0u : __popc(bits & ((1u << (8 * q)) - 1u)));
+          uint32_t v[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const uint32_t on = (byte >> e) & 1u;
+            v[e] = ld_packed<DT>(values, idx, on != 0);
+            idx += on;
+          }
+          if (DT == 0) {
+            chunk[q].x = pack_bf16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
+            chunk[q].y = pack_bf16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
+            chunk[q].z = pack_bf16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
+            chunk[q].w = pack_bf16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
+          } else {
+            chunk[q].x = v[0] | (v[1] << 16); chunk[q].y = v[2] | (v[3] << 16);
+            chunk[q].z = v[4] | (v[5] << 16); chunk[q].w = v[6] | (v[7] << 16);
+          }
+        }
+        if (!wait_stage()) break;
+        unsigned char* dst_row = smem + sa * kATileBytes + rowbase;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          *reinterpret_cast<uint4*>(dst_row + (((y + q) ^ xr) << 4)) = chunk[q];
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full_a + 8 * sa);
+        next_stage();
+        cur = nxt;
+      }
     }
-    }  // MODE != 2
   }
 
   // ================= epilogue: TMEM -> scratch partial tile =================
@@ -519,6 +557,7 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   if (p.taps == 0) p.taps = 1;
   p.o_real = d.c_out;
   if (static_cast<long long>(p.taps) * d.c_out > 2147483647LL / 256) return false;
+  if (p.taps > 1 && d.c_out > 65535) return false;    // grid of the tap reduction
   p.C = d.c_in; p.O = p.taps * d.c_out;
   p.copies = p.row_shift ? p.kw : p.taps;
   p.g_len = p.row_shift ? p.oh * p.in_w : p.T;         // elements per row of the bf16 gradient copy
@@ -535,8 +574,7 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   } else {
     // Columns come in units: one tap's output channels are cut into `upt` accumulators of acc_n
     // columns (a multiple of 16 with the fewest padded columns, then the widest); a CTA holds up
-    // to three units (<= 512 TMEM columns) and keeps at least three pipeline stages when it has
-    // several column tiles to choose from.
+    // to three units (<= 512 TMEM columns).
     int best_waste = -1;
     for (int c = 256; c >= 16; c -= 16) {
       const int upt = (p.o_real + c - 1) / c;
@@ -544,7 +582,7 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
       if (best_waste < 0 || waste < best_waste) { best_waste = waste; p.acc_n = c; p.upt = upt; }
     }
     p.n_units = p.taps * p.upt;
-    const int col_cap = (p.taps > 1) ? 384 : 512;
+    const int col_cap = 512;
     p.n_acc = 1;
     while (p.n_acc < 3 && p.n_acc < p.n_units && (p.n_acc + 1) * p.acc_n <= col_cap) ++p.n_acc;
   }
@@ -571,12 +609,17 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   p.splits = (p.total_ktiles + p.ktiles_per_split - 1) / p.ktiles_per_split;
   p.tmem_cols = 32;
   while (p.tmem_cols < p.n_cols) p.tmem_cols *= 2;
-  const int stage_bytes = kATileBytes + p.n_cols * 128;
-  int stages = (225 * 1024 - 1024) / stage_bytes;
-  if (stages > kMaxStages) stages = kMaxStages;
-  if (stages < 2) return false;
-  p.stages = stages;
-  p.smem_bytes = stages * stage_bytes + 1024;
+  // shared memory: gradient ring (3 tiles, 2 when they are large), then as many activation
+  // tiles as fit (up to 8)
+  const int budget = 224 * 1024 - 1024;
+  const int b_bytes = p.n_cols * 128;
+  int b_stages = (3 * b_bytes + 4 * kATileBytes <= budget) ? 3 : 2;
+  if (b_stages * b_bytes + 2 * kATileBytes > budget) return false;
+  int a_stages = (budget - b_stages * b_bytes) / kATileBytes;
+  if (a_stages > kMaxAStages) a_stages = kMaxAStages;
+  if (a_stages < 2) return false;
+  p.a_stages = a_stages; p.b_stages = b_stages;
+  p.smem_bytes = a_stages * kATileBytes + b_stages * b_bytes + 1024;
   *out = p;
   return true;
 }
