@@ -169,21 +169,107 @@ __device__ __forceinline__ unsigned short to_bf16_bits(float v) {
 }
 
 
+// ---- CTA pairs (cta_group::2): two CTAs of a cluster of 2 act as one MMA of M = 256 ---------
+// Each CTA holds 128 rows of A, half of the N rows of B and its own 128 x N accumulator; the
+// CTA of rank 0 issues the MMAs and owns the "full" barriers, commits arrive in both CTAs.
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;   // shared::cluster address -> the same offset in rank 0
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst),
+               "r"(cols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
+               : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b,
+                                               uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the mbarrier at this offset in both CTAs of the pair once the MMAs issued so far
+// have completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"(static_cast<unsigned short>(3))
+      : "memory");
+}
+// TMA load into this CTA's shared memory whose bytes count on rank 0's mbarrier at offset `bar`.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t smem_dst, const void* tmap, int x, int y,
+                                                 int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(smem_dst), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(bar & kPeerBitMask)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t smem_dst, const void* tmap, int x, int y,
+                                                 uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_dst), "l"(tmap), "r"(x), "r"(y), "r"(bar & kPeerBitMask)
+      : "memory");
+}
+// Arrive (release at cluster scope) on rank 0's mbarrier at offset `bar`.
+__device__ __forceinline__ void mbar_arrive_rank0(uint32_t bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar & kPeerBitMask)
+               : "memory");
+}
+// Suspended bounded wait with acquire at cluster scope (data written by the other CTA).
+__device__ __forceinline__ bool mbar_wait_suspend_cluster(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < (1u << 21); ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(1000u)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void fence_proxy_async_all() {
+  asm volatile("fence.proxy.async;" ::: "memory");
+}
+
 // The MMAs of one K-tile of 64: four K-steps into each of N_ACC accumulators of `acc_n` columns.
 // `da` / `db` are the descriptors of the stage's operands; a K-step advances the start-address
 // field by KSTEP (16-byte units: 2 for K-major rows, 128 for MN-major slabs), an accumulator's B
 // rows lie `acc_inc` units further.  The issuing thread's own instructions are the bound of
 // the tensor pipe when they are many (each MMA of 128 columns lasts only 64 clocks), so
 // nothing here is computed per MMA beyond two additions.
-template <int N_ACC, int KSTEP>
+template <int N_ACC, int KSTEP, int PAIR = 0>
 __device__ __forceinline__ void umma_ktile(uint32_t tmem_base, uint32_t acc_n, uint64_t da, uint64_t db,
                                            uint64_t acc_inc, uint32_t idesc, uint32_t accum) {
 #pragma unroll
   for (int a = 0; a < N_ACC; ++a) {
 #pragma unroll
-    for (int kk = 0; kk < 4; ++kk)
-      umma_bf16(tmem_base + a * acc_n, da + static_cast<uint64_t>(kk * KSTEP),
-                db + a * acc_inc + static_cast<uint64_t>(kk * KSTEP), idesc, kk > 0 ? 1u : accum);
+    for (int kk = 0; kk < 4; ++kk) {
+      if (PAIR)
+        umma_bf16_pair(tmem_base + a * acc_n, da + static_cast<uint64_t>(kk * KSTEP),
+                       db + a * acc_inc + static_cast<uint64_t>(kk * KSTEP), idesc, kk > 0 ? 1u : accum);
+      else
+        umma_bf16(tmem_base + a * acc_n, da + static_cast<uint64_t>(kk * KSTEP),
+                  db + a * acc_inc + static_cast<uint64_t>(kk * KSTEP), idesc, kk > 0 ? 1u : accum);
+    }
   }
 }
 

@@ -64,7 +64,7 @@ struct WordRaw {
   uint32_t nvalid;     // elements of the run that exist (0: nothing to do)
 };
 
-template <int DT, int MODE>
+template <int DT, int MODE, int PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ values,
                  const uint32_t* __restrict__ offsets, const __grid_constant__ CUtensorMap grad_map,
@@ -75,7 +75,10 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   // Two rings: activation tiles (16 KB each, many) and gradient tiles (n_cols rows each, few).
   // The activation ring is deep because rebuilding a tile takes longer than its MMAs; the
   // gradient tiles arrive by TMA well ahead and need only be double- or triple-buffered.
-  const int b_stage_bytes = p.n_cols * 128;
+  // In a CTA pair each CTA holds half of the gradient rows of every accumulator.
+  const int b_stage_bytes = p.n_cols * (PAIR ? 64 : 128);
+  const int acc_rows = PAIR ? p.acc_n / 2 : p.acc_n;     // gradient rows per accumulator in this CTA
+  const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
   unsigned char* b_ring = smem + p.a_stages * kATileBytes;
   __shared__ __align__(8) unsigned long long bars[2 * kMaxAStages + 2 * kMaxBStages + 1];
   __shared__ uint32_t tmem_slot;
@@ -101,7 +104,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   if (tid == 0) {
     tma_prefetch_desc(&grad_map);
     for (int s = 0; s < p.a_stages; ++s) {
-      mbar_init(full_a + 8 * s, kProdWarps / 2);       // the 8 warps that rebuild a tile
+      mbar_init(full_a + 8 * s, (PAIR ? 2 : 1) * (kProdWarps / 2));   // the 8 warps (of each CTA) that rebuild a tile
       mbar_init(empty_a + 8 * s, 1);
     }
     for (int s = 0; s < p.b_stages; ++s) {
@@ -112,41 +115,48 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
     fail = 0;
     fence_barrier_init();
   }
-  if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), p.tmem_cols);
+  if (warp == 0) {
+    if (PAIR) tmem_alloc_pair(smem_u32(&tmem_slot), p.tmem_cols);
+    else tmem_alloc(smem_u32(&tmem_slot), p.tmem_cols);
+  }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();          // both CTAs' barriers exist before either is arrived on
   tc_fence_after();
   const uint32_t tmem_base = tmem_slot;
 
   if (warp == 0) {
-    // ================= MMA issuer =================
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc(kTileM, p.acc_n) | (MODE == 0 ? ((1u << 15) | (1u << 16)) : 0u);
+    // ================= MMA issuer (rank 0 of a pair) =================
+    if (lane == 0 && cta_rank == 0) {
+      const uint32_t idesc = make_idesc(PAIR ? 2 * kTileM : kTileM, p.acc_n) | (MODE == 0 ? ((1u << 15) | (1u << 16)) : 0u);
       const uint64_t a_base = (MODE == 0) ? make_desc_mn(smem_u32(smem)) : make_desc(smem_u32(smem));
       const uint64_t b_base = (MODE == 0) ? make_desc_mn(smem_u32(b_ring)) : make_desc(smem_u32(b_ring));
       const uint64_t a_inc = static_cast<uint64_t>(kATileBytes >> 4);
       const uint64_t b_inc = static_cast<uint64_t>(b_stage_bytes >> 4);
-      const uint64_t acc_inc = static_cast<uint64_t>((p.acc_n * 128) >> 4);
+      const uint64_t acc_inc = static_cast<uint64_t>((acc_rows * 128) >> 4);
       constexpr int kStep = (MODE == 0) ? 128 : 2;
       uint64_t da = a_base, db = b_base;
       uint32_t pa = 0, pb = 0, accum = 0;
       int sa = 0, sb = 0;
       bool ok = true;
       for (int it = 0; it < n_kt; ++it) {
-        ok = mbar_wait_suspend(full_b + 8 * sb, pb) && mbar_wait_suspend(full_a + 8 * sa, pa);
+        ok = mbar_wait_suspend(full_b + 8 * sb, pb) &&
+             (PAIR ? mbar_wait_suspend_cluster(full_a + 8 * sa, pa) : mbar_wait_suspend(full_a + 8 * sa, pa));
         if (!ok) break;
         tc_fence_after();
-        if (n_acc_here == 1) umma_ktile<1, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
-        else if (n_acc_here == 2) umma_ktile<2, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
-        else umma_ktile<3, kStep>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
-        umma_commit(empty_a + 8 * sa);
-        umma_commit(empty_b + 8 * sb);
+        if (n_acc_here == 1) umma_ktile<1, kStep, PAIR>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
+        else if (n_acc_here == 2) umma_ktile<2, kStep, PAIR>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
+        else if (n_acc_here == 3) umma_ktile<3, kStep, PAIR>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
+        else umma_ktile<4, kStep, PAIR>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
+        if (PAIR) { umma_commit_pair(empty_a + 8 * sa); umma_commit_pair(empty_b + 8 * sb); }
+        else { umma_commit(empty_a + 8 * sa); umma_commit(empty_b + 8 * sb); }
         accum = 1;
         if (++sa == p.a_stages) { sa = 0; pa ^= 1; da = a_base; } else { da += a_inc; }
         if (++sb == p.b_stages) { sb = 0; pb ^= 1; db = b_base; } else { db += b_inc; }
       }
       if (!ok) { fail = 1; atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); }
-      umma_commit(acc_bar);
+      if (PAIR) umma_commit_pair(acc_bar);
+      else umma_commit(acc_bar);
     }
     __syncwarp();
   } else if (warp == 1) {
@@ -163,11 +173,21 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
           break;
         }
         const uint32_t b_addr = smem_u32(b_ring + sb * b_stage_bytes);
-        mbar_arrive_expect_tx(full_b + 8 * sb, static_cast<uint32_t>(n_acc_here * p.acc_n) * 128u);
+        // rank 0 announces the bytes of both CTAs' loads of this tile
+        if (cta_rank == 0)
+          mbar_arrive_expect_tx(full_b + 8 * sb, static_cast<uint32_t>(n_acc_here * p.acc_n) * 128u);
         if (MODE == 0) {
-          for (int g = 0; g < p.n_cols / 64; ++g)
-            tma_load_2d(b_addr + g * (kTileK * 128), &grad_map, o0 + g * 64, (kt_begin + it) * kTileK,
-                        full_b + 8 * sb);
+          if (PAIR) {
+            for (int a = 0; a < p.n_acc; ++a)
+              for (int g = 0; g < acc_rows / 64; ++g)
+                tma_load_2d_pair(b_addr + a * acc_rows * 128 + g * (kTileK * 128), &grad_map,
+                                 o0 + a * p.acc_n + static_cast<int>(cta_rank) * acc_rows + g * 64,
+                                 (kt_begin + it) * kTileK, full_b + 8 * sb);
+          } else {
+            for (int g = 0; g < p.n_cols / 64; ++g)
+              tma_load_2d(b_addr + g * (kTileK * 128), &grad_map, o0 + g * 64, (kt_begin + it) * kTileK,
+                          full_b + 8 * sb);
+          }
         } else {
           const int p0 = kin * kTileK;
           for (int a = 0; a < n_acc_here; ++a) {
@@ -182,8 +202,9 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
               copy = tap - r * p.kw;
               x = p0 + (p.pad - r) * p.in_w;
             }
-            tma_load_3d(b_addr + a * p.acc_n * 128, &grad_map, x, copy * p.o_real + o_lo, img,
-                        full_b + 8 * sb);
+            const int grow = copy * p.o_real + o_lo + static_cast<int>(cta_rank) * acc_rows;
+            if (PAIR) tma_load_3d_pair(b_addr + a * acc_rows * 128, &grad_map, x, grow, img, full_b + 8 * sb);
+            else tma_load_3d(b_addr + a * acc_rows * 128, &grad_map, x, grow, img, full_b + 8 * sb);
           }
           if (++kin == p.tiles_per_img) { kin = 0; ++img; }
         }
@@ -285,9 +306,9 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
           }
           b0 += seg; left -= seg; ox = 0; ++oy;
         }
-        fence_proxy_async();
+        if (PAIR) fence_proxy_async_all(); else fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(full_a + 8 * sa);
+        if (lane == 0) { if (PAIR) mbar_arrive_rank0(full_a + 8 * sa); else mbar_arrive(full_a + 8 * sa); }
         next_stage();
       }
     } else {
@@ -396,9 +417,9 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
 #pragma unroll
         for (int q = 0; q < 4; ++q)
           *reinterpret_cast<uint4*>(dst_row + (((y + q) ^ xr) << 4)) = chunk[q];
-        fence_proxy_async();
+        if (PAIR) fence_proxy_async_all(); else fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(full_a + 8 * sa);
+        if (lane == 0) { if (PAIR) mbar_arrive_rank0(full_a + 8 * sa); else mbar_arrive(full_a + 8 * sa); }
         next_stage();
         cur = nxt;
       }
@@ -441,7 +462,11 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+  if (PAIR) cluster_sync_all();          // neither CTA leaves while the pair's MMAs or arrivals may touch it
+  if (warp == 0) {
+    if (PAIR) tmem_dealloc_pair(tmem_base, p.tmem_cols);
+    else tmem_dealloc(tmem_base, p.tmem_cols);
+  }
 }
 
 // Shifted bf16 copies of the output gradient of a k x k stride-1 convolution (Eq. 2 summed over
@@ -562,7 +587,20 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   p.copies = p.row_shift ? p.kw : p.taps;
   p.g_len = p.row_shift ? p.oh * p.in_w : p.T;         // elements per row of the bf16 gradient copy
   p.pitch = (p.mode == 0) ? p.O : (p.g_len + 7) / 8 * 8;
-  if (p.mode == 0) {
+  p.m_tiles = (p.C + kTileM - 1) / kTileM;
+  // Two or more row tiles: CTA pairs (each CTA 128 rows, the pair shares every gradient tile).
+  p.pair = (p.m_tiles >= 2) ? 1 : 0;
+  if (p.pair) p.m_tiles = (p.m_tiles + 1) / 2 * 2;
+  if (p.mode == 0 && p.pair) {
+    // accumulators of 128 columns (each CTA of the pair loads a 64-column slab of each), up to four
+    const int units = (p.O + 127) / 128;
+    p.acc_n = 128;
+    int best_pad = -1;
+    for (int na = 4; na >= 1; --na) {
+      const int padded = (units + na - 1) / na * na;
+      if (best_pad < 0 || padded < best_pad) { best_pad = padded; p.n_acc = na; }
+    }
+  } else if (p.mode == 0) {
     // columns come in slabs of 64; per CTA two accumulators of 192 or 128 columns, or one small one
     const int g = (p.O + 63) / 64;
     if (g <= 4) { p.n_acc = 1; p.acc_n = g * 64; }
@@ -588,7 +626,6 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   }
   p.n_cols = p.acc_n * p.n_acc;
   p.n_tiles = (p.mode == 0) ? (p.O + p.n_cols - 1) / p.n_cols : (p.n_units + p.n_acc - 1) / p.n_acc;
-  p.m_tiles = (p.C + kTileM - 1) / kTileM;
   p.tiles_per_img = (p.T + kTileK - 1) / kTileK;
   const long long total = static_cast<long long>(p.imgs) * p.tiles_per_img;
   if (total > 2147483647LL / 4) return false;
@@ -612,7 +649,7 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   // shared memory: gradient ring (3 tiles, 2 when they are large), then as many activation
   // tiles as fit (up to 8)
   const int budget = 224 * 1024 - 1024;
-  const int b_bytes = p.n_cols * 128;
+  const int b_bytes = p.n_cols * (p.pair ? 64 : 128);
   int b_stages = (3 * b_bytes + 4 * kATileBytes <= budget) ? 3 : 2;
   if (b_stages * b_bytes + 2 * kATileBytes > budget) return false;
   int a_stages = (budget - b_stages * b_bytes) / kATileBytes;
@@ -683,7 +720,8 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
     const cuuint64_t dims[3] = {static_cast<cuuint64_t>(p.g_len), rows, static_cast<cuuint64_t>(p.imgs)};
     const cuuint64_t strides[2] = {static_cast<cuuint64_t>(p.pitch) * 2,
                                    static_cast<cuuint64_t>(p.pitch) * rows * 2};
-    const cuuint32_t box[3] = {static_cast<cuuint32_t>(kTileK), static_cast<cuuint32_t>(p.acc_n), 1};
+    const cuuint32_t box[3] = {static_cast<cuuint32_t>(kTileK),
+                               static_cast<cuuint32_t>(p.pair ? p.acc_n / 2 : p.acc_n), 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, grad_bf16, dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -695,13 +733,36 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            p.smem_bytes);
     if (err != cudaSuccess) return err;
-    kernel<<<grid, kThreads, p.smem_bytes, stream>>>(act.bitmap, act.values, act.block_offsets, map,
-                                                     partial, status, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = static_cast<size_t>(p.smem_bytes);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = p.pair ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, act.bitmap, act.values, act.block_offsets, map, partial,
+                              status, p);
   };
-  if (p.mode == 0) e = act.dt == 0 ? launch(dw_direct_kernel<0, 0>) : launch(dw_direct_kernel<1, 0>);
-  else if (p.mode == 2) e = act.dt == 0 ? launch(dw_direct_kernel<0, 2>) : launch(dw_direct_kernel<1, 2>);
-  else e = act.dt == 0 ? launch(dw_direct_kernel<0, 1>) : launch(dw_direct_kernel<1, 1>);
+  const int key = p.mode * 4 + (act.dt ? 2 : 0) + p.pair;
+  switch (key) {
+    case 0: e = launch(dw_direct_kernel<0, 0, 0>); break;
+    case 1: e = launch(dw_direct_kernel<0, 0, 1>); break;
+    case 2: e = launch(dw_direct_kernel<1, 0, 0>); break;
+    case 3: e = launch(dw_direct_kernel<1, 0, 1>); break;
+    case 4: e = launch(dw_direct_kernel<0, 1, 0>); break;
+    case 5: e = launch(dw_direct_kernel<0, 1, 1>); break;
+    case 6: e = launch(dw_direct_kernel<1, 1, 0>); break;
+    case 7: e = launch(dw_direct_kernel<1, 1, 1>); break;
+    case 8: e = launch(dw_direct_kernel<0, 2, 0>); break;
+    case 9: e = launch(dw_direct_kernel<0, 2, 1>); break;
+    case 10: e = launch(dw_direct_kernel<1, 2, 0>); break;
+    default: e = launch(dw_direct_kernel<1, 2, 1>); break;
+  }
   note_launches(1);
   return e;
 }
