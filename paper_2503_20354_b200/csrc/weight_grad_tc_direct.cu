@@ -21,6 +21,8 @@
 // order by the caller.  Every wait is bounded and ends in SURGEON_ERR_TIMEOUT.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "surgeon_internal.cuh"
 #include "tc_common.cuh"
 #include "weight_grad_tc_conv.cuh"
@@ -33,9 +35,20 @@ using namespace tc;
 
 constexpr int kTileM = 128;
 constexpr int kTileK = 64;
-constexpr int kProdWarps = 16;
+constexpr int kGroups = 2;                       // producer groups of 8 warps, one K-tile in flight each
+constexpr int kProdWarps = 8 * kGroups;
 constexpr int kProdThreads = kProdWarps * 32;
 constexpr int kThreads = 64 + kProdThreads;     // warp 0: MMA, warp 1: TMA, warps 2..17: producers
+// CTA pairs (cta_group::2) halve the gradient traffic per MMA.  They measured slower than single
+// CTAs while the activation producers are the bound (a pair waits for the slower of its two
+// tiles), so they are off unless the environment variable SURGEON_DW_PAIRS is set to 1.
+static bool use_pairs() {
+  static const bool on = [] {
+    const char* e = std::getenv("SURGEON_DW_PAIRS");
+    return e && e[0] == '1';
+  }();
+  return on;
+}
 constexpr int kMaxAStages = 8;
 constexpr int kMaxBStages = 4;
 constexpr int kATileBytes = kTileM * kTileK * 2;              // 16 KB
@@ -104,7 +117,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   if (tid == 0) {
     tma_prefetch_desc(&grad_map);
     for (int s = 0; s < p.a_stages; ++s) {
-      mbar_init(full_a + 8 * s, (PAIR ? 2 : 1) * (kProdWarps / 2));   // the 8 warps (of each CTA) that rebuild a tile
+      mbar_init(full_a + 8 * s, (PAIR ? 2 : 1) * 8);   // the 8 warps (of each CTA) that rebuild a tile
       mbar_init(empty_a + 8 * s, 1);
     }
     for (int s = 0; s < p.b_stages; ++s) {
@@ -214,7 +227,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
     __syncwarp();
   } else {
     // ================= producers =================
-    // Warps 2..9 rebuild the even K-tiles of this CTA's range, warps 10..17 the odd ones.  A lane
+    // Group g (warps 2 + 8g .. 9 + 8g) rebuilds the K-tiles g, g + kGroups, ... of this CTA's range.  A lane
     // owns one run of 32 consecutive elements per tile (linear: 32 channels of one row t; conv: 32
     // positions of one channel) = 64 bytes of the operand tile.
     const int pw = warp - 2;
@@ -227,7 +240,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
     const uint32_t rowbase = (MODE == 0) ? (part >> 1) * (kTileK * 128) + row * 128 : row * 128;
     // ring position of this group's tile `it` (= it % a_stages) and how often it has wrapped
     int sa = wg % p.a_stages;
-    uint32_t round = 0;
+    uint32_t round = wg / p.a_stages;
     auto wait_stage = [&]() -> bool {
       if (round > 0 && lane == 0 && !mbar_wait_suspend(empty_a + 8 * sa, (round - 1) & 1)) {
         fail = 1;                                  // one lane polls; the warp follows
@@ -237,15 +250,15 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
       return fail == 0;
     };
     auto next_stage = [&]() {
-      sa += 2;
-      if (sa >= p.a_stages) { sa -= p.a_stages; ++round; }
+      sa += kGroups;
+      while (sa >= p.a_stages) { sa -= p.a_stages; ++round; }
     };
     if (MODE == 2) {
       // 1x1 stride-2 conv: the run's 32 output positions sample every other element of every
       // other input row.  Per output-row segment: 64 bitmap bits from the segment's first input
       // element, the even ones are the segment's bits; a kept element's place in the packed
       // vector counts the odd (skipped) bits before it as well.
-      for (int it = wg; it < n_kt; it += 2) {
+      for (int it = wg; it < n_kt; it += kGroups) {
         const int kt = kt_begin + it;
         const int img = kt / p.tiles_per_img;
         const int q0 = (kt - img * p.tiles_per_img) * kTileK + 32 * part;     // first output position
@@ -330,7 +343,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         n_run = (c0 + row < p.C) ? 1 : 0;
         j_run = (static_cast<long long>(img) * p.C + (c0 + row)) * p.T;
       }
-      const long long j_step = (MODE == 0) ? 2LL * kTileK * p.C : static_cast<long long>(p.C) * p.T;
+      const long long j_step = (MODE == 0) ? static_cast<long long>(kGroups) * kTileK * p.C : static_cast<long long>(p.C) * p.T;
       auto fetch = [&]() {                 // metadata of the run at the current position
         WordRaw r;
         r.base = 0; r.next = 0; r.words = make_uint4(0, 0, 0, 0); r.j = 0; r.nvalid = 0;
@@ -364,18 +377,18 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         return r;
       };
       auto advance = [&]() {               // two K-tiles on
-        if (MODE == 0) { t_row += 2 * kTileK; j_run += j_step; }
+        if (MODE == 0) { t_row += kGroups * kTileK; j_run += j_step; }
         else {
-          kin += 2;
+          kin += kGroups;
           while (kin >= p.tiles_per_img) { kin -= p.tiles_per_img; j_run += j_step; }
         }
       };
       WordRaw cur = {};
       if (wg < n_kt) cur = fetch();
-      for (int it = wg; it < n_kt; it += 2) {
+      for (int it = wg; it < n_kt; it += kGroups) {
         WordRaw nxt = {};
         advance();
-        if (it + 2 < n_kt) nxt = fetch();             // in flight while this tile is rebuilt
+        if (it + kGroups < n_kt) nxt = fetch();             // in flight while this tile is rebuilt
         // bits of the run and rank of its first kept element
         const uint32_t wq = (cur.j >> 5) & 3, sh = cur.j & 31;
         uint32_t rank = cur.base;
@@ -428,8 +441,8 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
 
   // ================= epilogue: TMEM -> scratch partial tile =================
   if (warp >= 2) {
-    // 16 warps: a warp may read the 32 TMEM lanes of its quarter (warp % 4); the four warps of a
-    // quarter take every fourth group of 16 columns
+    // a warp may read the 32 TMEM lanes of its quarter (warp % 4); the warps of a quarter take
+    // the groups of 16 columns in turn
     const bool done = mbar_wait(acc_bar, 0, 64);
     tc_fence_after();
     if (done && !fail) {
@@ -437,7 +450,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
       const int c = c0 + lane_grp * 32 + static_cast<int>(lane);
       float* out = partial + static_cast<long long>(split) * p.O * p.C;
       const int cols_here = n_acc_here * p.acc_n;
-      for (int col = 16 * ((warp - 2) >> 2); col < cols_here; col += 64) {
+      for (int col = 16 * ((warp - 2) >> 2); col < cols_here; col += 16 * (kProdWarps / 4)) {
         uint32_t r[16];
         tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_grp * 32) << 16) + col, r);
         int row0, n_ok;                   // first partial row of the 16 columns, how many exist
@@ -589,7 +602,7 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   p.pitch = (p.mode == 0) ? p.O : (p.g_len + 7) / 8 * 8;
   p.m_tiles = (p.C + kTileM - 1) / kTileM;
   // Two or more row tiles: CTA pairs (each CTA 128 rows, the pair shares every gradient tile).
-  p.pair = (p.m_tiles >= 2) ? 1 : 0;
+  p.pair = (p.m_tiles >= 2 && use_pairs()) ? 1 : 0;
   if (p.pair) p.m_tiles = (p.m_tiles + 1) / 2 * 2;
   if (p.mode == 0 && p.pair) {
     // accumulators of 128 columns (each CTA of the pair loads a 64-column slab of each), up to four
