@@ -160,7 +160,7 @@ def barrier(world: int):
 class Stack:
     """Device-resident inputs, stores, outputs and scratch of one replica of the workload."""
 
-    def __init__(self, layers, path: int, seed: int, device, worst_case_store=True):
+    def __init__(self, layers, path: int, seed: int, device, worst_case_store=True, n_streams=1):
         from paper_2503_20354_b200 import binding as B
         from paper_2503_20354_b200 import workloads as W
         self.B, self.layers, self.path, self.device = B, layers, path, device
@@ -174,18 +174,43 @@ class Stack:
         self.store = [B.CompressedActivation(l.n_act, l.dt, 0.0, device) for l in layers]
         ws1 = max(s.sizes.workspace_bytes for s in self.store)
         ws2 = max(B.surgeon_weight_grad_workspace(d) for d in self.desc)
-        self.ws = torch.empty(max(ws1, ws2, 256), dtype=torch.uint8, device=device)
+        # Layers are independent of one another (a layer's store is written once in the forward
+        # pass and read once in the backward pass), so they are issued round-robin on n_streams
+        # streams, each with its own scratch: the short dependent kernels of one layer overlap
+        # with those of its neighbours.  Both loops fork from and join the caller's stream.
+        self.n_streams = max(1, int(n_streams))
+        self.streams = [torch.cuda.Stream(device=device) for _ in range(self.n_streams)] if self.n_streams > 1 else []
+        self.ws = [torch.empty(max(ws1, ws2, 256), dtype=torch.uint8, device=device)
+                   for _ in range(self.n_streams)]
         self.ratios = None
+
+    def _fork(self):
+        main = torch.cuda.current_stream(self.device)
+        for st in self.streams:
+            st.wait_stream(main)
+
+    def _join(self):
+        main = torch.cuda.current_stream(self.device)
+        for st in self.streams:
+            main.wait_stream(st)
 
     def step(self, ev=None):
         B = self.B
         if ev: ev[0].record()
         self.ratios = B.surgeon_layer_ratios(self.gi, self.lam, allow_degenerate=True)   # Eq. 5-7
+        self._fork()
         for i in range(len(self.layers)):                                                # forward
-            B.surgeon_prune_compact(self.x[i], float(self.ratios[i]), out=self.store[i], workspace=self.ws)
+            k = i % self.n_streams
+            B.surgeon_prune_compact(self.x[i], float(self.ratios[i]), out=self.store[i], workspace=self.ws[k],
+                                    stream=self.streams[k] if self.streams else None)
+        self._join()
         if ev: ev[1].record()
-        for i in reversed(range(len(self.layers))):                                      # backward
-            B.surgeon_weight_grad(self.store[i], self.desc[i], self.g[i], dw=self.dw[i], workspace=self.ws)
+        self._fork()
+        for j, i in enumerate(reversed(range(len(self.layers)))):                        # backward
+            k = j % self.n_streams
+            B.surgeon_weight_grad(self.store[i], self.desc[i], self.g[i], dw=self.dw[i], workspace=self.ws[k],
+                                  stream=self.streams[k] if self.streams else None)
+        self._join()
         if ev: ev[2].record()
 
 
@@ -260,7 +285,7 @@ def run_ours(args, rank, world, local):
         if len(layers) < 2:
             raise SystemExit("--layers must name at least two layers of the stack (the ratio rule needs two)")
     path = B.PATH_FP32 if args.path == "fp32" else B.PATH_TENSOR_CORE
-    stack = Stack(layers, path, args.seed + rank, device)
+    stack = Stack(layers, path, args.seed + rank, device, n_streams=args.streams)
     torch.cuda.synchronize()
     peaks = load_peaks()
 
@@ -321,7 +346,7 @@ def run_ours(args, rank, world, local):
         "dtype": "bf16" if path == B.PATH_TENSOR_CORE else "f32", "data": "synthetic",
         "config": {"workload": desc_text, "layers": len(layers), "ratios": "GI/LAM rule, GI~LogNormal(0,1)",
                    "path": args.path, "l2": "inputs larger than L2 (%.2f GB read per step)" % ((dense + sum(g.numel() * 4 for g in stack.g)) / 1e9),
-                   "replicas": world},
+                   "replicas": world, "streams": stack.n_streams},
         "parts": {
             "prune_compact": {"ms": round(prune_ms, 4), "GB/s": round(prune_gbs, 1),
                               "frac_hbm": round(prune_gbs / float(peaks["hbm_gbs"]), 4),
@@ -468,6 +493,8 @@ def main():
     ap.add_argument("--layers", default=None, help="comma-separated layer names: run only these (profiling)")
     ap.add_argument("--path", default="tc", choices=["tc", "fp32"])
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--streams", type=int, default=4,
+                    help="streams the independent layers are issued on (1 = the caller's stream only)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--no-e2e", dest="e2e", action="store_false", help="skip the host-buffer leg (profiling runs)")
