@@ -17,6 +17,8 @@
 //
 // Every wait on an mbarrier is bounded; when one gives up the CTA records SURGEON_ERR_TIMEOUT in
 // the scratch status word, frees its tensor memory and returns.
+#include <cuda.h>
+
 #include "surgeon_internal.cuh"
 #include "tc_common.cuh"
 #include "weight_grad_tc_conv.cuh"
@@ -427,6 +429,252 @@ dw_tc_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ value
   if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
 }
 
+// ---- conv layers: the same GEMM with two producer groups and the gradient by TMA ---------------
+// Group g (4 warps) fills the K-tiles g, g + 2, ... of the CTA's range, each group with its own
+// patch, so the load latency of one group's decompression hides behind the other group's gather.
+// The output gradient is a bf16 copy written by a pre-pass ([B][O][pitch]); one thread of the
+// group starts its TMA load when the stage is free.  The gather copies 8 output positions per
+// task; when they lie in one output row and inside the map it is 8 strided shared-memory reads
+// without per-element tests.
+constexpr int kGGroups = 2;
+constexpr int kGGroupWarps = 4;
+constexpr int kGGroupThreads = kGGroupWarps * 32;
+constexpr int kGThreads = 32 + kGGroups * kGGroupThreads;
+constexpr int kGPatchBytes = 24 * 1024;      // per group
+constexpr int kGPatchElems = kGPatchBytes / 2;
+
+__device__ __forceinline__ void ggroup_sync(int g) {
+  asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "n"(kGGroupThreads) : "memory");
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kGThreads, 1)
+dw_conv_im2col_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ values,
+                      const uint32_t* __restrict__ offsets,
+                      const __grid_constant__ CUtensorMap grad_map, float* __restrict__ partial,
+                      uint32_t* __restrict__ status, TcParams p) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  const int b_bytes = p.tile_n * 128;
+  const int stage_bytes = kTileM * 128 + b_bytes;
+  unsigned char* patch_base = smem + p.stages * stage_bytes;
+  __shared__ __align__(8) unsigned long long bars[2 * kMaxStages + 1];
+  __shared__ RowInfo rows[kTileM];
+  __shared__ int2 chunk_yx[kGGroups][8];      // output (y, x) of the first position of each chunk
+  __shared__ uint32_t tmem_slot;
+  __shared__ volatile uint32_t fail;
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  const uint32_t lane = lane_id();
+  const int m_tile = blockIdx.x, n_tile = blockIdx.y, split = blockIdx.z;
+  const int nn0 = m_tile * kTileM;
+  const int o0 = n_tile * p.tile_n;
+  const int kt_begin = split * p.ktiles_per_split;
+  const int kt_end = min(kt_begin + p.ktiles_per_split, p.total_ktiles);
+  const int n_kt = kt_end - kt_begin;
+
+  const uint32_t full_bar = smem_u32(bars);
+  const uint32_t empty_bar = smem_u32(bars + kMaxStages);
+  const uint32_t acc_bar = smem_u32(bars + 2 * kMaxStages);
+  if (tid == 0) {
+    tma_prefetch_desc(&grad_map);
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(full_bar + 8 * s, kGGroupWarps + 1);   // the group's warps + the thread that starts the TMA
+      mbar_init(empty_bar + 8 * s, 1);
+    }
+    mbar_init(acc_bar, 1);
+    fail = 0;
+    fence_barrier_init();
+  }
+  for (int i = tid; i < kTileM; i += kGThreads) {
+    const int nn = nn0 + i;
+    RowInfo ri;
+    if (nn < p.n_gemm) {
+      const int c = nn / p.RS;
+      const int rs = nn - c * p.RS;
+      ri.c = static_cast<short>(c);
+      ri.r = static_cast<signed char>(rs / p.KW);
+      ri.s = static_cast<signed char>(rs - (rs / p.KW) * p.KW);
+    } else {
+      ri.c = -1; ri.r = 0; ri.s = 0;
+    }
+    rows[i] = ri;
+  }
+  if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), p.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_slot;
+
+  if (warp == 0) {
+    // ================= MMA issuer =================
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(kTileM, p.tile_n);
+      const uint32_t smem0 = smem_u32(smem);
+      const uint64_t a_base = make_desc(smem0);
+      const uint64_t b_base = make_desc(smem0 + kTileM * 128);
+      const uint64_t stage_inc = static_cast<uint64_t>(stage_bytes >> 4);
+      uint64_t da = a_base, db = b_base;
+      uint32_t parity = 0, accum = 0;
+      int s = 0;
+      bool ok = true;
+      for (int it = 0; it < n_kt; ++it) {
+        ok = mbar_wait_suspend(full_bar + 8 * s, parity);
+        if (!ok) break;
+        tc_fence_after();
+        umma_ktile<1, 2>(tmem_base, p.tile_n, da, db, 0, idesc, accum);
+        umma_commit(empty_bar + 8 * s);
+        accum = 1;
+        if (++s == p.stages) { s = 0; parity ^= 1; da = a_base; db = b_base; }
+        else { da += stage_inc; db += stage_inc; }
+      }
+      if (!ok) { fail = 1; atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); }
+      umma_commit(acc_bar);
+    }
+    __syncwarp();
+  } else {
+    // ================= producers =================
+    const int g = (warp - 1) / kGGroupWarps;
+    const int gtid = tid - 32 - g * kGGroupThreads;
+    unsigned short* patch = reinterpret_cast<unsigned short*>(patch_base + g * kGPatchBytes);
+    const int first_c = rows[0].c;       // M tiles never start past the end
+    int last_c = first_c;
+    for (int i = kTileM - 1; i >= 0; --i) {
+      if (rows[i].c >= 0) { last_c = rows[i].c; break; }
+    }
+    int s = g % p.stages;
+    uint32_t round = g / p.stages;
+    for (int it = g; it < n_kt; it += kGGroups) {
+      if (round > 0 && gtid == 0 && !mbar_wait_suspend(empty_bar + 8 * s, (round - 1) & 1)) {
+        fail = 1;
+        atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+      }
+      const int kt = kt_begin + it;
+      const int img = kt / p.tiles_per_img;
+      const int p0 = (kt - img * p.tiles_per_img) * kTileK;
+      if (gtid < 8) {                    // where each 8-position chunk of the tile starts
+        const int pp = p0 + 8 * gtid;
+        const int y = pp / p.OW;
+        chunk_yx[g][gtid] = make_int2(y, pp - y * p.OW);
+      }
+      ggroup_sync(g);                    // after it, every thread of the group reads the same `fail`
+      if (fail) break;
+      unsigned char* a_tile = smem + s * stage_bytes;
+      if (gtid == 0) {
+        mbar_arrive_expect_tx(full_bar + 8 * s, static_cast<uint32_t>(b_bytes));
+        tma_load_3d(smem_u32(a_tile) + kTileM * 128, &grad_map, p0, o0, img, full_bar + 8 * s);
+      }
+      const int k_valid = min(kTileK, p.P - p0);
+      const int y_first = p0 / p.OW;
+      const int y_last = (p0 + k_valid - 1) / p.OW;
+      int iy_lo = y_first * p.stride - p.pad;
+      int iy_hi = y_last * p.stride + p.KH - 1 - p.pad;
+      if (iy_lo < 0) iy_lo = 0;
+      if (iy_hi > p.H - 1) iy_hi = p.H - 1;
+      const int range_len = (iy_hi - iy_lo + 1) * p.W;
+      const int runs = (range_len + 31) >> 5;
+      for (int cg = first_c; cg <= last_c; cg += p.group_ch) {
+        const int cg_end = min(cg + p.group_ch, last_c + 1);
+        const int n_tasks = (cg_end - cg) * runs;       // one task = 32 consecutive elements
+        for (int t = gtid; t < n_tasks; t += kGGroupThreads) {
+          const int ci = t / runs, run = t - ci * runs;
+          const long long start =
+              ((static_cast<long long>(img) * p.C + cg + ci) * p.H + iy_lo) * p.W + 32 * run;
+          decompress_run<DT>(bitmap, values, offsets, p.n_words, start,
+                             min(32, range_len - 32 * run), patch + ci * p.ch_pitch + 32 * run);
+        }
+        ggroup_sync(g);
+        int row_lo = cg * p.RS - nn0;
+        int row_hi = cg_end * p.RS - nn0;
+        if (row_lo < 0) row_lo = 0;
+        if (row_hi > kTileM || cg_end > last_c) row_hi = kTileM;   // last group also zeroes pad rows
+        const int tasks = (row_hi - row_lo) * 8;
+        for (int t = gtid; t < tasks; t += kGGroupThreads) {
+          const int row = row_lo + (t >> 3), chunk = t & 7;
+          const RowInfo ri = rows[row];
+          uint32_t h[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) h[e] = 0;
+          const int pp0 = p0 + chunk * 8;
+          if (ri.c >= 0 && pp0 < p.P) {
+            const unsigned short* src = patch + (ri.c - cg) * p.ch_pitch;
+            const int2 yx = chunk_yx[g][chunk];
+            const int iy = yx.x * p.stride + ri.r - p.pad;
+            const int ix0 = yx.y * p.stride + ri.s - p.pad;
+            if (yx.y + 7 < p.OW && pp0 + 7 < p.P) {
+              // the 8 positions lie in one output row
+              if (iy >= iy_lo && iy <= iy_hi) {
+                const unsigned short* rowp = src + (iy - iy_lo) * p.W;
+                if (ix0 >= 0 && ix0 + 7 * p.stride < p.W) {
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) h[e] = rowp[ix0 + e * p.stride];
+                } else {
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) {
+                    const int ix = ix0 + e * p.stride;
+                    if (ix >= 0 && ix < p.W) h[e] = rowp[ix];
+                  }
+                }
+              }
+            } else {
+              int pp = pp0, y = yx.x, x = yx.y;
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const int iy2 = y * p.stride + ri.r - p.pad;
+                const int ix = x * p.stride + ri.s - p.pad;
+                if (pp < p.P && iy2 >= iy_lo && iy2 <= iy_hi && ix >= 0 && ix < p.W)
+                  h[e] = src[(iy2 - iy_lo) * p.W + ix];
+                ++pp; ++x;
+                if (x == p.OW) { x = 0; ++y; }
+              }
+            }
+          }
+          uint4 out;
+          out.x = h[0] | (h[1] << 16); out.y = h[2] | (h[3] << 16);
+          out.z = h[4] | (h[5] << 16); out.w = h[6] | (h[7] << 16);
+          *reinterpret_cast<uint4*>(a_tile + tile_off(row, chunk)) = out;
+        }
+        ggroup_sync(g);   // the patch is overwritten by the next channel group / tile
+      }
+      fence_proxy_async();   // generic-proxy writes -> visible to the tensor core's reads
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full_bar + 8 * s);
+      s += kGGroups;
+      while (s >= p.stages) { s -= p.stages; ++round; }
+    }
+  }
+
+  // ================= epilogue: TMEM -> scratch partial tile =================
+  if (warp >= 1) {
+    const bool done = mbar_wait(acc_bar, 0, 64);
+    tc_fence_after();
+    if (done && !fail) {
+      const int lane_grp = warp & 3;              // TMEM lanes this warp may read
+      const int row = lane_grp * 32 + static_cast<int>(lane);
+      const int nn = nn0 + row;
+      float* out = partial + static_cast<long long>(split) * p.O * p.n_gemm;
+      for (int col = 16 * ((warp - 1) >> 2); col < p.tile_n; col += 32) {
+        uint32_t r[16];
+        tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_grp * 32) << 16) + col, r);
+        if (nn < p.n_gemm) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int o = o0 + col + e;
+            if (o < p.O) out[static_cast<long long>(o) * p.n_gemm + nn] = __uint_as_float(r[e]);
+          }
+        }
+      }
+    } else if (!done && lane == 0) {
+      atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT));
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+}
+
 // Sums the split partials in order and writes (or adds to) dw; copies the device status into
 // the activation's header when a wait timed out.
 __global__ void __launch_bounds__(256)
@@ -532,6 +780,35 @@ size_t smem_bytes(const TcParams& p) {
   return static_cast<size_t>(p.stages) * (kTileM * 128 + p.tile_n * 128) + kPatchBytes + 2048;
 }
 
+// Plan of dw_conv_im2col_kernel: the tiling of `plan`, two patches of kGPatchBytes, and the
+// bf16 gradient copy (rows padded to a multiple of 8 elements for the tensor map).
+bool plan_im2col(const surgeon_layer_desc& d, int dt, TcParams* out, int* pitch) {
+  if (d.kind != 1) return false;
+  TcParams p;
+  if (!plan(d, dt, &p)) return false;
+  const long long per_ch = (static_cast<long long>(p.max_rows) * p.W + 31) / 32 * 32;
+  if (per_ch > kGPatchElems) return false;
+  p.ch_pitch = static_cast<int>(per_ch);
+  p.group_ch = static_cast<int>(kGPatchElems / per_ch);
+  const int stage_bytes = kTileM * 128 + p.tile_n * 128;
+  int stages = (224 * 1024 - kGGroups * kGPatchBytes - 1024) / stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) return false;
+  p.stages = stages;
+  *pitch = (p.P + 7) / 8 * 8;
+  *out = p;
+  return true;
+}
+
+size_t im2col_smem_bytes(const TcParams& p) {
+  return static_cast<size_t>(p.stages) * (kTileM * 128 + p.tile_n * 128) + kGGroups * kGPatchBytes + 1024;
+}
+
+size_t im2col_grad_bytes(const TcParams& p, int pitch) {
+  const size_t b = static_cast<size_t>(p.B) * p.O * pitch * 2;
+  return (b + 255) & ~static_cast<size_t>(255);
+}
+
 }  // namespace
 
 static size_t fast_partial_bytes(const FastParams& f) {
@@ -551,6 +828,10 @@ size_t weight_grad_tc_workspace(const surgeon_layer_desc& d) {
   if (plan_conv_fast(d, &f))
     return kStatusBytes + fast_partial_bytes(f) + conv_fast_grad_bf16_bytes(f);
   TcParams p;
+  int pitch = 0;
+  if (plan_im2col(d, 0, &p, &pitch))
+    return kStatusBytes + ((static_cast<size_t>(p.splits) * p.O * p.n_gemm * sizeof(float) + 255) & ~size_t(255)) +
+           im2col_grad_bytes(p, pitch);
   if (!plan(d, 0, &p)) return 0;
   return kStatusBytes + static_cast<size_t>(p.splits) * p.O * p.n_gemm * sizeof(float);
 }
@@ -589,6 +870,54 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
     return cudaGetLastError();
   }
   TcParams p;
+  int pitch = 0;
+  if (plan_im2col(d, act.dt, &p, &pitch)) {
+    p.n_words = (act.n + 31) / 32;
+    const size_t pbytes = (static_cast<size_t>(p.splits) * p.O * p.n_gemm * sizeof(float) + 255) & ~size_t(255);
+    void* grad_bf16 = reinterpret_cast<char*>(partial) + pbytes;
+    if (pitch != p.P)
+      e = launch_grad_to_bf16_rows(grad_out, static_cast<long long>(p.B) * p.O, p.P, pitch, grad_bf16, stream);
+    else
+      e = launch_grad_to_bf16(grad_out, static_cast<long long>(p.B) * p.O * p.P, grad_bf16, stream);
+    if (e != cudaSuccess) return e;
+    using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+    const EncodeFn encode = reinterpret_cast<EncodeFn>(tensor_map_encode_fn());
+    if (!encode) return cudaErrorNotSupported;
+    CUtensorMap map;
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(p.P), static_cast<cuuint64_t>(p.O),
+                                static_cast<cuuint64_t>(p.B)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(pitch) * 2,
+                                   static_cast<cuuint64_t>(pitch) * p.O * 2};
+    const cuuint32_t box[3] = {static_cast<cuuint32_t>(kTileK), static_cast<cuuint32_t>(p.tile_n), 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, grad_bf16, dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+    const size_t smem = im2col_smem_bytes(p);
+    dim3 grid(p.m_tiles, p.n_tiles, p.splits);
+    if (act.dt == 0) {
+      e = cudaFuncSetAttribute(dw_conv_im2col_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               static_cast<int>(smem));
+      if (e != cudaSuccess) return e;
+      dw_conv_im2col_kernel<0><<<grid, kGThreads, smem, stream>>>(act.bitmap, act.values, act.block_offsets,
+                                                                 map, partial, status, p);
+    } else {
+      e = cudaFuncSetAttribute(dw_conv_im2col_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               static_cast<int>(smem));
+      if (e != cudaSuccess) return e;
+      dw_conv_im2col_kernel<1><<<grid, kGThreads, smem, stream>>>(act.bitmap, act.values, act.block_offsets,
+                                                                 map, partial, status, p);
+    }
+    const long long mn = static_cast<long long>(p.O) * p.n_gemm;
+    reduce_splits_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
+        partial, mn, p.splits, dw, accumulate, status, act.header);
+    note_launches(2);
+    return cudaGetLastError();
+  }
   if (!plan(d, act.dt, &p)) return cudaErrorNotSupported;
   p.n_words = (act.n + 31) / 32;
   const size_t smem = smem_bytes(p);

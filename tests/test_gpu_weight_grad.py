@@ -90,6 +90,13 @@ SHAPES = [
     W.conv("t5x5_hw12", 2, 24, 12, 40, 5, 1, 2),
     W.Layer("t2x3_pad1", 1, 3, 16, 9, 11, 24, 2, 3, 1, 1),
     W.conv("t3x3_hw14_c136", 2, 136, 14, 72, 3),
+    # the two-group im2col kernel: 3x3 stride 2 on 28- and 14-wide maps with channels past one
+    # patch group, 5x5 stride 2, 7x7 stride 3, an output row shorter than a chunk of 8
+    W.conv("g3x3s2_hw28_c40", 2, 40, 28, 136, 3, 2),
+    W.conv("g3x3s2_hw14_c136", 3, 136, 14, 24, 3, 2),
+    W.conv("g5x5s2_hw19", 2, 6, 19, 16, 5, 2, 2),
+    W.conv("g7x7s3_hw30", 1, 5, 30, 8, 7, 3, 3, dist="normal"),
+    W.conv("g3x3s2_hw10", 4, 8, 10, 8, 3, 2),
 ]
 
 
