@@ -430,14 +430,14 @@ dw_tc_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ value
 }
 
 // ---- conv layers: the same GEMM with two producer groups and the gradient by TMA ---------------
-// Group g (4 warps) fills the K-tiles g, g + 2, ... of the CTA's range, each group with its own
+// Group g (8 warps) fills the K-tiles g, g + 2, ... of the CTA's range, each group with its own
 // patch, so the load latency of one group's decompression hides behind the other group's gather.
 // The output gradient is a bf16 copy written by a pre-pass ([B][O][pitch]); one thread of the
 // group starts its TMA load when the stage is free.  The gather copies 8 output positions per
 // task; when they lie in one output row and inside the map it is 8 strided shared-memory reads
 // without per-element tests.
 constexpr int kGGroups = 2;
-constexpr int kGGroupWarps = 4;
+constexpr int kGGroupWarps = 8;
 constexpr int kGGroupThreads = kGGroupWarps * 32;
 constexpr int kGThreads = 32 + kGGroups * kGGroupThreads;
 constexpr int kGPatchBytes = 24 * 1024;      // per group
@@ -655,7 +655,7 @@ dw_conv_im2col_kernel(const uint32_t* __restrict__ bitmap, const void* __restric
       const int row = lane_grp * 32 + static_cast<int>(lane);
       const int nn = nn0 + row;
       float* out = partial + static_cast<long long>(split) * p.O * p.n_gemm;
-      for (int col = 16 * ((warp - 1) >> 2); col < p.tile_n; col += 32) {
+      for (int col = 16 * ((warp - 1) >> 2); col < p.tile_n; col += 16 * (kGGroups * kGGroupWarps / 4)) {
         uint32_t r[16];
         tmem_ld16(tmem_base + (static_cast<uint32_t>(lane_grp * 32) << 16) + col, r);
         if (nn < p.n_gemm) {
