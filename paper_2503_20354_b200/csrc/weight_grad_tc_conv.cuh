@@ -55,6 +55,7 @@ struct DirectParams {
   int acc_n, n_acc, n_cols; // columns per accumulator, accumulators per CTA, their product
   int m_tiles, n_tiles, splits;
   int tiles_per_img, total_ktiles, ktiles_per_split;
+  int rows_per_tile;        // channels per row tile (128, or fewer when C is spread evenly; a multiple of 16)
   int pair;                 // 1: CTA pairs (cta_group::2) over two row tiles; m_tiles is then even
   int a_stages, b_stages;   // depth of the activation-tile and gradient-tile rings
   int tmem_cols, smem_bytes;

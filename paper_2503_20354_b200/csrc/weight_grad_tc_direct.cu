@@ -101,7 +101,8 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   const int warp = tid >> 5;
   const uint32_t lane = lane_id();
   const int m_tile = blockIdx.x, n_tile = blockIdx.y, split = blockIdx.z;
-  const int c0 = m_tile * kTileM;
+  const int c0 = m_tile * p.rows_per_tile;           // first input channel of the CTA's row tile
+  const int rows_here = max(0, min(p.rows_per_tile, p.C - c0));   // tile rows that hold a channel
   const int o0 = n_tile * p.n_cols;                  // linear: first gradient column of the CTA
   const int u0 = n_tile * p.n_acc;                   // conv: first column unit of the CTA
   const int n_acc_here = (MODE == 0) ? p.n_acc : min(p.n_acc, p.n_units - u0);
@@ -253,7 +254,24 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
       sa += kGroups;
       while (sa >= p.a_stages) { sa -= p.a_stages; ++round; }
     };
-    if (MODE == 2) {
+    if (MODE != 0 && 16 * w8 >= rows_here) {
+      // The warp's 16 rows hold no channel (the channels are spread evenly over the row tiles,
+      // so every tile of a layer has idle warps when C is not a multiple of 128): they stay zero
+      // in every stage, and the warp only keeps the barrier counts whole.
+      for (int st = 0; st < p.a_stages; ++st) {
+        unsigned char* dst_row = smem + st * kATileBytes + rowbase;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          *reinterpret_cast<uint4*>(dst_row + (((y + q) ^ xr) << 4)) = make_uint4(0, 0, 0, 0);
+      }
+      for (int it = wg; it < n_kt; it += kGroups) {
+        if (!wait_stage()) break;
+        if (PAIR) fence_proxy_async_all(); else fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) { if (PAIR) mbar_arrive_rank0(full_a + 8 * sa); else mbar_arrive(full_a + 8 * sa); }
+        next_stage();
+      }
+    } else if (MODE == 2) {
       // 1x1 stride-2 conv: the run's 32 output positions sample every other element of every
       // other input row.  Per output-row segment: 64 bitmap bits from the segment's first input
       // element, the even ones are the segment's bits; a kept element's place in the packed
@@ -263,7 +281,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         const int img = kt / p.tiles_per_img;
         const int q0 = (kt - img * p.tiles_per_img) * kTileK + 32 * part;     // first output position
         const int c = c0 + row;
-        int left = (c < p.C) ? min(32, p.T - q0) : 0;
+        int left = (row < rows_here) ? min(32, p.T - q0) : 0;
         if (!wait_stage()) break;
         unsigned char* dst_row = smem + sa * kATileBytes + rowbase;
 #pragma unroll
@@ -340,7 +358,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
       } else {
         const int img = kt_first / p.tiles_per_img;
         kin = kt_first - img * p.tiles_per_img;
-        n_run = (c0 + row < p.C) ? 1 : 0;
+        n_run = (row < rows_here) ? 1 : 0;
         j_run = (static_cast<long long>(img) * p.C + (c0 + row)) * p.T;
       }
       const long long j_step = (MODE == 0) ? static_cast<long long>(kGroups) * kTileK * p.C : static_cast<long long>(p.C) * p.T;
@@ -463,7 +481,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
           const int o_lo = (u - tap * p.upt) * p.acc_n + (col - a * p.acc_n);
           row0 = tap * p.o_real + o_lo; n_ok = p.o_real - o_lo;
         }
-        if (c < p.C) {
+        if (lane_grp * 32 + static_cast<int>(lane) < rows_here) {
 #pragma unroll
           for (int e = 0; e < 16; ++e)
             if (e < n_ok) out[static_cast<long long>(row0 + e) * p.C + c] = __uint_as_float(r[e]);
@@ -601,6 +619,8 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   p.g_len = p.row_shift ? p.oh * p.in_w : p.T;         // elements per row of the bf16 gradient copy
   p.pitch = (p.mode == 0) ? p.O : (p.g_len + 7) / 8 * 8;
   p.m_tiles = (p.C + kTileM - 1) / kTileM;
+  // conv: the channels are spread evenly over the row tiles, in units of a warp's 16 rows
+  p.rows_per_tile = (p.mode == 0) ? kTileM : ((p.C + p.m_tiles - 1) / p.m_tiles + 15) / 16 * 16;
   // Two or more row tiles: CTA pairs (each CTA 128 rows, the pair shares every gradient tile).
   p.pair = (p.m_tiles >= 2 && use_pairs()) ? 1 : 0;
   if (p.pair) p.m_tiles = (p.m_tiles + 1) / 2 * 2;
