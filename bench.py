@@ -77,8 +77,40 @@ class ClockSampler:
 
     def __init__(self, device_index: int):
         self.lines, self.proc, self.idx = [], None, device_index
+        self.nvml, self.samples, self.stop_flag, self.t = None, [], False, None
+
+    def _nvml_loop(self):
+        n = self.nvml
+        h = self.handle
+        while not self.stop_flag:
+            try:
+                sm = n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM)
+                mx = n.nvmlDeviceGetMaxClockInfo(h, n.NVML_CLOCK_SM)
+                try:
+                    r = n.nvmlDeviceGetCurrentClocksEventReasons(h)
+                except Exception:
+                    r = n.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                self.samples.append((sm, mx, int(r)))
+            except Exception:
+                pass
+            time.sleep(0.01)
 
     def start(self):
+        # NVML in a thread (a sample every 10 ms, reading only); nvidia-smi as the fall-back
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            if vis and not vis.split(",")[self.idx].isdigit():
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(vis.split(",")[self.idx])
+            else:
+                self.handle = pynvml.nvmlDeviceGetHandleByIndex(int(vis.split(",")[self.idx]) if vis else self.idx)
+            self.nvml = pynvml
+            self.t = threading.Thread(target=self._nvml_loop, daemon=True)
+            self.t.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             vis = os.environ.get("CUDA_VISIBLE_DEVICES")
             idx = vis.split(",")[self.idx] if vis else str(self.idx)
@@ -95,6 +127,18 @@ class ClockSampler:
             self.lines.append(line.strip())
 
     def stop(self):
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        if self.nvml is not None:
+            self.stop_flag = True
+            self.t.join(timeout=2)
+            bits = {"sw_power_cap": 0x4, "hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20,
+                    "hw_thermal_slowdown": 0x40}
+            reasons = sorted(k for k, b in bits.items() if any(r & b for _, _, r in self.samples))
+            sm = [x[0] for x in self.samples]
+            mx = [x[1] for x in self.samples]
+            return {"sm_mhz": float(np.median(sm)) if sm else None,
+                    "sm_max_mhz": float(max(mx)) if mx else None,
+                    "samples": len(sm), "reasons": reasons, "source": "nvml, 10 ms"}
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.15)
@@ -104,7 +148,6 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for l in self.lines:
             f = [v.strip() for v in l.split(",")]
             if len(f) < 9:
@@ -118,7 +161,7 @@ class ClockSampler:
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None,
                 "sm_max_mhz": float(max(mx)) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "source": "nvidia-smi, 100 ms"}
 
 
 def dist_setup(n_gpus: int):
@@ -484,7 +527,7 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="wrn28", choices=["wrn28", "tiny", "resnet50", "vit", "sweep"])
