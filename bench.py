@@ -536,7 +536,7 @@ def main():
     ap.add_argument("--layers", default=None, help="comma-separated layer names: run only these (profiling)")
     ap.add_argument("--path", default="tc", choices=["tc", "fp32"])
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--streams", type=int, default=4,
+    ap.add_argument("--streams", type=int, default=8,
                     help="streams the independent layers are issued on (1 = the caller's stream only)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
