@@ -487,13 +487,35 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
 }
 
 // n_keep == 0 (ratio 1, or an empty tensor): nothing to select.
-__global__ void header_empty_kernel(surgeon_header* hdr, uint32_t sentinel) {
+__global__ void header_empty_kernel(surgeon_header* hdr, uint32_t sentinel, uint32_t* offsets,
+                                    long long n_blocks) {
+  if (n_blocks > 0) offsets[n_blocks] = 0u;      // the sentinel entry of the block offsets
   hdr->threshold_key = sentinel;
   hdr->status = SURGEON_OK;
   hdr->n_keep = 0;
   hdr->n_greater = 0;
   hdr->tie_quota = 0;
 }
+
+constexpr unsigned long long kCountMask = 0x7FFFFFFFull;
+constexpr int kRows = 4;                 // rows of 32 lanes x 16 bytes per warp
+constexpr int kTileWarps = kTileVecs / (kRows * 32);   // warps of the generic per-tile kernels
+static_assert(kTileWarps * kRows * 32 == kTileVecs, "compaction tile");
+constexpr int kCompactThreads = kTileWarps * 32;
+
+// Defined with the compaction kernels below; the count kernel emits the boundary tile itself.
+template <int DT, bool SLOW>
+__device__ __forceinline__ void compact_tile(const typename Elem<DT>::type* __restrict__ x,
+                                             long long n, const uint4 (&q)[kRows], int tile,
+                                             uint32_t tau, long long quota, bool ties,
+                                             long long gt_tile_before, long long eq_tile_before,
+                                             surgeon_header* __restrict__ hdr,
+                                             uint32_t* __restrict__ bitmap,
+                                             typename Elem<DT>::type* __restrict__ values,
+                                             uint32_t* __restrict__ offsets);
+template <int DT>
+__device__ __forceinline__ void load_tile(const typename Elem<DT>::type* __restrict__ x,
+                                          long long n, int tile, uint4 (&q)[kRows]);
 
 // ---- threshold (where still open), per-chunk counts, exclusive scan ------------------------------
 // Launched cooperatively (all CTAs resident), so that the steps can be separated by grid-wide
@@ -549,12 +571,16 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
              uint32_t* __restrict__ hist_fb, const uint32_t* __restrict__ cnt_gt,
              const uint32_t* __restrict__ cand_cnt, const void* __restrict__ slots_v,
              unsigned long long* __restrict__ val, unsigned long long* __restrict__ prefix,
-             unsigned long long* __restrict__ partial, int tiles) {
+             unsigned long long* __restrict__ partial, int tiles,
+             uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
+             uint32_t* __restrict__ offsets) {
   using E = typename Elem<DT>::type;
   constexpr uint32_t kMask = Elem<DT>::kKeyMask;
   constexpr int EPV = 16 / sizeof(E);
   constexpr long long kChunkElems = static_cast<long long>(kTileVecs) * EPV;
   __shared__ uint32_t s_hist[kBinsB];          // level B / fall-back digit histogram
+  __shared__ int s_bnd;                        // the chunk inside which the tie quota ends, if this CTA owns it
+  __shared__ unsigned long long s_bnd_prefix;
   __shared__ uint32_t scratch[32];
   __shared__ uint32_t res[2];
   __shared__ unsigned long long s_tot[32];
@@ -566,6 +592,7 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
   uint32_t epoch = 0;
   const uint32_t mode = __ldcg(&st->mode);
   uint32_t tau = 0, n_greater = 0;
+  if (tid == 0) s_bnd = -1;                    // read after several barriers below
 
   if (mode == 1u) {
     // ---- fall-back: exact radix select over the tensor itself, one digit per round ----
@@ -755,14 +782,26 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
       prefix[c] = ex;
       const long long eq_b = static_cast<long long>(ex & 0x7FFFFFFFull);
       const long long eq_e = static_cast<long long>((ex + v) & 0x7FFFFFFFull);
-      if (eq_b < quota && eq_e > quota) st->boundary_plus1 = static_cast<uint32_t>(c) + 1u;
+      if (eq_b < quota && eq_e > quota) { s_bnd = c; s_bnd_prefix = ex; }
     }
     carry += __shfl_sync(kFull, incl, 31);
+  }
+  // The chunk inside which the tie quota ends is emitted here, with its ties ranked by index, by
+  // the first two warps of the CTA that owns it; the compaction kernels skip that chunk.
+  __syncthreads();
+  if (s_bnd >= 0 && warp < kTileWarps) {
+    const unsigned long long pb = s_bnd_prefix;
+    uint4 q[kRows];
+    load_tile<DT>(x, n, s_bnd, q);
+    compact_tile<DT, true>(x, n, q, s_bnd, tau, quota, false, static_cast<long long>(pb >> 31),
+                           static_cast<long long>(pb & kCountMask), hdr, bitmap,
+                           reinterpret_cast<E*>(values_v), offsets);
   }
   if (c_end == tiles && c_begin < tiles) {
     // the CTA that owns the last chunk also writes the totals and checks them
     __syncthreads();
     if (tid == 0) {
+      offsets[(n + SURGEON_BLOCK - 1) >> kBlockShift] = k;     // the sentinel entry of the block offsets
       unsigned long long total = 0;
       for (int b = 0; b <= static_cast<int>(blockIdx.x); ++b) total += __ldcg(partial + b);
       prefix[tiles] = total;
@@ -776,12 +815,6 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
 }
 
 // ---- compaction -----------------------------------------------------------------------------
-
-constexpr unsigned long long kCountMask = 0x7FFFFFFFull;
-constexpr int kRows = 4;                 // rows of 32 lanes x 16 bytes per warp
-constexpr int kTileWarps = kTileVecs / (kRows * 32);   // warps of the generic per-tile kernels
-static_assert(kTileWarps * kRows * 32 == kTileVecs, "compaction tile");
-constexpr int kCompactThreads = kTileWarps * 32;
 
 // Keep only the lowest `allowed` set bits of `m`.
 __device__ __forceinline__ uint32_t lowest_set_bits(uint32_t m, long long allowed) {
@@ -848,7 +881,7 @@ __device__ __forceinline__ void compact_tile(const typename Elem<DT>::type* __re
   const uint32_t gt_warp = __reduce_add_sync(kFull, __popc(g_all));
   const uint32_t eq_warp = SLOW ? __reduce_add_sync(kFull, __popc(e_all)) : 0u;
   if (lane == 0) { s_gt[warp] = gt_warp; s_eq[warp] = eq_warp; }
-  __syncthreads();
+  asm volatile("bar.sync 1, %0;" ::"n"(kCompactThreads) : "memory");   // the tile's two warps only
 
   long long gt_before = gt_tile_before, eq_before = eq_tile_before;
 #pragma unroll
@@ -972,7 +1005,7 @@ __device__ __forceinline__ void load_tile(const typename Elem<DT>::type* __restr
 }
 
 // One small CTA per tile: used for tensors too small for the streaming kernel.  The one tile
-// inside which the tie quota ends (if any) is left to compact_boundary_kernel.
+// inside which the tie quota ends (if any) is left to the count kernel.
 template <int DT>
 __global__ void __launch_bounds__(kCompactThreads)
 compact_small_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restrict__ hdr,
@@ -992,31 +1025,6 @@ compact_small_kernel(const void* __restrict__ xv, long long n, surgeon_header* _
   compact_tile<DT, false>(x, n, q, tile, tau, quota, /*ties=*/eq_e <= quota,
                           static_cast<long long>(pb >> 31), eq_b, hdr, bitmap,
                           reinterpret_cast<E*>(values_v), offsets);
-}
-
-// One CTA: finds the tile inside which the tie quota ends and emits it with ties ranked by index.
-template <int DT>
-__global__ void __launch_bounds__(kCompactThreads)
-compact_boundary_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restrict__ hdr,
-                        uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
-                        uint32_t* __restrict__ offsets,
-                        const unsigned long long* __restrict__ prefix,
-                        const SelectState* __restrict__ st, int tiles) {
-  using E = typename Elem<DT>::type;
-  const E* __restrict__ x = reinterpret_cast<const E*>(xv);
-  const long long quota = hdr->tie_quota;
-  if (threadIdx.x == 0)   // the sentinel entry of the block offsets
-    offsets[(n + SURGEON_BLOCK - 1) >> kBlockShift] = static_cast<uint32_t>(hdr->n_keep);
-  const int lo = static_cast<int>(st->boundary_plus1) - 1;   // found by the count kernel's scan
-  if (lo < 0 || lo >= tiles) return;
-  const unsigned long long pb = prefix[lo];
-  const long long eq_b = static_cast<long long>(pb & kCountMask);
-  if (eq_b >= quota) return;                            // the quota ends exactly between tiles
-  uint4 q[kRows];
-  load_tile<DT>(x, n, lo, q);
-  compact_tile<DT, true>(x, n, q, lo, hdr->threshold_key, quota, false,
-                         static_cast<long long>(pb >> 31), eq_b, hdr, bitmap,
-                         reinterpret_cast<E*>(values_v), offsets);
 }
 
 // ---- streaming compaction ---------------------------------------------------------------------
@@ -1101,7 +1109,7 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
     unsigned char* region = ring + s * kCsStageBytes + warp * 4096;   // this warp's 32 rows
     const long long eq_b = static_cast<long long>(pb & kCountMask);
     const long long eq_e = static_cast<long long>(pe & kCountMask);
-    const bool boundary = eq_b < quota && eq_e > quota;   // left to compact_boundary_kernel
+    const bool boundary = eq_b < quota && eq_e > quota;   // left to the count kernel
     if (chunk < n_chunks && !boundary) {
       // ---- this lane's row: 8 vectors, un-swizzled ----
       uint4 q[8];
@@ -1320,7 +1328,8 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
   const bool streamed = n > kSampleMinN && make_row_map(x, n_rows_full, &map);
 
   if (k == 0) {
-    header_empty_kernel<<<1, 1, 0, stream>>>(out.header, Elem<DT>::kSentinel);
+    header_empty_kernel<<<1, 1, 0, stream>>>(out.header, Elem<DT>::kSentinel, out.block_offsets,
+                                             (n + SURGEON_BLOCK - 1) >> kBlockShift);
     note_launches(1);
     if (n > 0) {   // nothing is kept: the scan is all zeros
       e = cudaMemsetAsync(prefix, 0, static_cast<size_t>(L.tiles + 1) * 8, stream);
@@ -1361,8 +1370,11 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
       const uint32_t* cc = cand_cnt;
       const void* sl = slots;
       int tiles = n_chunks;
+      uint32_t* bm = out.bitmap;
+      void* vals = out.values;
+      uint32_t* offs = out.block_offsets;
       void* args[] = {&xa, &na, &ka, &st, &hdr, &hist_b, &hist_fb, &cg, &cc, &sl, &val, &prefix,
-                      &partial, &tiles};
+                      &partial, &tiles, &bm, &vals, &offs};
       e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(count_kernel<DT>), dim3(grid),
                                       dim3(kSelThreads), args, 0, stream);
       if (e != cudaSuccess) return e;
@@ -1380,9 +1392,7 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
     else
       compact_small_kernel<DT><<<static_cast<unsigned>(L.tiles), kCompactThreads, 0, stream>>>(
           x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix);
-    compact_boundary_kernel<DT><<<1, kCompactThreads, 0, stream>>>(
-        x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix, st, n_chunks);
-    note_launches(2);
+    note_launches(1);
   }
   return cudaGetLastError();
 }

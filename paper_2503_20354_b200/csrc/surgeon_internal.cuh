@@ -55,7 +55,7 @@ struct SelectState {
   uint32_t shiftA;               // level A bin of a key = (key - lo_key) >> shiftA
   uint32_t binA, rankA, aboveA;  // level A: bin of the threshold, its rank inside, candidates above
   uint32_t fb_prefix, fb_rank, fb_above;   // fall-back select: key bits fixed so far, rank, count above
-  uint32_t boundary_plus1;       // 1 + the chunk inside which the tie quota ends, 0 if none
+  uint32_t reserved0;            // (unused)
   uint32_t pad[12];
 };
 static_assert(sizeof(SelectState) == 128, "SelectState layout");
