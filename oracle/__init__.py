@@ -44,6 +44,11 @@ def _load():
         c = ctypes
         lib.oracle_layer_ratios.restype = c.c_int
         lib.oracle_layer_ratios.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_void_p]
+        lib.oracle_gradient_importance.restype = c.c_double
+        lib.oracle_gradient_importance.argtypes = [c.c_void_p, c.c_int64]
+        lib.oracle_layer_ratios_rule.restype = c.c_int
+        lib.oracle_layer_ratios_rule.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_double,
+                                                 c.c_void_p]
         lib.oracle_n_keep.restype = c.c_int64
         lib.oracle_n_keep.argtypes = [c.c_int64, c.c_double]
         lib.oracle_select.restype = None
@@ -95,6 +100,26 @@ def layer_ratios(gi, lam):
     p = np.empty_like(g)
     st = _load().oracle_layer_ratios(_ptr(g), _ptr(m), int(g.size), _ptr(p))
     return int(st), p
+
+
+RULE_BOTH, RULE_NO_GRADIENT, RULE_NO_MEMORY, RULE_STATIC = 0, 1, 2, 3
+
+
+def layer_ratios_rule(gi, lam, rule: int, p_static: float = 0.0):
+    """Eq. 5-7 with one factor of Eq. 6 left out ("w/o G", "w/o M") or a global static ratio."""
+    g = np.ascontiguousarray(gi, dtype=np.float64)
+    m = np.ascontiguousarray(lam, dtype=np.float64)
+    assert g.ndim == 1 and g.shape == m.shape
+    p = np.empty_like(g)
+    st = _load().oracle_layer_ratios_rule(_ptr(g), _ptr(m), int(g.size), int(rule), float(p_static),
+                                          _ptr(p))
+    return int(st), p
+
+
+def gradient_importance(dw) -> float:
+    """Eq. 4: root mean square of a layer's weight-gradient entries (fp32 in, double out)."""
+    w = np.ascontiguousarray(dw, dtype=np.float32).reshape(-1)
+    return float(_load().oracle_gradient_importance(_ptr(w), int(w.size)))
 
 
 def n_keep(n: int, ratio: float) -> int:

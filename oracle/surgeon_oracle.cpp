@@ -98,6 +98,57 @@ int oracle_layer_ratios(const double* G, const double* m, int l, double* p) {
   return 0;
 }
 
+// Eq. 4: Gradient Importance of one layer, G = sqrt( sum_j (dw_j)^2 / N ), the root mean square
+// of the layer's N weight-gradient entries.  One pass in index order, squares and sum in double.
+// N = 0 has no mean: returns 0.
+double oracle_gradient_importance(const float* dw, int64_t n) {
+  if (n <= 0) return 0.0;
+  double sum = 0.0;
+  for (int64_t j = 0; j < n; ++j) {
+    const double v = static_cast<double>(dw[j]);
+    sum += v * v;
+  }
+  return std::sqrt(sum / static_cast<double>(n));
+}
+
+// The ratio rule with one factor of Eq. 6 left out, as in the paper's ablation (Section 5.3,
+// the table of strategies), and the global static ratio it is compared with (Section 5.3,
+// "global static sparsity").  The paper names the variants without formulas; the reading is:
+//   rule 0  "Ours"    I_i = Norm(M_i) * Norm(G_i)        (Eq. 6 as printed)
+//   rule 1  "w/o G"   I_i = Norm(M_i)                    (the gradient factor replaced by 1)
+//   rule 2  "w/o M"   I_i = Norm(G_i)                    (the memory factor replaced by 1)
+//   rule 3  static    p_i = p_static for every layer     (no importance at all)
+// followed by Eq. 7 unchanged for rules 0-2.  Returns 0, or 3 when max_j I_j is zero.
+int oracle_layer_ratios_rule(const double* G, const double* m, int l, int rule, double p_static,
+                             double* p) {
+  if (rule == 3) {
+    for (int i = 0; i < l; ++i) p[i] = p_static;
+    return 0;
+  }
+  double total = 0.0;
+  for (int i = 0; i < l; ++i) total += m[i];
+  std::vector<double> M(l), I(l);
+  for (int i = 0; i < l; ++i) M[i] = -std::log(m[i] / total);
+  double maxM = 0.0, maxG = 0.0;
+  for (int i = 0; i < l; ++i) {
+    maxM = std::max(maxM, M[i]);
+    maxG = std::max(maxG, G[i]);
+  }
+  double maxI = 0.0;
+  for (int i = 0; i < l; ++i) {
+    const double normM = (rule == 2) ? 1.0 : ((maxM > 0.0) ? M[i] / maxM : 0.0);
+    const double normG = (rule == 1) ? 1.0 : ((maxG > 0.0) ? G[i] / maxG : 0.0);
+    I[i] = normM * normG;
+    maxI = std::max(maxI, I[i]);
+  }
+  if (!(maxI > 0.0)) {
+    for (int i = 0; i < l; ++i) p[i] = 0.0;
+    return 3;
+  }
+  for (int i = 0; i < l; ++i) p[i] = 1.0 - I[i] / maxI;
+  return 0;
+}
+
 // Algorithm 1: prune step: how many elements "ratio p" removes.  The paper does not state the
 // rounding; the reading is n_prune = floor(p*n) with the product taken once in double, and
 // the kept count is what remains.
