@@ -70,6 +70,42 @@ surgeon_status surgeon_layer_ratios(const double* gi, const double* lam, int32_t
                                     double* ratios_out);
 
 /* ------------------------------------------------------------------------------------------
+ * Section 5.3 (the ablation's strategies) and the global static ratio it is compared with: the
+ * rule of Eq. 5-7 with one factor of Eq. 6 left out.  The paper names the variants without
+ * formulas; here the missing factor is 1 and Eq. 7 is unchanged:
+ *   SURGEON_RULE_BOTH         I_i = Norm(M_i) * Norm(G_i)   (= surgeon_layer_ratios)
+ *   SURGEON_RULE_NO_GRADIENT  I_i = Norm(M_i)               ("w/o G"; gi may be NULL)
+ *   SURGEON_RULE_NO_MEMORY    I_i = Norm(G_i)               ("w/o M"; lam may be NULL)
+ *   SURGEON_RULE_STATIC       p_i = static_ratio            (gi and lam may be NULL)
+ * Arguments, units and errors as for surgeon_layer_ratios; static_ratio outside [0,1] or an
+ * unknown rule is INVALID_ARG.
+ * ---------------------------------------------------------------------------------------- */
+typedef enum {
+  SURGEON_RULE_BOTH = 0,
+  SURGEON_RULE_NO_GRADIENT = 1,
+  SURGEON_RULE_NO_MEMORY = 2,
+  SURGEON_RULE_STATIC = 3
+} surgeon_ratio_rule;
+surgeon_status surgeon_layer_ratios_rule(const double* gi, const double* lam, int32_t n_layers,
+                                         surgeon_ratio_rule rule, double static_ratio,
+                                         double* ratios_out);
+
+/* ------------------------------------------------------------------------------------------
+ * Eq. 4: Gradient Importance of one layer, G = sqrt( sum_j (dw_j)^2 / N ): the root mean square
+ * of the N entries of the layer's weight gradient, the G_i that surgeon_layer_ratios takes.
+ * dw: DEVICE pointer to n_weights fp32 values (as written by surgeon_weight_grad).  gi_out:
+ * DEVICE pointer to one double.  workspace: DEVICE scratch of at least
+ * SURGEON_GI_WORKSPACE_BYTES bytes, 8-byte aligned, owned by the caller, not shared with a call
+ * in flight.  Squares and sums are taken in double, in a fixed order, so the result is bitwise
+ * reproducible.  n_weights = 0 gives 0.  Asynchronous on cuda_stream.
+ * Errors: INVALID_ARG (null pointer, n_weights < 0), BUFFER_TOO_SMALL, CUDA.
+ * ---------------------------------------------------------------------------------------- */
+#define SURGEON_GI_WORKSPACE_BYTES 8192
+surgeon_status surgeon_gradient_importance(const float* dw, int64_t n_weights, double* gi_out,
+                                           void* workspace, size_t workspace_bytes,
+                                           void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * Algorithm 1: prune step ("prune A_i with ratio p"): the kept count and the buffer sizes.
  * Pure host arithmetic.  n_prune = floor(ratio * n) evaluated in IEEE double, n_keep = n -
  * n_prune.  Any out pointer may be NULL.  bitmap_bytes = 4*ceil(n/32); values_bytes =

@@ -66,6 +66,12 @@ def lib():
         l = C.CDLL(LIB_PATH)
         l.surgeon_layer_ratios.restype = C.c_int
         l.surgeon_layer_ratios.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        l.surgeon_layer_ratios_rule.restype = C.c_int
+        l.surgeon_layer_ratios_rule.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int, C.c_double,
+                                                C.c_void_p]
+        l.surgeon_gradient_importance.restype = C.c_int
+        l.surgeon_gradient_importance.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p,
+                                                  C.c_size_t, C.c_void_p]
         l.surgeon_compact_sizes.restype = C.c_int
         l.surgeon_compact_sizes.argtypes = [C.c_int64, C.c_int, C.c_double, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_void_p, C.c_void_p]
@@ -131,6 +137,45 @@ def surgeon_layer_ratios(gi, lam, allow_degenerate: bool = False) -> np.ndarray:
     out = np.empty_like(g)
     st = lib().surgeon_layer_ratios(g.ctypes.data, m.ctypes.data, int(g.size), out.ctypes.data)
     _check(st, "surgeon_layer_ratios", allow=(SURGEON_ERR_DEGENERATE,) if allow_degenerate else ())
+    return out
+
+
+SURGEON_RULE_BOTH, SURGEON_RULE_NO_GRADIENT, SURGEON_RULE_NO_MEMORY, SURGEON_RULE_STATIC = 0, 1, 2, 3
+SURGEON_GI_WORKSPACE_BYTES = 8192
+
+
+def surgeon_layer_ratios_rule(gi, lam, rule: int, static_ratio: float = 0.0,
+                              allow_degenerate: bool = False) -> np.ndarray:
+    """The ratio rule with one factor left out ("w/o G", "w/o M") or a global static ratio."""
+    g = None if gi is None else np.ascontiguousarray(gi, dtype=np.float64)
+    m = None if lam is None else np.ascontiguousarray(lam, dtype=np.float64)
+    ref = g if g is not None else m
+    if ref is None or ref.ndim != 1 or (g is not None and m is not None and g.shape != m.shape):
+        raise ValueError("gi and lam must be 1-D and of equal length (one of them may be None)")
+    out = np.empty(ref.shape, dtype=np.float64)
+    st = lib().surgeon_layer_ratios_rule(None if g is None else g.ctypes.data,
+                                         None if m is None else m.ctypes.data, int(ref.size),
+                                         int(rule), float(static_ratio), out.ctypes.data)
+    _check(st, "surgeon_layer_ratios_rule",
+           allow=(SURGEON_ERR_DEGENERATE,) if allow_degenerate else ())
+    return out
+
+
+def surgeon_gradient_importance(dw: torch.Tensor, out: Optional[torch.Tensor] = None,
+                                workspace: Optional[torch.Tensor] = None,
+                                stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Eq. 4 on the device: a one-element float64 tensor holding sqrt(mean(dw^2))."""
+    if not dw.is_cuda or not dw.is_contiguous() or dw.dtype != torch.float32:
+        raise ValueError("dw must be a contiguous fp32 CUDA tensor")
+    if out is None:
+        out = torch.empty(1, dtype=torch.float64, device=dw.device)
+    if workspace is None:
+        workspace = torch.empty(SURGEON_GI_WORKSPACE_BYTES, dtype=torch.uint8, device=dw.device)
+    st = lib().surgeon_gradient_importance(dw.data_ptr() if dw.numel() else None, dw.numel(),
+                                           out.data_ptr(), workspace.data_ptr(),
+                                           workspace.numel() * workspace.element_size(),
+                                           _stream_ptr(stream))
+    _check(st, "surgeon_gradient_importance")
     return out
 
 

@@ -113,6 +113,49 @@ surgeon_status surgeon_layer_ratios(const double* gi, const double* lam, int32_t
   return SURGEON_OK;
 }
 
+surgeon_status surgeon_layer_ratios_rule(const double* gi, const double* lam, int32_t n_layers,
+                                         surgeon_ratio_rule rule, double static_ratio,
+                                         double* ratios_out) {
+  if (!ratios_out || n_layers <= 0) return SURGEON_ERR_INVALID_ARG;
+  if (rule == SURGEON_RULE_BOTH) return surgeon_layer_ratios(gi, lam, n_layers, ratios_out);
+  if (rule == SURGEON_RULE_STATIC) {
+    if (!(static_ratio >= 0.0 && static_ratio <= 1.0)) return SURGEON_ERR_INVALID_ARG;
+    for (int i = 0; i < n_layers; ++i) ratios_out[i] = static_ratio;
+    return SURGEON_OK;
+  }
+  double i_max = 0.0;
+  if (rule == SURGEON_RULE_NO_GRADIENT) {
+    // Eq. 5, then Eq. 6 with the gradient factor taken as 1: I_i = M_i / max M
+    if (!lam) return SURGEON_ERR_INVALID_ARG;
+    double total = 0.0;
+    for (int i = 0; i < n_layers; ++i) {
+      if (!isfinite(lam[i]) || !(lam[i] > 0.0)) return SURGEON_ERR_INVALID_ARG;
+      total += lam[i];
+    }
+    for (int i = 0; i < n_layers; ++i) {
+      ratios_out[i] = -log(lam[i] / total);
+      if (ratios_out[i] > i_max) i_max = ratios_out[i];
+    }
+  } else if (rule == SURGEON_RULE_NO_MEMORY) {
+    // Eq. 6 with the memory factor taken as 1: I_i = G_i / max G
+    if (!gi) return SURGEON_ERR_INVALID_ARG;
+    for (int i = 0; i < n_layers; ++i) {
+      if (!isfinite(gi[i]) || gi[i] < 0.0) return SURGEON_ERR_INVALID_ARG;
+      ratios_out[i] = gi[i];
+      if (gi[i] > i_max) i_max = gi[i];
+    }
+  } else {
+    return SURGEON_ERR_INVALID_ARG;
+  }
+  if (!(i_max > 0.0)) {
+    for (int i = 0; i < n_layers; ++i) ratios_out[i] = 0.0;
+    return SURGEON_ERR_DEGENERATE;
+  }
+  // Eq. 7 (the inner normalisation cancels against the outer one)
+  for (int i = 0; i < n_layers; ++i) ratios_out[i] = 1.0 - ratios_out[i] / i_max;
+  return SURGEON_OK;
+}
+
 surgeon_status surgeon_compact_sizes(int64_t n, surgeon_dtype dt, double ratio, int64_t* n_keep,
                                      size_t* bitmap_bytes, size_t* values_bytes,
                                      size_t* offsets_bytes, size_t* workspace_bytes) {
@@ -188,6 +231,19 @@ surgeon_status surgeon_decompress(const surgeon_compressed* act, void* x_out, vo
       !aligned16(act->block_offsets))
     return SURGEON_ERR_INVALID_ARG;
   const cudaError_t e = launch_decompress(*act, x_out, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? SURGEON_OK : SURGEON_ERR_CUDA;
+}
+
+surgeon_status surgeon_gradient_importance(const float* dw, int64_t n_weights, double* gi_out,
+                                           void* workspace, size_t workspace_bytes,
+                                           void* cuda_stream) {
+  if (!gi_out || !workspace || n_weights < 0 || (n_weights > 0 && !dw)) return SURGEON_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 7u) || (reinterpret_cast<uintptr_t>(gi_out) & 7u) ||
+      (reinterpret_cast<uintptr_t>(dw) & 3u))
+    return SURGEON_ERR_INVALID_ARG;
+  if (workspace_bytes < SURGEON_GI_WORKSPACE_BYTES) return SURGEON_ERR_BUFFER_TOO_SMALL;
+  const cudaError_t e = launch_gradient_importance(dw, n_weights, gi_out, workspace,
+                                                   static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SURGEON_OK : SURGEON_ERR_CUDA;
 }
 

@@ -101,6 +101,9 @@ cudaError_t launch_prune_compact(const void* x, int64_t n, int dt, int64_t k,
                                  const surgeon_compressed& out, void* workspace,
                                  cudaStream_t stream);
 cudaError_t launch_decompress(const surgeon_compressed& act, void* x_out, cudaStream_t stream);
+// Eq. 4 on device: *gi_out = sqrt(sum dw^2 / n); workspace = SURGEON_GI_WORKSPACE_BYTES of scratch.
+cudaError_t launch_gradient_importance(const float* dw, long long n, double* gi_out,
+                                       void* workspace, cudaStream_t stream);
 
 size_t weight_grad_fp32_workspace(const surgeon_layer_desc& d);
 cudaError_t launch_weight_grad_fp32(const surgeon_compressed& act, const surgeon_layer_desc& d,

@@ -26,7 +26,8 @@ def test_exports_every_declared_symbol():
     names = set(re.findall(r"\b(surgeon_[a-z_0-9]+)\s*\(", text))
     assert {"surgeon_layer_ratios", "surgeon_compact_sizes", "surgeon_prune_compact",
             "surgeon_weight_grad", "surgeon_weight_grad_workspace", "surgeon_decompress",
-            "surgeon_status_string"} <= names
+            "surgeon_status_string", "surgeon_layer_ratios_rule",
+            "surgeon_gradient_importance"} <= names
     l = ctypes.CDLL(B.LIB_PATH)
     for n in names:
         assert hasattr(l, n), n
@@ -60,6 +61,30 @@ def test_ratios_errors():
         with pytest.raises(B.SurgeonError) as e:
             B.surgeon_layer_ratios(gi, lam)
         assert e.value.status == B.SURGEON_ERR_INVALID_ARG
+
+
+def test_ratio_rule_variants_match_oracle():
+    for layers in (W.wrn28_10(), W.resnet50(), W.vit_b16()):
+        gi = W.gradient_importance(len(layers), seed=1)
+        lam = np.array([l.act_bytes for l in layers], dtype=np.float64)
+        for rule in (oracle.RULE_BOTH, oracle.RULE_NO_GRADIENT, oracle.RULE_NO_MEMORY):
+            _, ref = oracle.layer_ratios_rule(gi, lam, rule)
+            np.testing.assert_allclose(B.surgeon_layer_ratios_rule(gi, lam, rule), ref, rtol=0, atol=1e-14)
+        _, ref = oracle.layer_ratios_rule(gi, lam, oracle.RULE_STATIC, 0.9)
+        assert np.array_equal(B.surgeon_layer_ratios_rule(gi, lam, B.SURGEON_RULE_STATIC, 0.9), ref)
+    # the factor that is left out need not be passed
+    np.testing.assert_allclose(B.surgeon_layer_ratios_rule(None, [8, 4, 2, 2], B.SURGEON_RULE_NO_GRADIENT),
+                               [2 / 3, 1 / 3, 0, 0], rtol=0, atol=1e-12)
+    np.testing.assert_allclose(B.surgeon_layer_ratios_rule([3, 3, 1, 2], None, B.SURGEON_RULE_NO_MEMORY),
+                               [0, 0, 2 / 3, 1 / 3], rtol=0, atol=1e-15)
+    for args in (([1.0, 2.0], [1.0, 1.0], 7, 0.0), ([1.0, 2.0], [1.0, 1.0], B.SURGEON_RULE_STATIC, 1.5),
+                 (None, [1.0, 1.0], B.SURGEON_RULE_NO_MEMORY, 0.0), ([1.0, -2.0], None, B.SURGEON_RULE_NO_MEMORY, 0.0)):
+        with pytest.raises(B.SurgeonError) as e:
+            B.surgeon_layer_ratios_rule(*args)
+        assert e.value.status == B.SURGEON_ERR_INVALID_ARG
+    with pytest.raises(B.SurgeonError) as e:
+        B.surgeon_layer_ratios_rule([0.0, 0.0], None, B.SURGEON_RULE_NO_MEMORY)
+    assert e.value.status == B.SURGEON_ERR_DEGENERATE
 
 
 def test_compact_sizes_match_oracle_kept_count():
