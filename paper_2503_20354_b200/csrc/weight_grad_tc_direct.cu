@@ -266,7 +266,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
       }
       for (int it = wg; it < n_kt; it += kGroups) {
         if (!wait_stage()) break;
-        if (PAIR) fence_proxy_async_all(); else fence_proxy_async();
+        fence_proxy_async();
         __syncwarp();
         if (lane == 0) { if (PAIR) mbar_arrive_rank0(full_a + 8 * sa); else mbar_arrive(full_a + 8 * sa); }
         next_stage();
@@ -337,7 +337,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
           }
           b0 += seg; left -= seg; ox = 0; ++oy;
         }
-        if (PAIR) fence_proxy_async_all(); else fence_proxy_async();
+        fence_proxy_async();
         __syncwarp();
         if (lane == 0) { if (PAIR) mbar_arrive_rank0(full_a + 8 * sa); else mbar_arrive(full_a + 8 * sa); }
         next_stage();
@@ -448,7 +448,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
 #pragma unroll
         for (int q = 0; q < 4; ++q)
           *reinterpret_cast<uint4*>(dst_row + (((y + q) ^ xr) << 4)) = chunk[q];
-        if (PAIR) fence_proxy_async_all(); else fence_proxy_async();
+        fence_proxy_async();
         __syncwarp();
         if (lane == 0) { if (PAIR) mbar_arrive_rank0(full_a + 8 * sa); else mbar_arrive(full_a + 8 * sa); }
         next_stage();
