@@ -683,7 +683,9 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   // tiles as fit (up to 8)
   const int budget = 224 * 1024 - 1024;
   const int b_bytes = p.n_cols * (p.pair ? 64 : 128);
-  int b_stages = (3 * b_bytes + 4 * kATileBytes <= budget) ? 3 : 2;
+  int b_stages = (budget - 4 * kATileBytes) / b_bytes;     // room for four activation tiles at least
+  if (b_stages > kMaxBStages) b_stages = kMaxBStages;
+  if (b_stages < 2) b_stages = 2;
   if (b_stages * b_bytes + 2 * kATileBytes > budget) return false;
   int a_stages = (budget - b_stages * b_bytes) / kATileBytes;
   if (a_stages > kMaxAStages) a_stages = kMaxAStages;
