@@ -168,11 +168,30 @@ def decompress(bitmap: np.ndarray, values: np.ndarray, n: int) -> np.ndarray:
     return out
 
 
-def prune_compact(x: np.ndarray, ratio: float, method: int = 1, block: int = BLOCK):
-    """Algorithm 1: prune and decompose steps in one call: dict with tau, k, c_gt, q, keep, bitmap, values, offsets."""
+def magnitude_keys(x: np.ndarray) -> np.ndarray:
+    """The bit pattern of every element with the sign bit cleared (0 for +0 and -0)."""
+    x = np.ascontiguousarray(x).reshape(-1)
+    return (x.view(np.uint32) & np.uint32(0x7FFFFFFF)) if _dt_of(x) == 0 else \
+        (x.view(np.uint16) & np.uint16(0x7FFF)).astype(np.uint32)
+
+
+def prune_compact(x: np.ndarray, ratio: float, method: int = 1, block: int = BLOCK,
+                  drop_zeros: bool = False):
+    """Algorithm 1: prune and decompose steps in one call: dict with tau, k, c_gt, q, keep, bitmap, values, offsets.
+
+    drop_zeros: the store variant that does not spend a value on a kept element that is exactly
+    zero (Algorithm 1's decompose step caches "non-zero values"): the selection is the same, then
+    the zeros among the kept elements are taken out again.  The dense tensor it stands for is
+    unchanged, so is every weight gradient; k becomes the number of stored values."""
     x = np.ascontiguousarray(x).reshape(-1)
     k = n_keep(x.size, ratio)
     keep, tau, cgt, q = select(x, k, method)
+    if drop_zeros:
+        keep = keep.copy()
+        keep[magnitude_keys(x) == 0] = 0
+        k = int(keep.sum(dtype=np.int64))
+        if tau == 0:
+            q = 0
     bitmap, values, offsets = compact(x, keep, block)
     return dict(k=k, tau=tau, c_gt=cgt, q=q, keep=keep, bitmap=bitmap, values=values,
                 offsets=offsets)

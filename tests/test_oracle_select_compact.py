@@ -187,3 +187,33 @@ def test_config1_kept_counts_and_zero_threshold():
         assert r["k"] == k == int(r["keep"].sum())
         if ratio == 0.3:   # k exceeds the ~50 % non-zeros: threshold key 0, kept zeros by index
             assert r["tau"] == 0 and r["q"] > 0
+
+
+def test_drop_zeros_variant():
+    """The store that spends no value on kept zeros: a hand-worked case, the unchanged dense tensor,
+    and equality with the plain store when nothing kept is zero."""
+    x = np.array([0.0, 3.0, -0.0, -1.0, 2.0, 0.0], dtype=np.float32)
+    # ratio 1/6 removes one element: the kept five are 3, 2, -1 and the zeros at 0 and 2 (lowest indices)
+    a = oracle.prune_compact(x, 1.0 / 6.0)
+    assert a["k"] == 5 and a["bitmap"].tolist() == [0b011111]
+    b = oracle.prune_compact(x, 1.0 / 6.0, drop_zeros=True)
+    assert b["k"] == 3 and b["bitmap"].tolist() == [0b011010]
+    assert b["values"].tolist() == [3.0, -1.0, 2.0] and b["offsets"].tolist() == [0, 3]
+    rng = np.random.default_rng(8)
+    for dt in (np.float32, "bf16"):
+        r = np.maximum(rng.standard_normal(5000), 0).astype(np.float32)           # half zeros
+        xx = r if dt is np.float32 else (r.view(np.uint32) >> 16).astype(np.uint16)
+        for ratio in (0.0, 0.3, 0.6):
+            a = oracle.prune_compact(xx, ratio)
+            b = oracle.prune_compact(xx, ratio, drop_zeros=True)
+            da = oracle.decompress(a["bitmap"], a["values"], xx.size)
+            db = oracle.decompress(b["bitmap"], b["values"], xx.size)
+            assert np.array_equal(da, db)                                          # same dense tensor
+            keys = oracle.magnitude_keys(xx)
+            assert b["k"] == int(((a["keep"] == 1) & (keys != 0)).sum()) == b["values"].size
+            assert not (oracle.magnitude_keys(b["values"]) == 0).any()
+            assert b["offsets"][-1] == b["k"]
+        pos = xx[keys != 0]
+        a = oracle.prune_compact(pos, 0.4)
+        b = oracle.prune_compact(pos, 0.4, drop_zeros=True)
+        assert np.array_equal(a["bitmap"], b["bitmap"]) and np.array_equal(a["values"], b["values"])
