@@ -162,6 +162,20 @@ surgeon_status surgeon_prune_compact(const void* x, int64_t n, surgeon_dtype dt,
                                      size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Algorithm 1, decompose step ("the non-zero values ... and a 1-bit index"): the same call with
+ * store options.  SURGEON_STORE_DROP_ZEROS: the selection is unchanged, but a kept element that
+ * is exactly zero (+0 or -0; post-ReLU data at a low ratio has many) gets no bit and no value.
+ * The dense tensor the store stands for, and every weight gradient computed from it, are the
+ * same; header->n_keep and the last block offset then give the number of STORED values, which is
+ * at most the count surgeon_compact_sizes reports (size the buffers from that).  flags = 0 is
+ * surgeon_prune_compact.  Unknown flag bits: INVALID_ARG.
+ * ---------------------------------------------------------------------------------------- */
+#define SURGEON_STORE_DROP_ZEROS 1u
+surgeon_status surgeon_prune_compact_flags(const void* x, int64_t n, surgeon_dtype dt, double ratio,
+                                           uint32_t flags, surgeon_compressed* out, void* workspace,
+                                           size_t workspace_bytes, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * No counterpart in the paper: surgeon_prune_compact for callers that cannot allocate device
  * memory.  A hook that runs while the framework's allocator is locked or its pool is frozen, a
  * plug-in behind an interface that forbids cudaMalloc, or a process that gave away its whole

@@ -78,6 +78,9 @@ def lib():
         l.surgeon_prune_compact.restype = C.c_int
         l.surgeon_prune_compact.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_double,
                                             C.POINTER(Compressed), C.c_void_p, C.c_size_t, C.c_void_p]
+        l.surgeon_prune_compact_flags.restype = C.c_int
+        l.surgeon_prune_compact_flags.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_double, C.c_uint32,
+                                                  C.POINTER(Compressed), C.c_void_p, C.c_size_t, C.c_void_p]
         l.surgeon_prune_compact_static.restype = C.c_int
         l.surgeon_prune_compact_static.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_double,
                                                    C.POINTER(Compressed), C.c_void_p]
@@ -233,16 +236,23 @@ class CompressedActivation:
         """Host copies for comparison: (bitmap uint32, values, offsets uint32, Header)."""
         nw = (self.n + 31) // 32
         bitmap = self.bitmap[:nw].cpu().numpy().view(np.uint32)
-        vals = self.values[: self.n_keep].cpu()
+        hdr = self.read_header()
+        vals = self.values[: int(hdr.n_keep)].cpu()    # the stored count (= n_keep unless zeros are dropped)
         vals = vals.view(torch.int16).numpy().view(np.uint16) if self.dt == SURGEON_BF16 else vals.numpy()
         offs = self.block_offsets[: self.sizes.offsets_bytes // 4].cpu().numpy().view(np.uint32)
-        return bitmap, vals, offs, self.read_header()
+        return bitmap, vals, offs, hdr
+
+
+SURGEON_STORE_DROP_ZEROS = 1
 
 
 def surgeon_prune_compact(x: torch.Tensor, ratio: float, out: Optional[CompressedActivation] = None,
                           workspace: Optional[torch.Tensor] = None,
-                          stream: Optional[torch.cuda.Stream] = None) -> CompressedActivation:
-    """Prune ``x`` (CUDA tensor, fp32 or bf16, contiguous) at ``ratio`` into a compressed store."""
+                          stream: Optional[torch.cuda.Stream] = None,
+                          flags: int = 0) -> CompressedActivation:
+    """Prune ``x`` (CUDA tensor, fp32 or bf16, contiguous) at ``ratio`` into a compressed store.
+    ``flags=SURGEON_STORE_DROP_ZEROS``: kept zeros get no bit and no value (the header's n_keep
+    is then the stored count; ``out.sizes.n_keep`` stays the upper bound the buffers are sized for)."""
     if not x.is_cuda or not x.is_contiguous():
         raise ValueError("x must be a contiguous CUDA tensor")
     dt = dtype_code(x.dtype)
@@ -256,9 +266,10 @@ def surgeon_prune_compact(x: torch.Tensor, ratio: float, out: Optional[Compresse
         out.ratio, out.sizes = float(ratio), sizes
     if workspace is None:
         workspace = torch.empty(sizes.workspace_bytes, dtype=torch.uint8, device=x.device)
-    st = lib().surgeon_prune_compact(x.data_ptr(), n, dt, float(ratio), C.byref(out.c),
-                                     workspace.data_ptr(), workspace.numel() * workspace.element_size(),
-                                     _stream_ptr(stream))
+    st = lib().surgeon_prune_compact_flags(x.data_ptr(), n, dt, float(ratio), int(flags), C.byref(out.c),
+                                           workspace.data_ptr(),
+                                           workspace.numel() * workspace.element_size(),
+                                           _stream_ptr(stream))
     _check(st, "surgeon_prune_compact")
     return out
 

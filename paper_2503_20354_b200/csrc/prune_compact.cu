@@ -268,7 +268,8 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
                 long long n_rows_full, uint32_t k, SelectState* __restrict__ st,
                 uint32_t* __restrict__ hist_a, uint32_t* __restrict__ cnt_gt,
                 uint32_t* __restrict__ cand_cnt, void* __restrict__ slots_v,
-                surgeon_header* __restrict__ hdr, int n_chunks, int n_stage_tiles) {
+                surgeon_header* __restrict__ hdr, int n_chunks, int n_stage_tiles,
+                int drop_zeros) {
   using E = typename Elem<DT>::type;
   constexpr uint32_t kMask = Elem<DT>::kKeyMask;
   constexpr int EPR = 128 / sizeof(E);
@@ -475,11 +476,13 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
   }
   if (lane == 0) {
     if (mode == 2) {
+      // store variant without kept zeros: a threshold of key 0 keeps the non-zero elements only
+      const bool nz = drop_zeros && tau == 0u;
       hdr->threshold_key = tau;
       hdr->status = __ldcg(&st->error);
-      hdr->n_keep = k;
+      hdr->n_keep = nz ? static_cast<long long>(n_greater) : static_cast<long long>(k);
       hdr->n_greater = n_greater;
-      hdr->tie_quota = static_cast<long long>(k) - n_greater;
+      hdr->tie_quota = nz ? 0 : static_cast<long long>(k) - n_greater;
     }
     st->mode = mode;
     __threadfence();
@@ -573,7 +576,7 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
              unsigned long long* __restrict__ val, unsigned long long* __restrict__ prefix,
              unsigned long long* __restrict__ partial, int tiles,
              uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
-             uint32_t* __restrict__ offsets) {
+             uint32_t* __restrict__ offsets, int drop_zeros) {
   using E = typename Elem<DT>::type;
   constexpr uint32_t kMask = Elem<DT>::kKeyMask;
   constexpr int EPV = 16 / sizeof(E);
@@ -672,15 +675,16 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
   } else {
     tau = hdr->threshold_key;
   }
+  const bool nz = drop_zeros && tau == 0u;       // store variant without kept zeros (see classify_kernel)
   if (mode != 2u && blockIdx.x == 0 && tid == 0) {
     hdr->threshold_key = tau;
     hdr->status = __ldcg(&st->error);
-    hdr->n_keep = k;
+    hdr->n_keep = nz ? static_cast<long long>(n_greater) : static_cast<long long>(k);
     hdr->n_greater = n_greater;
-    hdr->tie_quota = static_cast<long long>(k) - n_greater;
+    hdr->tie_quota = nz ? 0 : static_cast<long long>(k) - n_greater;
   }
 
-  const long long quota = (mode == 2u) ? hdr->tie_quota : static_cast<long long>(k) - n_greater;
+  const long long quota = (mode == 2u) ? hdr->tie_quota : (nz ? 0 : static_cast<long long>(k) - n_greater);
 
   // ---- per-chunk values; CTA b owns the chunks [b*per, (b+1)*per) ----
   const int per = (tiles + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
@@ -801,7 +805,9 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
     // the CTA that owns the last chunk also writes the totals and checks them
     __syncthreads();
     if (tid == 0) {
-      offsets[(n + SURGEON_BLOCK - 1) >> kBlockShift] = k;     // the sentinel entry of the block offsets
+      // the sentinel entry of the block offsets = the number of stored values
+      offsets[(n + SURGEON_BLOCK - 1) >> kBlockShift] =
+          nz ? static_cast<uint32_t>((mode == 2u) ? hdr->n_greater : n_greater) : k;
       unsigned long long total = 0;
       for (int b = 0; b <= static_cast<int>(blockIdx.x); ++b) total += __ldcg(partial + b);
       prefix[tiles] = total;
@@ -1284,7 +1290,7 @@ bool make_row_map(const void* x, long long n_rows_full, CUtensorMap* map) {
 }
 
 template <int DT>
-cudaError_t run_prune_compact(const void* x, long long n, long long k,
+cudaError_t run_prune_compact(const void* x, long long n, long long k, int drop_zeros,
                               const surgeon_compressed& out, void* workspace,
                               cudaStream_t stream) {
   using E = typename Elem<DT>::type;
@@ -1350,7 +1356,7 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
           static_cast<uint32_t>(n_seg), static_cast<uint32_t>(seg_stride), st, hist_s);
       classify_kernel<DT><<<stream_grid, kCsThreads, kCsSmem, stream>>>(
           map, x, n, n_rows_full, static_cast<uint32_t>(k), st, hist_a, cnt_gt, cand_cnt, slots,
-          out.header, n_chunks, n_stage_tiles);
+          out.header, n_chunks, n_stage_tiles, drop_zeros);
       note_launches(2);
     } else {
       // small tensor: straight to the fall-back select (mode = 1; the state is little-endian)
@@ -1374,7 +1380,7 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
       void* vals = out.values;
       uint32_t* offs = out.block_offsets;
       void* args[] = {&xa, &na, &ka, &st, &hdr, &hist_b, &hist_fb, &cg, &cc, &sl, &val, &prefix,
-                      &partial, &tiles, &bm, &vals, &offs};
+                      &partial, &tiles, &bm, &vals, &offs, &drop_zeros};
       e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(count_kernel<DT>), dim3(grid),
                                       dim3(kSelThreads), args, 0, stream);
       if (e != cudaSuccess) return e;
@@ -1401,9 +1407,9 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k,
 
 cudaError_t launch_prune_compact(const void* x, int64_t n, int dt, int64_t k,
                                  const surgeon_compressed& out, void* workspace,
-                                 cudaStream_t stream) {
-  return dt == 0 ? run_prune_compact<0>(x, n, k, out, workspace, stream)
-                 : run_prune_compact<1>(x, n, k, out, workspace, stream);
+                                 cudaStream_t stream, int drop_zeros) {
+  return dt == 0 ? run_prune_compact<0>(x, n, k, drop_zeros, out, workspace, stream)
+                 : run_prune_compact<1>(x, n, k, drop_zeros, out, workspace, stream);
 }
 
 cudaError_t launch_decompress(const surgeon_compressed& act, void* x_out, cudaStream_t stream) {

@@ -58,6 +58,39 @@ def test_distributions_and_ratios(dist, bf16):
 
 
 @pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("n", [1000, 65536 + 7, 300000, (1 << 22) + 77])
+def test_store_without_kept_zeros(n, bf16):
+    """SURGEON_STORE_DROP_ZEROS: bit-exact with the oracle's variant; at ratios that keep more than
+    the non-zero half of post-ReLU data the threshold key is 0 and the zeros are left out."""
+    x = _as(W.draw("relu_normal", n, seed=6, tag=n), bf16)
+    for ratio in (0.0, 0.3, 0.45, 0.6, 1.0):
+        comp, ref = assert_store_equals_oracle(x, ratio, drop_zeros=True, method=0 if n < 5000 else 1)
+        if ratio <= 0.45:
+            assert ref["tau"] == 0 and ref["k"] < oracle.n_keep(n, ratio)
+    # the dense tensor is the one of the plain store
+    a = B.surgeon_decompress(B.surgeon_prune_compact(x.cuda(), 0.3)).cpu()
+    b = B.surgeon_decompress(B.surgeon_prune_compact(x.cuda(), 0.3, flags=B.SURGEON_STORE_DROP_ZEROS)).cpu()
+    assert torch.equal(a.float(), b.float())
+    # all zeros: nothing is stored
+    z = torch.zeros(n, dtype=x.dtype)
+    assert_store_equals_oracle(z, 0.25, drop_zeros=True, method=0 if n < 5000 else 1)
+
+
+def test_store_without_kept_zeros_gives_the_same_weight_gradient():
+    layer = W.conv("nz", 4, 72, 16, 96, 3)
+    a = W.activation(layer, 13).cuda()
+    g = W.grad_out(layer, 13).cuda()
+    for path in (B.PATH_FP32, B.PATH_TENSOR_CORE):
+        d = B.layer_desc(layer, path)
+        dw_a = B.surgeon_weight_grad(B.surgeon_prune_compact(a, 0.2), d, g)
+        dw_b = B.surgeon_weight_grad(B.surgeon_prune_compact(a, 0.2, flags=B.SURGEON_STORE_DROP_ZEROS), d, g)
+        assert torch.equal(dw_a, dw_b)
+    with pytest.raises(B.SurgeonError) as e:
+        B.surgeon_prune_compact(a, 0.2, flags=6)
+    assert e.value.status == B.SURGEON_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("bf16", [False, True])
 def test_special_values(bf16):
     x = W.draw("normal", 5000, seed=3)
     x[7] = float("nan"); x[100] = float("inf"); x[101] = -float("inf"); x[9] = -0.0; x[10] = 0.0
