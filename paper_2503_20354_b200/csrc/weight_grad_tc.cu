@@ -690,28 +690,26 @@ reduce_splits_kernel(const float* __restrict__ partial, long long mn, int splits
 }
 
 // The same for a tap-stacked partial [splits][taps * O][C]: dw[o][c][tap] gets row tap * O + o.
-// One block sums 32 input channels of one output channel for all taps: the reads run along c
-// (contiguous in the partial), the writes along (c, tap) (contiguous in dw), transposed through
-// shared memory.  taps <= 49.
+// One block sums `chunk` input channels of one output channel for all taps: the reads
+// run along c (contiguous in the partial, a kilobyte per warp), the writes along (c, tap)
+// (contiguous in dw), transposed through shared memory.  taps <= 49.
 __global__ void __launch_bounds__(256)
 reduce_splits_taps_kernel(const float* __restrict__ partial, int o_real, int c_in, int taps,
-                          int splits, float* __restrict__ dw, int accumulate,
+                          int chunk, int splits, float* __restrict__ dw, int accumulate,
                           const uint32_t* __restrict__ status, surgeon_header* __restrict__ hdr) {
-  __shared__ float tile[32 * 49];
-  const int c0 = blockIdx.x * 32;
+  extern __shared__ float tile[];                  // [n_c][taps]
+  const int c0 = blockIdx.x * chunk;
   const int o = blockIdx.y;
   if (blockIdx.x == 0 && o == 0 && threadIdx.x == 0 && *status != 0 && hdr)
     atomicMax(&hdr->status, *status);
   const long long mn = static_cast<long long>(o_real) * c_in * taps;
-  const int n_c = min(32, c_in - c0);
-  for (int idx = threadIdx.x; idx < 32 * taps; idx += 256) {
-    const int tap = idx >> 5, cl = idx & 31;
-    if (cl < n_c) {
-      const long long src = (static_cast<long long>(tap) * o_real + o) * c_in + c0 + cl;
-      float s = partial[src];
-      for (int z = 1; z < splits; ++z) s += partial[z * mn + src];
-      tile[cl * taps + tap] = s;
-    }
+  const int n_c = min(chunk, c_in - c0);
+  for (int idx = threadIdx.x; idx < n_c * taps; idx += 256) {
+    const int tap = idx / n_c, cl = idx - tap * n_c;     // consecutive threads, consecutive channels
+    const float* src = partial + (static_cast<long long>(tap) * o_real + o) * c_in + c0 + cl;
+    float s = src[0];
+    for (int z = 1; z < splits; ++z) s += src[z * mn];
+    tile[cl * taps + tap] = s;
   }
   __syncthreads();
   float* out = dw + (static_cast<long long>(o) * c_in + c0) * taps;
@@ -850,8 +848,17 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
     if (e != cudaSuccess) return e;
     const long long mn = static_cast<long long>(dp.O) * dp.C;
     if (dp.taps > 1)
-      reduce_splits_taps_kernel<<<dim3((dp.C + 31) / 32, dp.o_real), 256, 0, stream>>>(
-          partial, dp.o_real, dp.C, dp.taps, dp.splits, dw, accumulate, status, act.header);
+    {
+      // the widest chunk of channels (coalescing) that still gives four blocks per SM
+      int chunk = 256;
+      while (chunk > 32 && (static_cast<long long>(dp.o_real) * ((dp.C + chunk - 1) / chunk) < 4LL * sm_count() ||
+                            chunk * dp.taps * 4 > 48 * 1024))
+        chunk >>= 1;
+      reduce_splits_taps_kernel<<<dim3((dp.C + chunk - 1) / chunk, dp.o_real), 256,
+                                  static_cast<size_t>(chunk) * dp.taps * sizeof(float), stream>>>(
+          partial, dp.o_real, dp.C, dp.taps, chunk, dp.splits, dw, accumulate, status, act.header);
+    }
+
     else
       reduce_splits_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
           partial, mn, dp.splits, dw, accumulate, status, act.header);
