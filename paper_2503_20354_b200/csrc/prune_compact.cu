@@ -1190,6 +1190,13 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
       // ---- kept values: gathered in place (packed order), then out as 16-byte vectors ----
       __syncwarp();                                // every lane has its row in registers
       E* outp = reinterpret_cast<E*>(region);
+      // Packed position p lives at swz(p): the 32-bit word index is XORed with the index of its
+      // 128-byte row.  Without it, lanes that keep their whole row (chunks before the end of a
+      // large tie quota, e.g. the zeros of post-ReLU data at a low ratio) all start a multiple
+      // of 32 words apart and every store of the gather is a 32-way bank conflict.
+      auto swz = [](uint32_t p) -> uint32_t {
+        return p ^ ((((p * static_cast<uint32_t>(sizeof(E))) >> 7) & 31u) << (DT == 0 ? 0 : 1));
+      };
       uint32_t pos = lane_pre;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -1197,11 +1204,11 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           if (DT == 0) {
-            if ((word[0] >> (4 * j + i)) & 1u) outp[pos++] = static_cast<E>(c[i]);
+            if ((word[0] >> (4 * j + i)) & 1u) outp[swz(pos++)] = static_cast<E>(c[i]);
           } else {
             const int e = 8 * j + 2 * i;
-            if ((word[e >> 5] >> (e & 31)) & 1u) outp[pos++] = static_cast<E>(c[i] & 0xFFFFu);
-            if ((word[e >> 5] >> ((e + 1) & 31)) & 1u) outp[pos++] = static_cast<E>(c[i] >> 16);
+            if ((word[e >> 5] >> (e & 31)) & 1u) outp[swz(pos++)] = static_cast<E>(c[i] & 0xFFFFu);
+            if ((word[e >> 5] >> ((e + 1) & 31)) & 1u) outp[swz(pos++)] = static_cast<E>(c[i] >> 16);
           }
         }
       }
@@ -1211,22 +1218,22 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
       uint32_t head = mis ? EPV - mis : 0;
       if (head > total) head = total;
       const uint32_t n_vec = (total - head) / EPV;
-      if (lane < head) dst[lane] = outp[lane];
+      if (lane < head) dst[lane] = outp[swz(lane)];
       for (uint32_t v = lane; v < n_vec; v += 32) {
-        const E* src = outp + head + v * EPV;
+        const uint32_t b = head + v * EPV;
         uint4 o;
         if (DT == 0) {
-          o = make_uint4(src[0], src[1], src[2], src[3]);
+          o = make_uint4(outp[swz(b)], outp[swz(b + 1)], outp[swz(b + 2)], outp[swz(b + 3)]);
         } else {
-          o = make_uint4(src[0] | (static_cast<uint32_t>(src[1]) << 16),
-                         src[2] | (static_cast<uint32_t>(src[3]) << 16),
-                         src[4 % EPV] | (static_cast<uint32_t>(src[5 % EPV]) << 16),
-                         src[6 % EPV] | (static_cast<uint32_t>(src[7 % EPV]) << 16));
+          o = make_uint4(outp[swz(b)] | (static_cast<uint32_t>(outp[swz(b + 1)]) << 16),
+                         outp[swz(b + 2)] | (static_cast<uint32_t>(outp[swz(b + 3)]) << 16),
+                         outp[swz(b + 4 % EPV)] | (static_cast<uint32_t>(outp[swz(b + 5 % EPV)]) << 16),
+                         outp[swz(b + 6 % EPV)] | (static_cast<uint32_t>(outp[swz(b + 7 % EPV)]) << 16));
         }
         *reinterpret_cast<uint4*>(dst + head + v * EPV) = o;
       }
       const uint32_t done = head + n_vec * EPV;
-      if (lane < total - done) dst[done + lane] = outp[done + lane];
+      if (lane < total - done) dst[done + lane] = outp[swz(done + lane)];
     }
     tc::fence_proxy_async();     // this warp's writes to the stage precede the next TMA fill
     __syncwarp();
