@@ -60,6 +60,7 @@ struct DirectParams {
   int a_stages, b_stages;   // depth of the activation-tile and gradient-tile rings
   int tmem_cols, smem_bytes;
   long long n_words;        // words of the bitmap (filled by the launcher)
+  const long long* n_keep_ptr;  // device address of the store's count of packed values (launcher)
   unsigned partial_blk;     // index of the bitmap's last block if it is partial, else 0xFFFFFFFF
 };
 bool plan_direct(const surgeon_layer_desc& d, DirectParams* out);

@@ -21,6 +21,7 @@
 // order by the caller.  Every wait is bounded and ends in SURGEON_ERR_TIMEOUT.
 #include <cuda.h>
 
+#include <cstddef>
 #include <cstdlib>
 
 #include "surgeon_internal.cuh"
@@ -52,6 +53,9 @@ static bool use_pairs() {
 constexpr int kMaxAStages = 8;
 constexpr int kMaxBStages = 4;
 constexpr int kATileBytes = kTileM * kTileK * 2;              // 16 KB
+// staging of packed values: per warp 16 rows of 64 + 16 bf16 (conv) or 8 rows of 128 + 16 (linear)
+constexpr int kStageBytesPerWarp = 16 * (64 + 16) * 2;
+constexpr int kStageBytes = kProdWarps * kStageBytesPerWarp;  // 40 KB
 
 // Shared-memory matrix descriptor of an MN-major operand with 128-byte swizzle: rows of 64
 // elements (128 bytes) per k, 8 rows per 1024-byte group (stride byte offset), the next 64
@@ -239,6 +243,9 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
     const uint32_t xr = row & 7;
     const uint32_t y = (MODE == 0) ? (part & 1) * 4 : part * 4;     // first 16-byte chunk of the run
     const uint32_t rowbase = (MODE == 0) ? (part >> 1) * (kTileK * 128) + row * 128 : row * 128;
+    // per-warp staging of the packed values of a tile's rows (after the two rings)
+    unsigned char* stg = b_ring + p.b_stages * b_stage_bytes + pw * kStageBytesPerWarp;
+    const uint32_t n_keep = static_cast<uint32_t>(__ldg(p.n_keep_ptr));   // packed values in the store
     // ring position of this group's tile `it` (= it % a_stages) and how often it has wrapped
     int sa = wg % p.a_stages;
     uint32_t round = wg / p.a_stages;
@@ -418,29 +425,105 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         rank += __popc(w0 & ((1u << sh) - 1u));
         uint32_t bits = __funnelshift_r(w0, w1, sh);
         bits = cur.nvalid >= 32 ? bits : (bits & ((1u << cur.nvalid) - 1u));
-        // The run as four 16-byte chunks of 8 elements: every element is one predicated load (its
-        // place in the packed vector advances with each kept element before it), so the 32 loads
-        // of a lane are independent and nothing is stored twice.
+        // ---- the packed values of the warp's rows -> shared memory, as bf16 ----
+        // The lanes of a row (2 for conv, 4 for linear) hold consecutive runs, so a row's kept
+        // values are one contiguous piece of the packed vector.  The warp copies every piece
+        // with aligned 16-byte loads, lane by lane (coalesced; the lane-per-run loads they
+        // replace touch a cache line per lane and saturate the L1 at low pruning ratios),
+        // converting fp32 to bf16 on the way; each row has its own slot.
+        constexpr int LPR = (MODE == 0) ? 4 : 2;              // lanes per row
+        constexpr int RPW = 32 / LPR;                         // rows per warp
+        constexpr int V = (DT == 0) ? 4 : 8;                  // packed values per 16-byte vector
+        constexpr int VMAX = (32 * LPR + V - 1) / V + 1;      // vectors a row's piece can span
+        constexpr int ITER = (RPW * VMAX + 31) / 32;
+        constexpr int kSlot = 32 * LPR + 16;                  // bf16 values per row slot (piece + alignment slack)
+        const uint32_t cnt = __popc(bits);
         uint4 chunk[4];
+        // Dense tiles of fp32 activations (more than 55 % of the warp's 1024 elements kept) go
+        // through the staging copy; for sparser ones the copy's fixed cost outweighs the
+        // scattered loads it saves, and bf16 values (half as many cache lines per load) never
+        // gain from it, so bf16 launches reserve no staging area.
+        const bool dense = DT == 0 && __reduce_add_sync(0xFFFFFFFFu, cnt) > 560u;
+        if (dense) {
+        uint32_t seg_len = cnt + __shfl_xor_sync(0xFFFFFFFFu, cnt, 1);
+        if (MODE == 0) seg_len += __shfl_xor_sync(0xFFFFFFFFu, seg_len, 2);
+        const uint32_t seg_start = __shfl_sync(0xFFFFFFFFu, rank, lane & ~(LPR - 1));
+        const uint32_t a0 = seg_start & ~static_cast<uint32_t>(V - 1);
+        const uint32_t nvec = seg_len ? (seg_start + seg_len - a0 + V - 1) / V : 0u;
+        __syncwarp();                                         // the previous tile's slot reads are done
+#pragma unroll
+        for (int i = 0; i < ITER; ++i) {
+          const int t = static_cast<int>(lane) + 32 * i;
+          const int r = min(t / VMAX, RPW - 1), v = t - (t / VMAX) * VMAX;
+          const uint32_t a0_r = __shfl_sync(0xFFFFFFFFu, a0, r * LPR);
+          const uint32_t nvec_r = __shfl_sync(0xFFFFFFFFu, nvec, r * LPR);
+          if (t < RPW * VMAX && static_cast<uint32_t>(v) < nvec_r) {
+            const uint32_t first = a0_r + static_cast<uint32_t>(v) * V;
+            unsigned char* dst = stg + r * (kSlot * 2) + v * 16 / (DT == 0 ? 2 : 1);
+            if (DT == 0) {
+              const float* src = reinterpret_cast<const float*>(values) + first;
+              float4 f;
+              if (first + V <= n_keep) f = __ldg(reinterpret_cast<const float4*>(src));
+              else {                                          // the vector that ends past the last value
+                f.x = first < n_keep ? __ldg(src) : 0.0f;
+                f.y = first + 1 < n_keep ? __ldg(src + 1) : 0.0f;
+                f.z = first + 2 < n_keep ? __ldg(src + 2) : 0.0f;
+                f.w = 0.0f;
+              }
+              *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16x2(f.x, f.y), pack_bf16x2(f.z, f.w));
+            } else {
+              const unsigned short* src = reinterpret_cast<const unsigned short*>(values) + first;
+              uint4 u;
+              if (first + V <= n_keep) u = __ldg(reinterpret_cast<const uint4*>(src));
+              else {
+                uint32_t h[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) h[e] = first + e < n_keep ? static_cast<uint32_t>(__ldg(src + e)) : 0u;
+                u = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+              }
+              *reinterpret_cast<uint4*>(dst) = u;
+            }
+          }
+        }
+        __syncwarp();
+        // ---- the run as four 16-byte chunks of 8 elements, read from the row's slot ----
+        const unsigned short* slot = reinterpret_cast<const unsigned short*>(
+            stg + (lane / LPR) * (kSlot * 2)) + (rank - a0);
+        uint32_t k = 0;                                       // kept elements of the run so far
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          const uint32_t byte = (bits >> (8 * q)) & 0xFFu;
-          uint32_t idx = rank + (q == 0 ? 0u : __popc(bits & ((1u << (8 * q)) - 1u)));
           uint32_t v[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
-            const uint32_t on = (byte >> e) & 1u;
-            v[e] = ld_packed<DT>(values, idx, on != 0);
-            idx += on;
+            const uint32_t on = (bits >> (8 * q + e)) & 1u;
+            v[e] = on ? static_cast<uint32_t>(slot[k]) : 0u;
+            k += on;
           }
-          if (DT == 0) {
-            chunk[q].x = pack_bf16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
-            chunk[q].y = pack_bf16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
-            chunk[q].z = pack_bf16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
-            chunk[q].w = pack_bf16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
-          } else {
-            chunk[q].x = v[0] | (v[1] << 16); chunk[q].y = v[2] | (v[3] << 16);
-            chunk[q].z = v[4] | (v[5] << 16); chunk[q].w = v[6] | (v[7] << 16);
+          chunk[q].x = v[0] | (v[1] << 16); chunk[q].y = v[2] | (v[3] << 16);
+          chunk[q].z = v[4] | (v[5] << 16); chunk[q].w = v[6] | (v[7] << 16);
+        }
+        } else {
+          // sparse: one predicated global load per element, all of a lane's loads independent
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t byte = (bits >> (8 * q)) & 0xFFu;
+            uint32_t idx = rank + (q == 0 ? 0u : __popc(bits & ((1u << (8 * q)) - 1u)));
+            uint32_t v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const uint32_t on = (byte >> e) & 1u;
+              v[e] = ld_packed<DT>(values, idx, on != 0);
+              idx += on;
+            }
+            if (DT == 0) {
+              chunk[q].x = pack_bf16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
+              chunk[q].y = pack_bf16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
+              chunk[q].z = pack_bf16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
+              chunk[q].w = pack_bf16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
+            } else {
+              chunk[q].x = v[0] | (v[1] << 16); chunk[q].y = v[2] | (v[3] << 16);
+              chunk[q].z = v[4] | (v[5] << 16); chunk[q].w = v[6] | (v[7] << 16);
+            }
           }
         }
         if (!wait_stage()) break;
@@ -578,6 +661,24 @@ using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, voi
 
 }  // namespace
 
+// Shared memory: the staging area of the packed values (fp32 activations only), the gradient
+// ring (as many tiles as fit beside four activation tiles, up to 4), then as many activation tiles
+// as fit (up to 8).
+static bool size_rings(DirectParams* p, int stage_bytes) {
+  const int budget = 224 * 1024 - 1024 - stage_bytes;
+  const int b_bytes = p->n_cols * (p->pair ? 64 : 128);
+  int b_stages = (budget - 4 * kATileBytes) / b_bytes;
+  if (b_stages > kMaxBStages) b_stages = kMaxBStages;
+  if (b_stages < 2) b_stages = 2;
+  if (b_stages * b_bytes + 2 * kATileBytes > budget) return false;
+  int a_stages = (budget - b_stages * b_bytes) / kATileBytes;
+  if (a_stages > kMaxAStages) a_stages = kMaxAStages;
+  if (a_stages < 2) return false;
+  p->a_stages = a_stages; p->b_stages = b_stages;
+  p->smem_bytes = a_stages * kATileBytes + b_stages * b_bytes + stage_bytes + 1024;
+  return true;
+}
+
 bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   DirectParams p{};
   if (d.kind == 0) {
@@ -679,19 +780,7 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   p.splits = (p.total_ktiles + p.ktiles_per_split - 1) / p.ktiles_per_split;
   p.tmem_cols = 32;
   while (p.tmem_cols < p.n_cols) p.tmem_cols *= 2;
-  // shared memory: gradient ring (3 tiles, 2 when they are large), then as many activation
-  // tiles as fit (up to 8)
-  const int budget = 224 * 1024 - 1024;
-  const int b_bytes = p.n_cols * (p.pair ? 64 : 128);
-  int b_stages = (budget - 4 * kATileBytes) / b_bytes;     // room for four activation tiles at least
-  if (b_stages > kMaxBStages) b_stages = kMaxBStages;
-  if (b_stages < 2) b_stages = 2;
-  if (b_stages * b_bytes + 2 * kATileBytes > budget) return false;
-  int a_stages = (budget - b_stages * b_bytes) / kATileBytes;
-  if (a_stages > kMaxAStages) a_stages = kMaxAStages;
-  if (a_stages < 2) return false;
-  p.a_stages = a_stages; p.b_stages = b_stages;
-  p.smem_bytes = a_stages * kATileBytes + b_stages * b_bytes + 1024;
+  if (!size_rings(&p, kStageBytes)) return false;   // the launcher sizes them again for the dtype
   *out = p;
   return true;
 }
@@ -706,7 +795,10 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
                           const float* grad_out, void* grad_bf16, float* partial,
                           uint32_t* status, cudaStream_t stream) {
   DirectParams p = plan;
+  if (!size_rings(&p, act.dt == 0 ? kStageBytes : 0)) return cudaErrorInvalidValue;
   p.n_words = (act.n + 31) / 32;
+  p.n_keep_ptr = reinterpret_cast<const long long*>(reinterpret_cast<const char*>(act.header) +
+                                                    offsetof(surgeon_header, n_keep));
   p.partial_blk = (act.n % SURGEON_BLOCK) ? static_cast<unsigned>(act.n / SURGEON_BLOCK) : 0xFFFFFFFFu;
   cudaError_t e;
   if (p.row_shift) {
