@@ -221,7 +221,10 @@ constexpr int kCsThreads = (kCsWarps + 1) * 32;
 constexpr int kCsStageRows = kCsWarps * 32;
 constexpr int kCsStageBytes = kCsStageRows * 128;
 constexpr int kCsStages = 3;
-constexpr size_t kCsSmem = static_cast<size_t>(kCsStages) * kCsStageBytes + 1024;
+// The ring starts on a 4 KB boundary: every warp's 4 KB part of a stage is then 4 KB-aligned, which
+// the compaction's gather uses to swizzle full shared-memory addresses.
+constexpr uintptr_t kCsAlign = 4096;
+constexpr size_t kCsSmem = static_cast<size_t>(kCsStages) * kCsStageBytes + kCsAlign;
 static_assert(kCsStageRows * 128 / 16 == kCsWarps * kTileVecs, "a warp's 32 rows are one chunk");
 
 // This lane's row (8 vectors) out of the swizzled stage; the ragged last row of the tensor, which
@@ -252,6 +255,28 @@ __device__ __forceinline__ int load_row(const unsigned char* region, const typen
   }
   return static_cast<int>(nv);
 }
+// bf16 keys are compared two at a time inside their 32-bit word: a key is at most 0x7FFF, so
+// key + (0x8000 - t) carries into bit 15 of its half exactly when key >= t, and never into the
+// other half.  The flag bits of the 16 words of a group of 32 elements are collected in one mask,
+// word i shifted right by i: bit (15 - i) is element 2i, bit (31 - i) element 2i + 1.
+__device__ __forceinline__ uint32_t ge_const(uint32_t t) {       // t in [0, 0x8000]
+  return (0x8000u - t) * 0x10001u;
+}
+__device__ __forceinline__ uint32_t pair_flags(uint32_t keys2, uint32_t c, int i) {
+  return ((keys2 + c) >> i) & (0x80008000u >> i);
+}
+// The same mask in element order (bit e = element e).
+__device__ __forceinline__ uint32_t pairs_to_element_order(uint32_t m) {
+  const uint32_t r = __brev(m);              // bit (16 + i): element 2i, bit i: element 2i + 1
+  auto spread = [](uint32_t x) {             // bit i -> bit 2i, for x < 2^16
+    x = (x | (x << 8)) & 0x00FF00FFu;
+    x = (x | (x << 4)) & 0x0F0F0F0Fu;
+    x = (x | (x << 2)) & 0x33333333u;
+    x = (x | (x << 1)) & 0x55555555u;
+    return x;
+  };
+  return spread(r >> 16) | (spread(r & 0xFFFFu) << 1);
+}
 __device__ __forceinline__ uint32_t valid_mask(int nv, int w) {
   const int left = nv - 32 * w;
   return left >= 32 ? 0xFFFFFFFFu : (left <= 0 ? 0u : ((1u << left) - 1u));
@@ -277,7 +302,7 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
   constexpr int kSlot = (DT == 0) ? 64 : 128;
   extern __shared__ __align__(1024) unsigned char cs_smem_raw[];
   unsigned char* ring = reinterpret_cast<unsigned char*>(
-      (reinterpret_cast<uintptr_t>(cs_smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+      (reinterpret_cast<uintptr_t>(cs_smem_raw) + kCsAlign - 1) & ~(kCsAlign - 1));
   __shared__ __align__(8) unsigned long long bars[2 * kCsStages];
   __shared__ uint32_t s_hist[kBinsA];
   __shared__ uint32_t s_tot[2];
@@ -293,6 +318,9 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
   const uint32_t cand_lo = hi_key >= lo_key ? lo_key : 0xFFFFFFFFu;
   const uint32_t range = hi_key >= lo_key ? hi_key - lo_key : 0u;
   const uint32_t shiftA = st->shiftA;
+  // bf16: the two comparisons as additions on packed pairs of keys (hi_key <= 0x7FFF there)
+  const uint32_t c_above = ge_const(hi_key >= 0x7FFFu ? 0x8000u : hi_key + 1u);
+  const uint32_t c_lo = hi_key >= lo_key ? ge_const(lo_key > 0x8000u ? 0x8000u : lo_key) : 0u;
   const uint32_t full_bar = smem_u32(bars);
   const uint32_t empty_bar = smem_u32(bars + kCsStages);
   if (tid == 0) {
@@ -340,37 +368,49 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
         uint4 q[8];
         const long long grow = static_cast<long long>(chunk) * 32 + lane;
         const int nv = load_row<DT>(region, x, n, n_rows_full, grow, q);
-        uint32_t aw[WPL], cw[WPL];
+        uint32_t cw[WPL];
+        uint32_t ac = 0, cc = 0;
+        if (DT == 0) {
+          uint32_t aw = 0;
+          cw[0] = 0;
 #pragma unroll
-        for (int w = 0; w < WPL; ++w) { aw[w] = 0; cw[w] = 0; }
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t c[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const uint32_t c[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            if (DT == 0) {
+            for (int i = 0; i < 4; ++i) {
               const uint32_t key = c[i] & kMask;
-              aw[0] |= (key > hi_key ? 1u : 0u) << (4 * j + i);
+              aw |= (key > hi_key ? 1u : 0u) << (4 * j + i);
               cw[0] |= (key - cand_lo <= range ? 1u : 0u) << (4 * j + i);
-            } else {
-              const int e = 8 * j + 2 * i;
-              const uint32_t k0 = c[i] & kMask, k1 = (c[i] >> 16) & kMask;
-              aw[e >> 5] |= (k0 > hi_key ? 1u : 0u) << (e & 31);
-              aw[e >> 5] |= (k1 > hi_key ? 1u : 0u) << ((e + 1) & 31);
-              cw[e >> 5] |= (k0 - cand_lo <= range ? 1u : 0u) << (e & 31);
-              cw[e >> 5] |= (k1 - cand_lo <= range ? 1u : 0u) << ((e + 1) & 31);
             }
           }
-        }
-        uint32_t ac = 0, cc = 0;
+          const uint32_t vm = valid_mask(nv, 0);
+          cw[0] &= vm;
+          ac = __popc(aw & vm);
+        } else {
+          // above: key >= hi_key + 1; inside the bracket: key >= lo_key and not above
+          uint32_t ga[WPL], gl[WPL];
 #pragma unroll
-        for (int w = 0; w < WPL; ++w) {
-          const uint32_t vm = valid_mask(nv, w);
-          aw[w] &= vm;
-          cw[w] &= vm;
-          ac += __popc(aw[w]);
-          cc += __popc(cw[w]);
+          for (int w = 0; w < WPL; ++w) { ga[w] = 0; gl[w] = 0; }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t c[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int pw = 4 * j + i;           // packed word of the row: elements 2pw, 2pw + 1
+              const uint32_t keys2 = c[i] & 0x7FFF7FFFu;
+              ga[(pw >> 4) % WPL] |= pair_flags(keys2, c_above, pw & 15);
+              gl[(pw >> 4) % WPL] |= pair_flags(keys2, c_lo, pw & 15);
+            }
+          }
+#pragma unroll
+          for (int w = 0; w < WPL; ++w) {
+            ac += __popc(ga[w]);        // zeros that fill a ragged row are never above
+            const uint32_t in = gl[w] & ~ga[w];
+            cw[w] = in ? (pairs_to_element_order(in) & valid_mask(nv, w)) : 0u;
+          }
         }
+#pragma unroll
+        for (int w = 0; w < WPL; ++w) cc += __popc(cw[w]);
         const uint32_t a_tot = __reduce_add_sync(kFull, ac);
         const uint32_t c_tot = __reduce_add_sync(kFull, cc);
         if (lane == 0) { cnt_gt[chunk] = a_tot; cand_cnt[chunk] = c_tot; }
@@ -1053,7 +1093,7 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
   constexpr int LPB = 32 / BPC;                // lanes per offset block: 4 / 2
   extern __shared__ __align__(1024) unsigned char cs_smem_raw[];
   unsigned char* ring = reinterpret_cast<unsigned char*>(
-      (reinterpret_cast<uintptr_t>(cs_smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+      (reinterpret_cast<uintptr_t>(cs_smem_raw) + kCsAlign - 1) & ~(kCsAlign - 1));
   __shared__ __align__(8) unsigned long long bars[2 * kCsStages];
   const E* __restrict__ x = reinterpret_cast<const E*>(xv);
   E* __restrict__ values = reinterpret_cast<E*>(values_v);
@@ -1144,6 +1184,7 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
       uint32_t word[WPL];
 #pragma unroll
       for (int w = 0; w < WPL; ++w) word[w] = 0;
+      const uint32_t c_thr = ge_const(thr > 0x8000u ? 0x8000u : thr);   // bf16: packed pairs of keys
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const uint32_t c[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
@@ -1152,11 +1193,14 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
           if (DT == 0) {
             word[0] |= ((c[i] & kMask) >= thr ? 1u : 0u) << (4 * j + i);
           } else {
-            const int e = 8 * j + 2 * i;          // element index inside the row
-            word[e >> 5] |= ((c[i] & kMask) >= thr ? 1u : 0u) << (e & 31);
-            word[e >> 5] |= (((c[i] >> 16) & kMask) >= thr ? 1u : 0u) << ((e + 1) & 31);
+            const int pw = 4 * j + i;             // packed word of the row: elements 2pw, 2pw + 1
+            word[(pw >> 4) % WPL] |= pair_flags(c[i] & 0x7FFF7FFFu, c_thr, pw & 15);
           }
         }
+      }
+      if (DT != 0) {
+#pragma unroll
+        for (int w = 0; w < WPL; ++w) word[w] = pairs_to_element_order(word[w]);
       }
 #pragma unroll
       for (int w = 0; w < WPL; ++w) {
@@ -1190,50 +1234,87 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
       // ---- kept values: gathered in place (packed order), then out as 16-byte vectors ----
       __syncwarp();                                // every lane has its row in registers
       E* outp = reinterpret_cast<E*>(region);
-      // Packed position p lives at swz(p): the 32-bit word index is XORed with the index of its
-      // 128-byte row.  Without it, lanes that keep their whole row (chunks before the end of a
-      // large tie quota, e.g. the zeros of post-ReLU data at a low ratio) all start a multiple
-      // of 32 words apart and every store of the gather is a 32-way bank conflict.
-      auto swz = [](uint32_t p) -> uint32_t {
+      // The byte at offset a of the packed sequence lives at a ^ ((a >> 5) & 0x7C): the 32-bit word
+      // index is XORed with the index of its 128-byte row.  Without it, lanes that keep their
+      // whole row (chunks before the end of a large tie quota, e.g. the zeros of post-ReLU data at
+      // a low ratio) all start a multiple of 32 words apart and every store of the gather is a
+      // 32-way bank conflict.  The region is 4 KB-aligned, so the same expression works on the
+      // full shared-memory address.
+      auto swz = [](uint32_t p) -> uint32_t {       // the same map on element indices
         return p ^ ((((p * static_cast<uint32_t>(sizeof(E))) >> 7) & 31u) << (DT == 0 ? 0 : 1));
       };
-      uint32_t pos = lane_pre;
+      // The sequence starts `mis` elements into the region when that fits, mis = the misalignment
+      // of its destination in `values`: 16-byte vectors of the region and of `values` then line up.
+      const uint32_t mis = static_cast<uint32_t>(kept_before % EPV);
+      const bool lined_up = total + mis <= static_cast<uint32_t>(32 * EPR);
+      const uint32_t shift = lined_up ? mis : 0u;
+      const uint32_t rbase = smem_u32(region);
+      uint32_t a = rbase + (lane_pre + shift) * static_cast<uint32_t>(sizeof(E));
+      auto put = [&](uint32_t v) {
+        const uint32_t pa = a ^ ((a >> 5) & 0x7Cu);
+        if (DT == 0) asm volatile("st.shared.u32 [%0], %1;" ::"r"(pa), "r"(v) : "memory");
+        else asm volatile("st.shared.u16 [%0], %1;" ::"r"(pa), "h"(static_cast<unsigned short>(v)) : "memory");
+        a += static_cast<uint32_t>(sizeof(E));
+      };
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const uint32_t c[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           if (DT == 0) {
-            if ((word[0] >> (4 * j + i)) & 1u) outp[swz(pos++)] = static_cast<E>(c[i]);
+            if ((word[0] >> (4 * j + i)) & 1u) put(c[i]);
           } else {
             const int e = 8 * j + 2 * i;
-            if ((word[e >> 5] >> (e & 31)) & 1u) outp[swz(pos++)] = static_cast<E>(c[i] & 0xFFFFu);
-            if ((word[e >> 5] >> ((e + 1) & 31)) & 1u) outp[swz(pos++)] = static_cast<E>(c[i] >> 16);
+            if ((word[(e >> 5) % WPL] >> (e & 31)) & 1u) put(c[i]);
+            if ((word[(e >> 5) % WPL] >> ((e + 1) & 31)) & 1u) put(c[i] >> 16);
           }
         }
       }
       __syncwarp();
-      E* dst = values + kept_before;
-      const uint32_t mis = static_cast<uint32_t>(kept_before % EPV);
-      uint32_t head = mis ? EPV - mis : 0;
-      if (head > total) head = total;
-      const uint32_t n_vec = (total - head) / EPV;
-      if (lane < head) dst[lane] = outp[swz(lane)];
-      for (uint32_t v = lane; v < n_vec; v += 32) {
-        const uint32_t b = head + v * EPV;
-        uint4 o;
-        if (DT == 0) {
-          o = make_uint4(outp[swz(b)], outp[swz(b + 1)], outp[swz(b + 2)], outp[swz(b + 3)]);
-        } else {
-          o = make_uint4(outp[swz(b)] | (static_cast<uint32_t>(outp[swz(b + 1)]) << 16),
-                         outp[swz(b + 2)] | (static_cast<uint32_t>(outp[swz(b + 3)]) << 16),
-                         outp[swz(b + 4 % EPV)] | (static_cast<uint32_t>(outp[swz(b + 5 % EPV)]) << 16),
-                         outp[swz(b + 6 % EPV)] | (static_cast<uint32_t>(outp[swz(b + 7 % EPV)]) << 16));
+      if (lined_up) {
+        // slots [mis, mis + total) of the region go to gbase[mis ...]; gbase is 16-byte aligned
+        E* gbase = values + (kept_before - mis);
+        const uint32_t end = mis + total;
+        const uint32_t v_first = mis ? 1u : 0u;    // first whole vector
+        const uint32_t v_end = end / EPV;          // one past the last whole vector
+        if (mis) {
+          const uint32_t sl = mis + lane;
+          if (sl < static_cast<uint32_t>(EPV) && sl < end) gbase[sl] = outp[swz(sl)];
         }
-        *reinterpret_cast<uint4*>(dst + head + v * EPV) = o;
+        for (uint32_t g = v_first + lane; g < v_end; g += 32) {
+          // the four words of a vector share their row: one 16-byte load, words permuted by the XOR
+          const uint32_t la = g * 16u;
+          const uint32_t xr = (la >> 5) & 0x7Cu;
+          uint4 u = *reinterpret_cast<const uint4*>(region + (la ^ (xr & 0x70u)));
+          if (xr & 4u) { uint32_t t = u.x; u.x = u.y; u.y = t; t = u.z; u.z = u.w; u.w = t; }
+          if (xr & 8u) { uint32_t t = u.x; u.x = u.z; u.z = t; t = u.y; u.y = u.w; u.w = t; }
+          *reinterpret_cast<uint4*>(gbase + g * EPV) = u;
+        }
+        const uint32_t t0 = (v_end > v_first ? v_end : v_first) * EPV;
+        if (t0 + lane < end) gbase[t0 + lane] = outp[swz(t0 + lane)];
+      } else {
+        // a full chunk with a misaligned destination: no room for the shift, element-wise vectors
+        E* dst = values + kept_before;
+        uint32_t head = mis ? EPV - mis : 0;
+        if (head > total) head = total;
+        const uint32_t n_vec = (total - head) / EPV;
+        if (lane < head) dst[lane] = outp[swz(lane)];
+        for (uint32_t v = lane; v < n_vec; v += 32) {
+          const uint32_t b = head + v * EPV;
+          uint4 o;
+          if (DT == 0) {
+            o = make_uint4(outp[swz(b)], outp[swz(b + 1)], outp[swz(b + 2)], outp[swz(b + 3)]);
+          } else {
+            o = make_uint4(outp[swz(b)] | (static_cast<uint32_t>(outp[swz(b + 1)]) << 16),
+                           outp[swz(b + 2)] | (static_cast<uint32_t>(outp[swz(b + 3)]) << 16),
+                           outp[swz(b + 4 % EPV)] | (static_cast<uint32_t>(outp[swz(b + 5 % EPV)]) << 16),
+                           outp[swz(b + 6 % EPV)] | (static_cast<uint32_t>(outp[swz(b + 7 % EPV)]) << 16));
+          }
+          *reinterpret_cast<uint4*>(dst + head + v * EPV) = o;
+        }
+        const uint32_t done = head + n_vec * EPV;
+        if (lane < total - done) dst[done + lane] = outp[swz(done + lane)];
       }
-      const uint32_t done = head + n_vec * EPV;
-      if (lane < total - done) dst[done + lane] = outp[swz(done + lane)];
     }
     tc::fence_proxy_async();     // this warp's writes to the stage precede the next TMA fill
     __syncwarp();

@@ -113,6 +113,24 @@ def test_all_equal_and_two_level(bf16):
         assert_store_equals_oracle(_as(x, bf16), ratio)
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("odd", [1, 3, 5, 7])
+def test_fully_kept_chunks_behind_a_misaligned_kept_count(odd, bf16):
+    # A head of small magnitudes of which an odd number is kept, then large magnitudes that are all
+    # kept: every later 4 KB piece is written out whole, starting at a packed position that is not
+    # a multiple of a 16-byte vector.
+    n_head, n = 3 * 4096 + 40, 1 << 21
+    g = torch.Generator().manual_seed(17 + odd)
+    x = torch.empty(n)
+    x[:n_head] = torch.rand(n_head, generator=g) * 0.5 + 0.01
+    x[n_head:] = (torch.rand(n - n_head, generator=g) * 8.0 + 2.0) * torch.where(
+        torch.rand(n - n_head, generator=g) < 0.5, -1.0, 1.0)
+    keep_head = 1000 + odd
+    ratio = (n_head - keep_head + 0.5) / n            # n - floor(ratio * n) = n - n_head + keep_head
+    comp, ref = assert_store_equals_oracle(_as(x, bf16), ratio)
+    assert ref["k"] == n - n_head + keep_head
+
+
 def test_repeat_calls_are_bitwise_identical_and_reuse_buffers():
     x = W.draw("ties16", 300000, seed=5).cuda()
     comp = B.surgeon_prune_compact(x, 0.7)
