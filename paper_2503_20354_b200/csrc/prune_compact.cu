@@ -224,6 +224,7 @@ constexpr int kCsStages = 3;
 // The ring starts on a 4 KB boundary: every warp's 4 KB part of a stage is then 4 KB-aligned, which
 // the compaction's gather uses to swizzle full shared-memory addresses.
 constexpr uintptr_t kCsAlign = 4096;
+constexpr int kMinTilesPerCta = 4;
 constexpr size_t kCsSmem = static_cast<size_t>(kCsStages) * kCsStageBytes + kCsAlign;
 static_assert(kCsStageRows * 128 / 16 == kCsWarps * kTileVecs, "a warp's 32 rows are one chunk");
 
@@ -1417,7 +1418,10 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k, int drop_
   const long long n_rows_full = n * static_cast<long long>(sizeof(E)) / 128;
   const int n_chunks = static_cast<int>(L.tiles);
   const int n_stage_tiles = (n_chunks + kCsWarps - 1) / kCsWarps;
-  const int stream_grid = n_stage_tiles < 2 * sms ? n_stage_tiles : 2 * sms;
+  // at least kMinTilesPerCta stages per CTA: a CTA's set-up and tail cost about two stages' time, and a
+  // small tensor then leaves SM slots to the kernels of other streams
+  const int want_ctas = (n_stage_tiles + kMinTilesPerCta - 1) / kMinTilesPerCta;
+  const int stream_grid = want_ctas < 2 * sms ? want_ctas : 2 * sms;
   CUtensorMap map;
   const bool streamed = n > kSampleMinN && make_row_map(x, n_rows_full, &map);
 
