@@ -7,7 +7,7 @@ saved activation (Algorithm 1: prune and decompose steps), and the weight gradie
 compressed store (its Reshape and gradient steps).  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                  [--workload wrn28|tiny|resnet50|vit|sweep] [--batch B] [--path tc|fp32]
+                  [--workload wrn28|tiny|resnet50|vit|segformer|sweep] [--batch B] [--path tc|fp32]
 
 N > 1 (launched with torch.distributed.run): every rank runs an independent replica of the
 step on its own GPU (the path has no exchange step); time is the max over ranks.
@@ -58,6 +58,8 @@ def get_layers(workload: str, batch):
         return W.resnet50(batch or 64), "ResNet-50-shaped stack, 224x224, batch %d, bf16 activations" % (batch or 64)
     if workload == "vit":
         return W.vit_b16(batch or 64), "ViT-B/16-shaped stack, batch %d, bf16 activations" % (batch or 64)
+    if workload == "segformer":
+        return W.segformer_b5(1024, batch or 1), "linear layers of a Segformer-B5-shaped encoder, 1024x1024, batch %d, bf16 activations" % (batch or 1)
     raise SystemExit("unknown workload %r" % workload)
 
 
@@ -530,7 +532,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="wrn28", choices=["wrn28", "tiny", "resnet50", "vit", "sweep"])
+    ap.add_argument("--workload", default="wrn28", choices=["wrn28", "tiny", "resnet50", "vit", "segformer", "sweep"])
     ap.add_argument("--sweep-sizes", type=int, default=5, help="how many of 2^20,22,24,26,28,30 the sweep covers")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--layers", default=None, help="comma-separated layer names: run only these (profiling)")

@@ -1423,7 +1423,7 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k, int drop_
   const int want_ctas = (n_stage_tiles + kMinTilesPerCta - 1) / kMinTilesPerCta;
   const int stream_grid = want_ctas < 2 * sms ? want_ctas : 2 * sms;
   CUtensorMap map;
-  const bool streamed = n > kSampleMinN && make_row_map(x, n_rows_full, &map);
+  const bool streamed = n * static_cast<long long>(sizeof(E)) >= kStreamMinBytes && make_row_map(x, n_rows_full, &map);
 
   if (k == 0) {
     header_empty_kernel<<<1, 1, 0, stream>>>(out.header, Elem<DT>::kSentinel, out.block_offsets,
@@ -1440,7 +1440,7 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k, int drop_
       long long n_seg = n_seg_all / 32;
       if (n_seg < 256) n_seg = 256;
       if (n_seg > 16384) n_seg = 16384;
-      const long long seg_stride = n_seg_all / n_seg;   // >= 1 because n > 65536
+      const long long seg_stride = n_seg_all / n_seg;   // >= 1: a streamed tensor has at least 2^22 elements
       const long long want = (n_seg + 127) / 128;
       const int grid = static_cast<int>(want < sms ? want : sms);
       sample_kernel<DT><<<grid, kSelThreads, kHistWords * 4, stream>>>(

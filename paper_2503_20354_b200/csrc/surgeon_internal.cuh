@@ -38,7 +38,11 @@ constexpr int kBinsA = 512;            // level A of the select among candidates
                                        // (key - lo_key), shifted so that the bracket fits
 constexpr int kBinsB = 4096;           // up to two further levels of 2048 bins each
 constexpr int kFbBins = 2048;          // digit histogram of the fall-back radix select
-constexpr int64_t kSampleMinN = 65536; // smaller tensors go straight to the fall-back select
+// Tensors below this size go straight to the fall-back select: its passes over a tensor that
+// stays in L2 finish sooner than the four dependent kernels of the sampled path.  Alone on the
+// GPU that holds up to 16-32 MB; next to other streams' kernels the fall-back's cooperative
+// grid (one CTA per 32 chunks) has to wait for them, and 4 MB is where both cases gain.
+constexpr int64_t kStreamMinBytes = 4 << 20;
 // Candidate slots: per chunk, room for 1/16 of its elements (fp32: 32-bit keys, bf16: 16-bit).
 constexpr int slot_entries(int dt) { return dt == 0 ? 64 : 128; }
 constexpr int slot_entry_bytes(int dt) { return dt == 0 ? 4 : 2; }

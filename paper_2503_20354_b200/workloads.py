@@ -2,7 +2,8 @@
 
 This module holds no arithmetic of the method (no ratios, thresholds, pruning or gradients):
 only the shapes of the networks the paper adapts (Section 5.1: WideResNet-28-10 at batch 200,
-ResNet-50 at batch 64) plus a ViT-B/16-shaped stack, and random tensors with the value
+ResNet-50 at batch 64, the linear layers of Segformer-B5 at batch 1) plus a ViT-B/16-shaped
+stack, and random tensors with the value
 distributions of their saved activations.  The tensors stand in for CIFAR10-C / ImageNet-C
 batches flowing through pre-trained backbones, which are not available offline.  The same bytes
 are handed to the CUDA library and to the CPU oracle by the tests and the benchmark.
@@ -34,6 +35,7 @@ class Layer:
     pad: int = 0
     dist: str = "relu_normal"   # distribution of the saved input activation
     dt: int = F32               # dtype of the saved activation
+    rows_per_sample: int = 0    # linear layers: rows T per sample (0: see shrink)
 
     @property
     def oh(self) -> int:
@@ -87,8 +89,8 @@ def conv(name, batch, c_in, hw, c_out, k, stride=1, pad=None, dist="relu_normal"
     return Layer(name, 1, batch, c_in, hw, hw, c_out, k, k, stride, pad, dist, dt)
 
 
-def linear(name, rows, c_in, c_out, dist="normal", dt=BF16) -> Layer:
-    return Layer(name, 0, rows, c_in, 1, 1, c_out, 1, 1, 1, 0, dist, dt)
+def linear(name, rows, c_in, c_out, dist="normal", dt=BF16, rows_per_sample=0) -> Layer:
+    return Layer(name, 0, rows, c_in, 1, 1, c_out, 1, 1, 1, 0, dist, dt, rows_per_sample)
 
 
 def tiny_conv(batch: int = 16) -> List[Layer]:
@@ -146,6 +148,30 @@ def vit_b16(batch: int = 64, dt: int = BF16, blocks: int = 12) -> List[Layer]:
     return L
 
 
+def segformer_b5(image: int = 1024, batch: int = 1, dt: int = BF16, depths=(3, 6, 40, 3)) -> List[Layer]:
+    """The linear layers of a Segformer-B5-shaped encoder (Section 5.1: semantic segmentation at
+    batch 1) on an image x image input: four stages of widths 64 / 128 / 320 / 512 on token grids
+    of 1/4, 1/8, 1/16 and 1/32 of the image side, attention with keys and values on a grid reduced
+    8 / 4 / 2 / 1 times per side, MLP ratio 4.  Per block: q, kv, proj, fc1, fc2.  The strided
+    reduction convolutions and the depthwise 3x3 convolution of the MLP (a grouped layer) are not
+    part of this stack."""
+    widths, reductions = (64, 128, 320, 512), (8, 4, 2, 1)
+    L = []
+    for s in range(4):
+        side = image // (4 << s)
+        t_q = side * side
+        t_kv = (side // reductions[s]) ** 2
+        c = widths[s]
+        for b in range(depths[s]):
+            n = f"s{s}b{b}"
+            L.append(linear(n + ".q", batch * t_q, c, c, "normal", dt, t_q))
+            L.append(linear(n + ".kv", batch * t_kv, c, 2 * c, "normal", dt, t_kv))
+            L.append(linear(n + ".proj", batch * t_q, c, c, "normal", dt, t_q))
+            L.append(linear(n + ".fc1", batch * t_q, c, 4 * c, "normal", dt, t_q))
+            L.append(linear(n + ".fc2", batch * t_q, 4 * c, c, "gelu_normal", dt, t_q))
+    return L
+
+
 def shrink(layers: List[Layer], batch: int) -> List[Layer]:
     """Same stack at a smaller batch (rows scale with the batch for linear layers)."""
     out = []
@@ -154,7 +180,7 @@ def shrink(layers: List[Layer], batch: int) -> List[Layer]:
             out.append(replace(l, batch=batch))
         else:
             full = l.batch
-            per = 197 if full % 197 == 0 else 1
+            per = l.rows_per_sample or (197 if full % 197 == 0 else 1)
             out.append(replace(l, batch=batch * per))
     return out
 

@@ -50,15 +50,16 @@ def test_empty_tensor(bf16):
 
 @pytest.mark.parametrize("bf16", [False, True])
 @pytest.mark.parametrize("dist", ["relu_normal", "normal", "student_t2", "ties16", "gelu_normal"])
-def test_distributions_and_ratios(dist, bf16):
-    n = (1 << 20) + 4321   # many tiles and a ragged tail
+@pytest.mark.parametrize("log2n", [20, 23])       # below / above the size where the sampled path starts
+def test_distributions_and_ratios(dist, log2n, bf16):
+    n = (1 << log2n) + 4321   # many tiles and a ragged tail
     x = _as(W.draw(dist, n, seed=2), bf16)
     for ratio in (0.1, 0.5, 0.9, 0.99):
         assert_store_equals_oracle(x, ratio)
 
 
 @pytest.mark.parametrize("bf16", [False, True])
-@pytest.mark.parametrize("n", [1000, 65536 + 7, 300000, (1 << 22) + 77])
+@pytest.mark.parametrize("n", [1000, 65536 + 7, 300000, (1 << 23) + 77])
 def test_store_without_kept_zeros(n, bf16):
     """SURGEON_STORE_DROP_ZEROS: bit-exact with the oracle's variant; at ratios that keep more than
     the non-zero half of post-ReLU data the threshold key is 0 and the zeros are left out."""
@@ -119,7 +120,7 @@ def test_fully_kept_chunks_behind_a_misaligned_kept_count(odd, bf16):
     # A head of small magnitudes of which an odd number is kept, then large magnitudes that are all
     # kept: every later 4 KB piece is written out whole, starting at a packed position that is not
     # a multiple of a 16-byte vector.
-    n_head, n = 3 * 4096 + 40, 1 << 21
+    n_head, n = 3 * 4096 + 40, 1 << 23
     g = torch.Generator().manual_seed(17 + odd)
     x = torch.empty(n)
     x[:n_head] = torch.rand(n_head, generator=g) * 0.5 + 0.01
