@@ -48,6 +48,10 @@ def load_peaks():
     return d
 
 
+# ncu launch lists of one step (profiles/launch_list_*_bench_step.md), weight-gradient kernels only
+DW_STEP_DRAM_BYTES = {"wrn28": 7552000000, "resnet50": 7263000000}
+
+
 def get_layers(workload: str, batch):
     from paper_2503_20354_b200 import workloads as W
     if workload == "wrn28":
@@ -377,9 +381,15 @@ def run_ours(args, rank, world, local):
     else:
         peak, bound, unit = FP32_ALU_TFLOPS, "alu", "TFLOP/s"
         peak_note = "derived: 148 SMs x 128 fp32 FMA lanes x 2 x 1.965 GHz"
+    # DRAM bytes the weight-gradient kernels of one step moved under ncu (dram__bytes_read.sum +
+    # dram__bytes_write.sum summed over their launches): known for the full-size stacks on the
+    # tensor-core path only, and only while those kernels are the ones the counters were taken on.
+    traffic = None
+    if path == B.PATH_TENSOR_CORE and args.batch is None and args.layers is None:
+        traffic = DW_STEP_DRAM_BYTES.get(args.workload)
     roofline = {"kernel": "weight gradient (all layers of one step)", "bound": bound,
                 "achieved": round(dw_tflops, 3), "peak": round(peak, 1), "unit": unit,
-                "frac": round(dw_tflops / peak, 4), "traffic": None, "peak_source": peak_note}
+                "frac": round(dw_tflops / peak, 4), "traffic": traffic, "peak_source": peak_note}
 
     # ---- end to end through the C ABI with host buffers --------------------------------------
     e2e = run_e2e(stack, layers, args, world, device, flops) if args.e2e else None
