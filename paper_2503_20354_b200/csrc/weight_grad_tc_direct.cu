@@ -620,7 +620,9 @@ grad_taps_bf16_kernel(const float* __restrict__ g, unsigned short* __restrict__ 
 // out[img][s * O + o][y * W + x'] = g[img][o][y][x' + pad - s] for the OH gradient rows y (zero
 // where the column lies outside the output map).  One thread reads a window of 8 + KW - 1
 // gradient values and writes 8 positions of every shift.
-template <int KW>
+// SAME: padding (KW - 1) / 2 with KW odd, so the output map is as wide as the input (a multiple of
+// 8): the 8 elements of a chunk are two aligned 16-byte loads, only the halo is fetched singly.
+template <int KW, bool SAME>
 __global__ void __launch_bounds__(256)
 grad_cols_bf16_kernel(const float* __restrict__ g, unsigned short* __restrict__ out,
                       long long chunks, DirectParams p) {
@@ -636,10 +638,24 @@ grad_cols_bf16_kernel(const float* __restrict__ g, unsigned short* __restrict__ 
     const int o = static_cast<int>(plane - img * p.o_real);
     const float* src = g + (plane * p.oh + y) * static_cast<long long>(p.ow);
     float f[8 + KW - 1];                               // f[j] = g[y][x0 + pad - (KW - 1) + j]
+    if (SAME) {
+      constexpr int H = (KW - 1) / 2;                  // f[j] = g[y][x0 - H + j]
+      const float4 a = __ldg(reinterpret_cast<const float4*>(src + x0));
+      const float4 b = __ldg(reinterpret_cast<const float4*>(src + x0 + 4));
+      f[H] = a.x; f[H + 1] = a.y; f[H + 2] = a.z; f[H + 3] = a.w;
+      f[H + 4] = b.x; f[H + 5] = b.y; f[H + 6] = b.z; f[H + 7] = b.w;
 #pragma unroll
-    for (int j = 0; j < 8 + KW - 1; ++j) {
-      const int x = x0 + p.pad - (KW - 1) + j;
-      f[j] = (x >= 0 && x < p.ow) ? __ldg(src + x) : 0.0f;
+      for (int j = 0; j < H; ++j) {
+        const int xl = x0 - H + j, xr = x0 + 8 + j;
+        f[j] = xl >= 0 ? __ldg(src + xl) : 0.0f;
+        f[H + 8 + j] = xr < p.ow ? __ldg(src + xr) : 0.0f;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8 + KW - 1; ++j) {
+        const int x = x0 + p.pad - (KW - 1) + j;
+        f[j] = (x >= 0 && x < p.ow) ? __ldg(src + x) : 0.0f;
+      }
     }
 #pragma unroll
     for (int sft = 0; sft < KW; ++sft) {
@@ -807,11 +823,22 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
     const long long cap = 32LL * sm_count();
     const int grid = static_cast<int>(want < 1 ? 1 : (want > cap ? cap : want));
     unsigned short* ob = static_cast<unsigned short*>(grad_bf16);
+    const bool same = (p.kw & 1) && p.pad == (p.kw - 1) / 2 && p.ow == p.in_w &&
+                      (reinterpret_cast<uintptr_t>(grad_out) & 15) == 0;
     switch (p.kw) {
-      case 2: grad_cols_bf16_kernel<2><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p); break;
-      case 3: grad_cols_bf16_kernel<3><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p); break;
-      case 5: grad_cols_bf16_kernel<5><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p); break;
-      default: grad_cols_bf16_kernel<7><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p); break;
+      case 2: grad_cols_bf16_kernel<2, false><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p); break;
+      case 3:
+        if (same) grad_cols_bf16_kernel<3, true><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p);
+        else grad_cols_bf16_kernel<3, false><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p);
+        break;
+      case 5:
+        if (same) grad_cols_bf16_kernel<5, true><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p);
+        else grad_cols_bf16_kernel<5, false><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p);
+        break;
+      default:
+        if (same) grad_cols_bf16_kernel<7, true><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p);
+        else grad_cols_bf16_kernel<7, false><<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p);
+        break;
     }
     note_launches(1);
     e = cudaGetLastError();
