@@ -697,13 +697,43 @@ __global__ void __launch_bounds__(256)
 reduce_splits_taps_kernel(const float* __restrict__ partial, int o_real, int c_in, int taps,
                           int chunk, int splits, float* __restrict__ dw, int accumulate,
                           const uint32_t* __restrict__ status, surgeon_header* __restrict__ hdr) {
-  extern __shared__ float tile[];                  // [n_c][taps]
+  extern __shared__ __align__(16) float tile[];    // [n_c][taps]
   const int c0 = blockIdx.x * chunk;
   const int o = blockIdx.y;
   if (blockIdx.x == 0 && o == 0 && threadIdx.x == 0 && *status != 0 && hdr)
     atomicMax(&hdr->status, *status);
   const long long mn = static_cast<long long>(o_real) * c_in * taps;
   const int n_c = min(chunk, c_in - c0);
+  float* out = dw + (static_cast<long long>(o) * c_in + c0) * taps;
+  if ((c_in & 3) == 0) {
+    // four channels per thread: 16-byte reads of the partials, 16-byte writes of dw (c0 is a
+    // multiple of 32 and n_c of 4, so both stay aligned); the split sums keep their order
+    const int n_c4 = n_c >> 2;
+    for (int idx = threadIdx.x; idx < n_c4 * taps; idx += 256) {
+      const int tap = idx / n_c4, cl = (idx - tap * n_c4) * 4;
+      const float* src = partial + (static_cast<long long>(tap) * o_real + o) * c_in + c0 + cl;
+      float4 s = *reinterpret_cast<const float4*>(src);
+      for (int z = 1; z < splits; ++z) {
+        const float4 v = *reinterpret_cast<const float4*>(src + z * mn);
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+      }
+      tile[cl * taps + tap] = s.x;
+      tile[(cl + 1) * taps + tap] = s.y;
+      tile[(cl + 2) * taps + tap] = s.z;
+      tile[(cl + 3) * taps + tap] = s.w;
+    }
+    __syncthreads();
+    const int n4 = (n_c * taps) >> 2;                  // n_c is a multiple of 4
+    for (int idx = threadIdx.x; idx < n4; idx += 256) {
+      float4 v = *reinterpret_cast<const float4*>(tile + 4 * idx);
+      if (accumulate) {
+        const float4 d = *reinterpret_cast<const float4*>(out + 4 * idx);
+        v.x += d.x; v.y += d.y; v.z += d.z; v.w += d.w;
+      }
+      *reinterpret_cast<float4*>(out + 4 * idx) = v;
+    }
+    return;
+  }
   for (int idx = threadIdx.x; idx < n_c * taps; idx += 256) {
     const int tap = idx / n_c, cl = idx - tap * n_c;     // consecutive threads, consecutive channels
     const float* src = partial + (static_cast<long long>(tap) * o_real + o) * c_in + c0 + cl;
@@ -712,7 +742,6 @@ reduce_splits_taps_kernel(const float* __restrict__ partial, int o_real, int c_i
     tile[cl * taps + tap] = s;
   }
   __syncthreads();
-  float* out = dw + (static_cast<long long>(o) * c_in + c0) * taps;
   for (int idx = threadIdx.x; idx < n_c * taps; idx += 256)
     out[idx] = accumulate ? out[idx] + tile[idx] : tile[idx];
 }
