@@ -689,6 +689,38 @@ reduce_splits_kernel(const float* __restrict__ partial, long long mn, int splits
   dw[i] = accumulate ? dw[i] + s : s;
 }
 
+// Four elements per thread (mn a multiple of 4, 16-byte aligned pointers).
+__global__ void __launch_bounds__(256)
+reduce_splits4_kernel(const float* __restrict__ partial, long long mn, int splits,
+                      float* __restrict__ dw, int accumulate, const uint32_t* __restrict__ status,
+                      surgeon_header* __restrict__ hdr) {
+  const long long i = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
+  if (i == 0 && *status != 0 && hdr) atomicMax(&hdr->status, *status);
+  if (i >= mn) return;
+  float4 s = *reinterpret_cast<const float4*>(partial + i);
+  for (int z = 1; z < splits; ++z) {
+    const float4 v = *reinterpret_cast<const float4*>(partial + z * mn + i);
+    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+  }
+  if (accumulate) {
+    const float4 d = *reinterpret_cast<const float4*>(dw + i);
+    s.x += d.x; s.y += d.y; s.z += d.z; s.w += d.w;
+  }
+  *reinterpret_cast<float4*>(dw + i) = s;
+}
+
+static void launch_reduce_splits(const float* partial, long long mn, int splits, float* dw,
+                                 int accumulate, const uint32_t* status, surgeon_header* hdr,
+                                 cudaStream_t stream) {
+  const bool vec = (mn & 3) == 0 && ((reinterpret_cast<uintptr_t>(partial) | reinterpret_cast<uintptr_t>(dw)) & 15) == 0;
+  if (vec)
+    reduce_splits4_kernel<<<static_cast<unsigned>((mn / 4 + 255) / 256), 256, 0, stream>>>(
+        partial, mn, splits, dw, accumulate, status, hdr);
+  else
+    reduce_splits_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
+        partial, mn, splits, dw, accumulate, status, hdr);
+}
+
 // The same for a tap-stacked partial [splits][taps * O][C]: dw[o][c][tap] gets row tap * O + o.
 // One block sums `chunk` input channels of one output channel for all taps: the reads
 // run along c (contiguous in the partial, a kilobyte per warp), the writes along (c, tap)
@@ -889,8 +921,7 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
     }
 
     else
-      reduce_splits_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
-          partial, mn, dp.splits, dw, accumulate, status, act.header);
+      launch_reduce_splits(partial, mn, dp.splits, dw, accumulate, status, act.header, stream);
     note_launches(1);
     return cudaGetLastError();
   }
@@ -900,8 +931,7 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
     e = launch_conv_fast(act, f, grad_out, grad_bf16, partial, status, stream);
     if (e != cudaSuccess) return e;
     const long long fmn = static_cast<long long>(f.O) * f.n_gemm;
-    reduce_splits_kernel<<<static_cast<unsigned>((fmn + 255) / 256), 256, 0, stream>>>(
-        partial, fmn, f.splits, dw, accumulate, status, act.header);
+    launch_reduce_splits(partial, fmn, f.splits, dw, accumulate, status, act.header, stream);
     note_launches(1);
     return cudaGetLastError();
   }
@@ -949,8 +979,7 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
                                                                  map, partial, status, p);
     }
     const long long mn = static_cast<long long>(p.O) * p.n_gemm;
-    reduce_splits_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
-        partial, mn, p.splits, dw, accumulate, status, act.header);
+    launch_reduce_splits(partial, mn, p.splits, dw, accumulate, status, act.header, stream);
     note_launches(2);
     return cudaGetLastError();
   }
@@ -973,8 +1002,7 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
                                                       partial, status, p);
   }
   const long long mn = static_cast<long long>(p.O) * p.n_gemm;
-  reduce_splits_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
-      partial, mn, p.splits, dw, accumulate, status, act.header);
+  launch_reduce_splits(partial, mn, p.splits, dw, accumulate, status, act.header, stream);
   note_launches(2);
   return cudaGetLastError();
 }
