@@ -443,8 +443,15 @@ grad_to_bf16_rows_kernel(const float* __restrict__ g, long long rows, int len, i
     const int c0 = static_cast<int>(i - r * per_row) * 8;
     const float* src = g + r * len + c0;
     float v[8];
+    if ((len & 3) == 0 && c0 + 8 <= len) {         // rows start on 16-byte boundaries
+      const float4 a = __ldg(reinterpret_cast<const float4*>(src));
+      const float4 b = __ldg(reinterpret_cast<const float4*>(src) + 1);
+      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+      v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    } else {
 #pragma unroll
-    for (int e = 0; e < 8; ++e) v[e] = (c0 + e < len) ? __ldg(src + e) : 0.0f;
+      for (int e = 0; e < 8; ++e) v[e] = (c0 + e < len) ? __ldg(src + e) : 0.0f;
+    }
     uint4 o;
     o.x = pack_bf16x2(v[0], v[1]); o.y = pack_bf16x2(v[2], v[3]);
     o.z = pack_bf16x2(v[4], v[5]); o.w = pack_bf16x2(v[6], v[7]);

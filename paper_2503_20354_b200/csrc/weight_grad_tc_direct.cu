@@ -620,6 +620,59 @@ grad_taps_bf16_kernel(const float* __restrict__ g, unsigned short* __restrict__ 
 // out[img][s * O + o][y * W + x'] = g[img][o][y][x' + pad - s] for the OH gradient rows y (zero
 // where the column lies outside the output map).  One thread reads a window of 8 + KW - 1
 // gradient values and writes 8 positions of every shift.
+// The same copies for a same-padded convolution (odd KW, padding (KW - 1) / 2, output map = input
+// map): the source of input position pos under tap (r, s) is the flat index
+// pos + (pad - r) * W + (pad - s) of the output gradient's plane, so one thread reads a window of
+// 8 + KW - 1 consecutive values for a row shift r and writes the KW column shifts from it; a value
+// is dropped where the shifted column leaves the row.
+template <int KW>
+__global__ void __launch_bounds__(256)
+grad_taps_same_bf16_kernel(const float* __restrict__ g, unsigned short* __restrict__ out,
+                           long long items, DirectParams p) {
+  constexpr int H = (KW - 1) / 2;
+  const int per_row = p.pitch >> 3;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < items;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    long long t = i / per_row;
+    const int chunk = static_cast<int>(i - t * per_row);
+    const int r = static_cast<int>(t % p.kh);
+    t /= p.kh;
+    const int o = static_cast<int>(t % p.o_real);
+    const long long img = t / p.o_real;
+    const float* src = g + (img * p.o_real + o) * static_cast<long long>(p.T);
+    const int pos0 = chunk * 8;
+    const int yy0 = pos0 / p.in_w;
+    int xx = pos0 - yy0 * p.in_w;
+    const int base = pos0 + (p.pad - r) * p.in_w - H;      // flat index of w[0]
+    float w[8 + 2 * H];
+#pragma unroll
+    for (int j = 0; j < 8 + 2 * H; ++j) {
+      const int q = base + j;
+      w[j] = (q >= 0 && q < p.T) ? __ldg(src + q) : 0.0f;
+    }
+    int xe[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      xe[e] = (pos0 + e < p.T) ? xx : -64;                 // past the map: no column is valid
+      if (++xx == p.in_w) xx = 0;
+    }
+#pragma unroll
+    for (int sft = 0; sft < KW; ++sft) {
+      float f[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int x = xe[e] + H - sft;
+        f[e] = (x >= 0 && x < p.in_w) ? w[e + 2 * H - sft] : 0.0f;
+      }
+      uint4 v;
+      v.x = pack_bf16x2(f[0], f[1]); v.y = pack_bf16x2(f[2], f[3]);
+      v.z = pack_bf16x2(f[4], f[5]); v.w = pack_bf16x2(f[6], f[7]);
+      const long long rowi = (img * p.taps + r * KW + sft) * p.o_real + o;
+      *reinterpret_cast<uint4*>(out + rowi * p.pitch + chunk * 8) = v;
+    }
+  }
+}
+
 // SAME: padding (KW - 1) / 2 with KW odd, so the output map is as wide as the input (a multiple of
 // 8): the 8 elements of a chunk are two aligned 16-byte loads, only the halo is fetched singly.
 template <int KW, bool SAME>
@@ -847,8 +900,19 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
     const long long want = (chunks + 255) / 256;
     const long long cap = 32LL * sm_count();
     const int grid = static_cast<int>(want < 1 ? 1 : (want > cap ? cap : want));
-    grad_taps_bf16_kernel<<<grid, 256, 0, stream>>>(grad_out, static_cast<unsigned short*>(grad_bf16),
-                                                    chunks, p);
+    unsigned short* ob = static_cast<unsigned short*>(grad_bf16);
+    const bool same = (p.kw & 1) && p.kh == p.kw && p.pad == (p.kw - 1) / 2 && p.ow == p.in_w &&
+                      p.oh == p.in_h && (p.kw == 3 || p.kw == 5 || p.kw == 7);
+    if (same) {
+      const long long items = chunks / p.kw;        // one thread per row shift writes the kw column shifts
+      const long long want_s = (items + 255) / 256;
+      const int grid_s = static_cast<int>(want_s < 1 ? 1 : (want_s > cap ? cap : want_s));
+      if (p.kw == 3) grad_taps_same_bf16_kernel<3><<<grid_s, 256, 0, stream>>>(grad_out, ob, items, p);
+      else if (p.kw == 5) grad_taps_same_bf16_kernel<5><<<grid_s, 256, 0, stream>>>(grad_out, ob, items, p);
+      else grad_taps_same_bf16_kernel<7><<<grid_s, 256, 0, stream>>>(grad_out, ob, items, p);
+    } else {
+      grad_taps_bf16_kernel<<<grid, 256, 0, stream>>>(grad_out, ob, chunks, p);
+    }
     note_launches(1);
     e = cudaGetLastError();
   } else if (p.mode != 0 && p.pitch != p.T)     // rows padded to a 16-byte pitch for the tensor map
