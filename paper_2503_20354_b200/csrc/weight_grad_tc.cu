@@ -698,6 +698,7 @@ reduce_splits4_kernel(const float* __restrict__ partial, long long mn, int split
   if (i == 0 && *status != 0 && hdr) atomicMax(&hdr->status, *status);
   if (i >= mn) return;
   float4 s = *reinterpret_cast<const float4*>(partial + i);
+#pragma unroll 4
   for (int z = 1; z < splits; ++z) {
     const float4 v = *reinterpret_cast<const float4*>(partial + z * mn + i);
     s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
@@ -745,6 +746,7 @@ reduce_splits_taps_kernel(const float* __restrict__ partial, int o_real, int c_i
       const int tap = idx / n_c4, cl = (idx - tap * n_c4) * 4;
       const float* src = partial + (static_cast<long long>(tap) * o_real + o) * c_in + c0 + cl;
       float4 s = *reinterpret_cast<const float4*>(src);
+#pragma unroll 4
       for (int z = 1; z < splits; ++z) {
         const float4 v = *reinterpret_cast<const float4*>(src + z * mn);
         s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
