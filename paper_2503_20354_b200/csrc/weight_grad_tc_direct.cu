@@ -768,6 +768,11 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
     // activation with the output gradient shifted by (pad - r, pad - s).  The shifted copies
     // (zero outside the map) are stacked as kh*kw*O gradient channels, which makes this the 1x1
     // problem with that many output channels; the activation operand is never expanded.
+    // 8-16 channels fill an eighth of the tile's rows here; as im2col rows (channels x taps) they
+    // fill a whole tile, and the gradient is read once instead of through shifted copies
+    // (16 -> 160 channels, 3x3 on 32x32, batch 200: 145 against 181 us).  Fewer channels still
+    // are quicker here (3 channels: 94 against 110 us).
+    if (d.c_in >= 8 && d.c_in <= 16) return false;
     p.mode = 1;
     p.taps = d.kh * d.kw;
     p.kh = d.kh; p.kw = d.kw; p.pad = d.pad; p.in_h = d.h; p.in_w = d.w;
