@@ -36,7 +36,6 @@ def test_own_arm_line():
     assert c["kind"] == "oracle" and c["cores"] >= 1 and c["value"] > 0 and c["sample"]
     e = d["e2e"]
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0
-    assert e["value"] < d["value"]                      # host copies are inside that timed region
     assert d["gpu_launches"] > 0 and d["value"] > 0 and d["ms_per_step"] > 0
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
 
