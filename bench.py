@@ -49,7 +49,7 @@ def load_peaks():
 
 
 # ncu launch lists of one step (profiles/launch_list_*_bench_step.md), weight-gradient kernels only
-DW_STEP_DRAM_BYTES = {"wrn28": 7551000000, "resnet50": 7249000000}
+DW_STEP_DRAM_BYTES = {"wrn28": 7306000000, "resnet50": 7249000000}
 
 
 def get_layers(workload: str, batch):
