@@ -19,13 +19,15 @@
 //   count    : fp32 resolves the threshold among the listed keys with two histogram levels;
 //              then the listed keys above / equal to the threshold complete the per-chunk counts,
 //              and an exclusive scan over chunks follows (cooperative launch, grid barriers).
-//   compact  : the second read.  A chunk's warp starts from its entry of the scan.  The one chunk
-//              inside which the tie quota ends is emitted by a separate small kernel that ranks
-//              ties by flat index.
+//              The one chunk inside which the tie quota ends is emitted here, by the CTA that
+//              finds it, with its ties ranked by flat index.
+//   compact  : the second read.  A chunk's warp starts from its entry of the scan and skips
+//              that one chunk.
 //
 // If the threshold falls outside the bracket, a slot overflows (massive ties at a non-zero
-// value) or the tensor is small, the count kernel runs an exact radix select over the tensor
-// and counts the chunks from the tensor.  The result is exact and unique either way.
+// value) or the tensor is below kStreamMinBytes, the count kernel runs an exact radix select
+// over the tensor and counts the chunks from the tensor (a small tensor is then emitted by
+// compact_small_kernel).  The result is exact and unique either way.
 // Every count fits 32 bits because n <= SURGEON_MAX_N < 2^31.
 #include <cuda.h>
 
