@@ -4,7 +4,8 @@
 // Reshape and gradient steps with Eq. 2:  D[c, o] = sum_k A[k, c] * G[k, o].
 //
 //   c (input channel)  -> MMA M, 128 per CTA (TMEM lanes)
-//   o (output channel) -> MMA N, one or two accumulators of up to 256 columns
+//   o (output channel, per tap for a k x k convolution) -> MMA N, one to three accumulators of
+//                         up to 256 columns, at most 512 in all
 //   k (row t, or image b and position p) -> MMA K, 64 per pipeline stage
 //
 // Operand layouts follow the memory order of the tensors, so that neither needs a transpose:
@@ -16,7 +17,8 @@
 // two tiles in flight: a lane owns a run of 32 consecutive elements (64 bytes of the swizzled
 // tile), finds the rank of its first kept element from the block offset and the block's bitmap
 // words, and rebuilds the run as four 16-byte chunks with one predicated load per element (all
-// independent).  The metadata of a lane's next run is fetched while the current one is rebuilt.
+// independent; fp32 tiles that are mostly kept go through a coalesced per-warp staging copy
+// instead).  The metadata of a lane's next run is fetched while the current one is rebuilt.
 // One thread issues the MMAs, one the TMA loads; split-K partial tiles are reduced in a fixed
 // order by the caller.  Every wait is bounded and ends in SURGEON_ERR_TIMEOUT.
 #include <cuda.h>
