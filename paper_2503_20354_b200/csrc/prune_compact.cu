@@ -610,8 +610,11 @@ __device__ __forceinline__ void for_slot_keys(const typename Elem<DT>::type* __r
 
 // prefix[c] = (elements kept for sure before chunk c) << 31 | (ties at the threshold before it),
 // c = 0 .. chunks (the last entry holds the totals).
+// The fp32 instance is held to 32 registers (a few spills), so that a CTA fits on an SM beside one
+// CTA of another stream's streaming kernel instead of waiting for an empty SM; the bf16 instance
+// would spill three times as much and measured slower that way.
 template <int DT>
-__global__ void __launch_bounds__(kSelThreads, 1)
+__global__ void __launch_bounds__(kSelThreads, DT == 0 ? 2 : 1)
 count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* __restrict__ st,
              surgeon_header* __restrict__ hdr, uint32_t* __restrict__ hist_b,
              uint32_t* __restrict__ hist_fb, const uint32_t* __restrict__ cnt_gt,
