@@ -611,8 +611,10 @@ __device__ __forceinline__ void for_slot_keys(const typename Elem<DT>::type* __r
 // prefix[c] = (elements kept for sure before chunk c) << 31 | (ties at the threshold before it),
 // c = 0 .. chunks (the last entry holds the totals).
 // The fp32 instance is held to 32 registers (a few spills), so that a CTA fits on an SM beside one
-// CTA of another stream's streaming kernel instead of waiting for an empty SM; the bf16 instance
-// would spill three times as much and measured slower that way.
+// CTA of another stream's streaming kernel instead of waiting for an empty SM (those kernels are
+// memory-bound in fp32 and lose nothing to the neighbour).  The bf16 streaming kernels are bound
+// by instruction issue: sharing their SM cost the ViT-shaped stack 6 % even with the spills moved
+// out of the way, so that instance keeps a whole SM.
 template <int DT>
 __global__ void __launch_bounds__(kSelThreads, DT == 0 ? 2 : 1)
 count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* __restrict__ st,
