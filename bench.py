@@ -1,23 +1,34 @@
 #!/usr/bin/env python
 """Benchmark of the dynamic-activation-sparsity hot path on B200.
 
-One step = one pass of the whole path over one batch of the WideResNet-28-10-shaped stack
-(batch 200, 28 conv layers, fp32 activations): per-layer ratios (Eq. 5-7), prune+compact of every
-saved activation (Algorithm 1: prune and decompose steps), and the weight gradient of every layer from its
-compressed store (its Reshape and gradient steps).  Prints ONE JSON line (rank 0).
+One step = one pass of the whole path over one batch of a layer stack: per-layer ratios (Eq. 5-7),
+prune+compact of every saved activation (Algorithm 1: prune and decompose steps), and the weight
+gradient of every layer from its compressed store (its Reshape and gradient steps).  Prints ONE
+JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                  [--workload wrn28|tiny|resnet50|vit|segformer|sweep] [--batch B] [--path tc|fp32]
+                  [--workload all|vit|wrn28|resnet50|resnet50_uniform|tiny|segformer|sweep]
+                  [--batch B] [--path tc|fp32]
+
+The default workload `all` runs, in one process, the ViT-B/16-shaped stack (the headline: `value`,
+`ms_per_step`, `roofline`, `e2e` and `cpu_baseline` are its figures), the WideResNet-28-10-shaped
+and ResNet-50-shaped stacks (the latter with ratios from Eq. 5-7 and with ratios drawn uniformly
+in [0.5, 0.95]) and the largest tensors of the prune+compact bandwidth sweep; every one of them
+reports under `workloads` with a roofline entry for prune+compact (HBM) and one for the weight
+gradient (tensor cores).
 
 N > 1 (launched with torch.distributed.run): every rank runs an independent replica of the
 step on its own GPU (the path has no exchange step); time is the max over ranks.
-`--impl reference` times the CPU oracle on a bounded sample of the same workload (rank 0 only).
+`--impl reference` times the CPU oracle on a bounded sample of the headline workload (rank 0 only).
 """
 from __future__ import annotations
 
 import argparse
+import glob
+import hashlib
 import json
 import os
+import re
 import subprocess
 import sys
 import threading
@@ -32,8 +43,10 @@ import torch
 
 METRIC = "prune+compact GB/s and sparse-act dW TFLOP/s, as % of B200 HBM/tensor peak"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}
 # fp32 CUDA-core peak for the fp32 path: 148 SMs x 128 FMA lanes x 2 flop x 1.965 GHz
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+HEADLINE = "vit"
 
 
 def load_peaks():
@@ -48,8 +61,30 @@ def load_peaks():
     return d
 
 
-# ncu launch lists of one step (profiles/launch_list_*_bench_step.md), weight-gradient kernels only
-DW_STEP_DRAM_BYTES = {"wrn28": 7306000000, "resnet50": 7249000000}
+def kernel_sources_hash() -> str:
+    """Hash of the CUDA sources: DRAM counters taken under ncu hold for the kernels as they were."""
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2503_20354_b200", "csrc")
+    for p in sorted(glob.glob(os.path.join(csrc, "*.cu")) + glob.glob(os.path.join(csrc, "*.cuh"))):
+        with open(p, "rb") as f:
+            h.update(os.path.basename(p).encode() + b"\0" + f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(workload: str, part: str):
+    """DRAM bytes per step (dram__bytes_read.sum + dram__bytes_write.sum over the launches of one
+    step, from an ncu capture) that `profiles/dram_traffic_per_step.md` records for this workload
+    and part ("prune_compact" / "weight_grad"); None when there is no record or the kernels'
+    sources have changed since the counters were taken."""
+    p = os.path.join(ROOT, "profiles", "dram_traffic_per_step.md")
+    if not os.path.exists(p):
+        return None
+    text = open(p).read()
+    m = re.search(r"sources hash:\s*`?([0-9a-f]{16})`?", text)
+    if not m or m.group(1) != kernel_sources_hash():
+        return None
+    m = re.search(r"^\|\s*%s\s*\|\s*%s\s*\|\s*([0-9]+)\s*\|" % (re.escape(workload), re.escape(part)), text, re.M)
+    return int(m.group(1)) if m else None
 
 
 def get_layers(workload: str, batch):
@@ -58,7 +93,7 @@ def get_layers(workload: str, batch):
         return W.wrn28_10(batch or 200), "WideResNet-28-10-shaped stack, 32x32, batch %d, fp32 activations" % (batch or 200)
     if workload == "tiny":
         return W.tiny_conv(batch or 16), "tiny conv 3x3 64->64 on [%d,64,32,32] fp32" % (batch or 16)
-    if workload == "resnet50":
+    if workload in ("resnet50", "resnet50_uniform"):
         return W.resnet50(batch or 64), "ResNet-50-shaped stack, 224x224, batch %d, bf16 activations" % (batch or 64)
     if workload == "vit":
         return W.vit_b16(batch or 64), "ViT-B/16-shaped stack, batch %d, bf16 activations" % (batch or 64)
@@ -67,12 +102,25 @@ def get_layers(workload: str, batch):
     raise SystemExit("unknown workload %r" % workload)
 
 
+# output-gradient scale per workload (the tiny and WideResNet configs: 0.01; ResNet-50 / ViT: 1e-3)
+SIGMA = {"wrn28": 0.01, "tiny": 0.01, "segformer": 0.01, "resnet50": 1e-3, "resnet50_uniform": 1e-3, "vit": 1e-3}
+
+
 def prune_alg_bytes(layer, n_keep: int) -> int:
     """Algorithmic bytes of prune+compact: two reads of the tensor (one to find the threshold,
     one to emit), the bitmap, the packed values and the block offsets."""
     es = 4 if layer.dt == 0 else 2
     n = layer.n_act
     return 2 * n * es + (n + 7) // 8 + n_keep * es + 4 * ((n + 127) // 128 + 1)
+
+
+def dw_min_bytes(layer, n_keep: int) -> int:
+    """Least bytes the weight gradient of a layer moves: the fp32 output gradient once, the
+    compressed store once, the fp32 weight gradient once."""
+    es = 4 if layer.dt == 0 else 2
+    n = layer.n_act
+    store = n_keep * es + (n + 7) // 8 + 4 * ((n + 127) // 128 + 1)
+    return 4 * int(np.prod(layer.grad_shape)) + store + 4 * layer.n_weight
 
 
 class ClockSampler:
@@ -209,14 +257,15 @@ def barrier(world: int):
 class Stack:
     """Device-resident inputs, stores, outputs and scratch of one replica of the workload."""
 
-    def __init__(self, layers, path: int, seed: int, device, worst_case_store=True, n_streams=1):
+    def __init__(self, layers, path: int, seed: int, device, n_streams=1, sigma=0.01, ratios="rule"):
         from paper_2503_20354_b200 import binding as B
         from paper_2503_20354_b200 import workloads as W
         self.B, self.layers, self.path, self.device = B, layers, path, device
         self.gi = W.gradient_importance(len(layers), seed)
         self.lam = np.array([l.act_bytes for l in layers], dtype=np.float64)
+        self.fixed_ratios = W.uniform_ratios(len(layers), seed) if ratios == "uniform" else None
         self.x = [W.activation(l, seed, i, device=device) for i, l in enumerate(layers)]
-        self.g = [W.grad_out(l, seed, i, device=device) for i, l in enumerate(layers)]
+        self.g = [W.grad_out(l, seed, i, sigma=sigma, device=device) for i, l in enumerate(layers)]
         self.desc = [B.layer_desc(l, path) for l in layers]
         self.dw = [torch.empty(l.dw_shape, dtype=torch.float32, device=device) for l in layers]
         # stores sized for ratio 0: ratios change every batch, the buffers do not
@@ -243,65 +292,253 @@ class Stack:
         for st in self.streams:
             main.wait_stream(st)
 
-    def step(self, ev=None):
+    def stream_of(self, k):
+        return self.streams[k] if self.streams else None
+
+    def compute_ratios(self):
+        if self.fixed_ratios is not None:
+            self.ratios = self.fixed_ratios
+        else:
+            self.ratios = self.B.surgeon_layer_ratios(self.gi, self.lam, allow_degenerate=True)   # Eq. 5-7
+        return self.ratios
+
+    def step(self, ev=None, x_ready=None, g_ready=None, dw_done=None):
+        """One pass.  `ev`: three events (start, after the forward loop, end).  The host-buffer leg
+        passes per-layer events: a layer's prune waits for x_ready[i], its weight gradient for
+        g_ready[i], and dw_done[i] is recorded after it."""
         B = self.B
         if ev: ev[0].record()
-        self.ratios = B.surgeon_layer_ratios(self.gi, self.lam, allow_degenerate=True)   # Eq. 5-7
+        self.compute_ratios()
         self._fork()
         for i in range(len(self.layers)):                                                # forward
             k = i % self.n_streams
+            st = self.stream_of(k)
+            if x_ready is not None:
+                (st or torch.cuda.current_stream(self.device)).wait_event(x_ready[i])
             B.surgeon_prune_compact(self.x[i], float(self.ratios[i]), out=self.store[i], workspace=self.ws[k],
-                                    stream=self.streams[k] if self.streams else None)
+                                    stream=st)
         self._join()
         if ev: ev[1].record()
         self._fork()
         for j, i in enumerate(reversed(range(len(self.layers)))):                        # backward
             k = j % self.n_streams
+            st = self.stream_of(k)
+            if g_ready is not None:
+                (st or torch.cuda.current_stream(self.device)).wait_event(g_ready[i])
             B.surgeon_weight_grad(self.store[i], self.desc[i], self.g[i], dw=self.dw[i], workspace=self.ws[k],
-                                  stream=self.streams[k] if self.streams else None)
+                                  stream=st)
+            if dw_done is not None:
+                dw_done[i].record(st or torch.cuda.current_stream(self.device))
         self._join()
         if ev: ev[2].record()
 
+    def per_layer_dw_us(self, reps=3):
+        """Each layer's weight gradient alone on the GPU (one stream, L2 not flushed: a layer's
+        gradient alone exceeds L2 on the large layers), median of `reps`."""
+        B = self.B
+        out = []
+        for i in range(len(self.layers)):
+            ts = []
+            for _ in range(reps + 1):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                B.surgeon_weight_grad(self.store[i], self.desc[i], self.g[i], dw=self.dw[i], workspace=self.ws[0])
+                e1.record()
+                e1.synchronize()
+                ts.append(e0.elapsed_time(e1) * 1e3)
+            out.append(float(np.median(ts[1:])))
+        return out
 
-def run_sweep(args, device):
-    """Prune+compact bandwidth sweep: single tensors of 2^20 .. 2^max elements, fp32 and bf16, four
-    value distributions, four ratios; L2 flushed (256 MB written) before every timed call."""
+
+def frac_entry(kind, achieved, peaks, path_tc=True, traffic=None, extra=None):
+    """A roofline entry.  HBM: against the measured copy bandwidth.  Tensor: against the measured
+    burst cuBLAS bf16 rate (a timed region of a fraction of a second runs at full clock, before
+    the power cap settles), with the sustained and the nominal fractions beside it."""
+    if kind == "hbm":
+        peak = float(peaks["hbm_gbs"])
+        d = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+             "frac": round(achieved / peak, 4), "traffic": traffic,
+             "peak_source": peaks["_source"] + " copy bandwidth",
+             "frac_nominal": round(achieved / NOMINAL["hbm_gbs"], 4)}
+    elif path_tc:
+        peak = float(peaks["bf16_tflops"])
+        sus = float(peaks.get("bf16_tflops_sustained", peak))
+        d = {"bound": "tensor", "achieved": round(achieved, 3), "peak": round(peak, 1), "unit": "TFLOP/s",
+             "frac": round(achieved / peak, 4), "traffic": traffic,
+             "peak_source": peaks["_source"] + " bf16 cuBLAS, burst",
+             "frac_sustained": round(achieved / sus, 4), "peak_sustained": round(sus, 1),
+             "frac_nominal": round(achieved / NOMINAL["bf16_tflops"], 4)}
+    else:
+        d = {"bound": "alu", "achieved": round(achieved, 3), "peak": round(FP32_ALU_TFLOPS, 1), "unit": "TFLOP/s",
+             "frac": round(achieved / FP32_ALU_TFLOPS, 4), "traffic": traffic,
+             "peak_source": "derived: 148 SMs x 128 fp32 FMA lanes x 2 x 1.965 GHz"}
+    if extra:
+        d.update(extra)
+    return d
+
+
+def run_stack(key, args, rank, world, device, peaks, path, keep_stack=False, sampler=None):
+    """Times one layer stack; returns (result dict, stack or None).  `sampler` records the clocks
+    during the timed region."""
+    from paper_2503_20354_b200 import binding as B
+    layers, desc_text = get_layers(key, args.batch)
+    if args.layers:      # profiling aid: keep only the named layers of the stack
+        keep = set(args.layers.split(","))
+        layers = [l for l in layers if l.name in keep]
+        desc_text += " (layers %s only)" % args.layers
+        if len(layers) < 2:
+            raise SystemExit("--layers must name at least two layers of the stack (the ratio rule needs two)")
+    uniform = key == "resnet50_uniform"
+    stack = Stack(layers, path, args.seed + rank, device, n_streams=args.streams, sigma=SIGMA[key],
+                  ratios="uniform" if uniform else "rule")
+    torch.cuda.synchronize()
+    for _ in range(args.warmup):
+        stack.step()
+    torch.cuda.synchronize()
+    barrier(world)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    launches0 = B.surgeon_launch_count()
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    if sampler is not None:
+        sampler.start()
+    t_begin.record()
+    for s in range(args.steps):
+        stack.step(evs[s])
+    t_end.record()
+    torch.cuda.synchronize()
+    barrier(world)
+    launches = B.surgeon_launch_count() - launches0
+    if sampler is not None:
+        res_clocks = sampler.stop()
+    total_ms = max_over_ranks(t_begin.elapsed_time(t_end), world, device)
+    prune_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
+    dw_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
+    ms_per_step = total_ms / args.steps
+    # device-side status of every store (one small read per layer, outside the timed region)
+    for s in stack.store:
+        h = s.read_header()
+        if h.status != 0:
+            raise SystemExit("device status %d in a compressed store" % h.status)
+    flops = sum(l.flops for l in layers)
+    pbytes = sum(prune_alg_bytes(l, s.sizes.n_keep) for l, s in zip(layers, stack.store))
+    stored = sum(s.stored_bytes for s in stack.store)
+    dense = sum(l.act_bytes for l in layers)
+    prune_gbs = pbytes / (prune_ms * 1e-3) / 1e9
+    dw_tflops = flops / (dw_ms * 1e-3) / 1e12
+    full = args.batch is None and args.layers is None
+    tc = path == B.PATH_TENSOR_CORE
+    # per-layer roofline time of the weight gradient: the slower of the tensor cores on the
+    # dense-equivalent flops and HBM on the least bytes (fp32 gradient + store + dW)
+    tpeak = float(peaks["bf16_tflops"]) * 1e12 if tc else FP32_ALU_TFLOPS * 1e12
+    hpeak = float(peaks["hbm_gbs"]) * 1e9
+    roof_us = [max(l.flops / tpeak, dw_min_bytes(l, s.sizes.n_keep) / hpeak) * 1e6
+               for l, s in zip(layers, stack.store)]
+    dw_entry = frac_entry("tensor", dw_tflops, peaks, tc,
+                          recorded_traffic(key, "weight_grad") if (full and tc) else None,
+                          {"kernel": "weight gradient (all layers of one step)", "ms": round(dw_ms, 4), "flops": flops,
+                           "roofline_ms": round(sum(roof_us) / 1e3, 4),
+                           "frac_of_layer_rooflines": round(sum(roof_us) / 1e3 / dw_ms, 4)})
+    pc_entry = frac_entry("hbm", prune_gbs, peaks, True,
+                          recorded_traffic(key, "prune_compact") if full else None,
+                          {"kernel": "surgeon_prune_compact (all kernels of all layers of one step)",
+                           "ms": round(prune_ms, 4), "algorithmic_bytes": pbytes})
+    res = {
+        "workload": desc_text, "layers": len(layers),
+        "ratios": "uniform in [0.5, 0.95]" if uniform else "Eq. 5-7, G_i ~ LogNormal(0,1)",
+        "mean_ratio": round(float(np.mean(stack.ratios)), 4),
+        "ms_per_step": round(ms_per_step, 4), "step_TFLOP/s": round(world * flops / (ms_per_step * 1e-3) / 1e12, 3),
+        "prune_compact": pc_entry, "weight_grad": dw_entry,
+        "store_bytes": stored, "dense_bytes": dense, "gpu_launches": int(launches),
+        "read_GB_per_step": round((dense + sum(g.numel() * 4 for g in stack.g)) / 1e9, 2),
+    }
+    if args.per_layer or key.startswith("resnet50"):
+        us = stack.per_layer_dw_us()
+        res["weight_grad"]["per_layer"] = {
+            "note": "each layer's call alone on one stream; roofline_us = max(flops / tensor peak, least bytes / HBM peak)",
+            "name": [l.name for l in layers], "us": [round(u, 1) for u in us],
+            "roofline_us": [round(r, 1) for r in roof_us],
+            "sum_us": round(sum(us), 1), "sum_roofline_us": round(sum(roof_us), 1),
+            "frac": round(sum(roof_us) / sum(us), 4)}
+    if sampler is not None:
+        res["clocks"] = res_clocks
+    if keep_stack:
+        return res, stack
+    del stack
+    torch.cuda.empty_cache()
+    return res, None
+
+
+SWEEP_DISTS = ("relu_normal", "normal", "student_t2", "ties16")
+SWEEP_RATIOS = (0.1, 0.5, 0.9, 0.99)
+
+
+def run_sweep_cases(args, device, peaks, sizes, dists, ratios, steps, warmup):
+    """Prune+compact on single tensors of 2^lg elements, fp32 and bf16; L2 flushed (256 MB written)
+    before every timed call.  Returns the list of cases."""
     from paper_2503_20354_b200 import binding as B
     from paper_2503_20354_b200 import workloads as W
-    peaks = load_peaks()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
-    sizes = [20, 22, 24, 26, 28, 30][: args.sweep_sizes]
     cases = []
-    launches0 = B.surgeon_launch_count()
     for bf16 in (False, True):
         for lg in sizes:
             n = 1 << lg
             es = 2 if bf16 else 4
-            for dist in ("relu_normal", "normal", "student_t2", "ties16"):
+            for dist in dists:
                 x = W.draw(dist, n, args.seed, device=device)
                 if bf16:
                     x = x.to(torch.bfloat16)
                 out = B.CompressedActivation(n, B.dtype_code(x.dtype), 0.0, device)
                 ws = torch.empty(out.sizes.workspace_bytes, dtype=torch.uint8, device=device)
-                for ratio in (0.1, 0.5, 0.9, 0.99):
+                for ratio in ratios:
                     ts = []
-                    for it in range(args.warmup + args.steps):
+                    for it in range(warmup + steps):
                         flush.zero_()
                         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                         e0.record()
                         B.surgeon_prune_compact(x, ratio, out=out, workspace=ws)
                         e1.record()
                         e1.synchronize()
-                        if it >= args.warmup:
+                        if it >= warmup:
                             ts.append(e0.elapsed_time(e1))
                     ms = float(np.median(ts))
                     k = out.sizes.n_keep
                     balg = 2 * n * es + n // 8 + k * es + 4 * (n // 128 + 1)
                     if out.read_header().status != 0:
                         raise SystemExit("device status in sweep case")
+                    gbs = balg / ms / 1e6
                     cases.append({"dtype": "bf16" if bf16 else "f32", "log2_n": lg, "dist": dist, "ratio": ratio,
-                                  "us": round(ms * 1e3, 1), "GB/s": round(balg / ms / 1e6, 1)})
+                                  "us": round(ms * 1e3, 1), "GB/s": round(gbs, 1),
+                                  "frac": round(gbs / float(peaks["hbm_gbs"]), 4)})
                 del x, out, ws
+    del flush
+    torch.cuda.empty_cache()
+    return cases
+
+
+def sweep_summary(cases, peaks, sizes):
+    """Median GB/s per dtype at the largest size, as roofline entries (ties16 apart: it takes the
+    exact fall-back select)."""
+    out = {"l2": "flushed before every call", "cases": cases}
+    top = sizes[-1]
+    for dt in ("f32", "bf16"):
+        main = [c["GB/s"] for c in cases if c["dtype"] == dt and c["log2_n"] == top and c["dist"] != "ties16"]
+        ties = [c["GB/s"] for c in cases if c["dtype"] == dt and c["log2_n"] == top and c["dist"] == "ties16"]
+        if main:
+            out["%s_2^%d" % (dt, top)] = frac_entry("hbm", float(np.median(main)), peaks, True, None,
+                                                    {"kernel": "surgeon_prune_compact (all kernels of a call)",
+                                                     "min_GB/s": round(min(main), 1), "max_GB/s": round(max(main), 1)})
+        if ties:
+            out["%s_2^%d_ties16" % (dt, top)] = {"min_GB/s": round(min(ties), 1), "max_GB/s": round(max(ties), 1)}
+    return out
+
+
+def run_sweep_line(args, device, peaks):
+    from paper_2503_20354_b200 import binding as B
+    sizes = [20, 22, 24, 26, 28, 30][: args.sweep_sizes]
+    launches0 = B.surgeon_launch_count()
+    cases = run_sweep_cases(args, device, peaks, sizes, SWEEP_DISTS, SWEEP_RATIOS, args.steps, args.warmup)
+    summ = sweep_summary(cases, peaks, sizes)
     big = [c["GB/s"] for c in cases if c["log2_n"] == sizes[-1]]
     val = float(np.median(big))
     print(json.dumps({
@@ -310,10 +547,8 @@ def run_sweep(args, device):
         "vs_baseline": None, "dtype": "u32", "data": "synthetic",
         "config": {"workload": "prune+compact sweep, 2^20..2^%d elements, fp32 and bf16" % sizes[-1],
                    "l2": "flushed before every call"},
-        "roofline": {"kernel": "surgeon_prune_compact (all kernels of a call)", "bound": "hbm", "achieved": round(val, 1),
-                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(val / float(peaks["hbm_gbs"]), 4),
-                     "traffic": None, "peak_source": peaks["_source"] + " copy bandwidth"},
-        "gpu_launches": int(B.surgeon_launch_count() - launches0), "cases": cases}))
+        "roofline": frac_entry("hbm", val, peaks, True, None, {"kernel": "surgeon_prune_compact (all kernels of a call)"}),
+        "gpu_launches": int(B.surgeon_launch_count() - launches0), "sweep": summ}))
 
 
 def run_ours(args, rank, world, local):
@@ -322,106 +557,74 @@ def run_ours(args, rank, world, local):
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     B.lib()
     device = torch.device("cuda", local if world > 1 else 0)
+    peaks = load_peaks()
     if args.workload == "sweep":
         if rank == 0:
-            run_sweep(args, device)
+            run_sweep_line(args, device, peaks)
         return
-    layers, desc_text = get_layers(args.workload, args.batch)
-    if args.layers:      # profiling aid: keep only the named layers of the stack
-        keep = set(args.layers.split(","))
-        layers = [l for l in layers if l.name in keep]
-        desc_text += " (layers %s only)" % args.layers
-        if len(layers) < 2:
-            raise SystemExit("--layers must name at least two layers of the stack (the ratio rule needs two)")
     path = B.PATH_FP32 if args.path == "fp32" else B.PATH_TENSOR_CORE
-    stack = Stack(layers, path, args.seed + rank, device, n_streams=args.streams)
-    torch.cuda.synchronize()
-    peaks = load_peaks()
-
-    for _ in range(args.warmup):
-        stack.step()
-    torch.cuda.synchronize()
-    barrier(world)
+    head_key = HEADLINE if args.workload == "all" else args.workload
+    others = ["wrn28", "resnet50", "resnet50_uniform"] if args.workload == "all" else []
 
     sampler = ClockSampler(local if world > 1 else 0)
-    sampler.start()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    launches0 = B.surgeon_launch_count()
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    t_begin.record()
-    for s in range(args.steps):
-        stack.step(evs[s])
-    t_end.record()
-    torch.cuda.synchronize()
-    barrier(world)
-    launches = B.surgeon_launch_count() - launches0
-    clocks = sampler.stop()
-    total_ms = max_over_ranks(t_begin.elapsed_time(t_end), world, device)
-    prune_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
-    dw_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
-    ms_per_step = total_ms / args.steps
-
-    # device-side status of every store (one small read per layer, outside the timed region)
-    for s in stack.store:
-        h = s.read_header()
-        if h.status != 0:
-            raise SystemExit("device status %d in a compressed store" % h.status)
-
+    head, stack = run_stack(head_key, args, rank, world, device, peaks, path, keep_stack=True, sampler=sampler)
+    clocks = head.pop("clocks")
+    layers = stack.layers
     flops = sum(l.flops for l in layers)
-    pbytes = sum(prune_alg_bytes(l, s.sizes.n_keep) for l, s in zip(layers, stack.store))
-    stored = sum(s.stored_bytes for s in stack.store)
-    dense = sum(l.act_bytes for l in layers)
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
-    prune_gbs = pbytes / (prune_ms * 1e-3) / 1e9
-    dw_tflops = flops / (dw_ms * 1e-3) / 1e12
-    if path == B.PATH_TENSOR_CORE:
-        peak, bound, unit = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])), "tensor", "TFLOP/s"
-        peak_note = "%s bf16 cuBLAS, sustained" % peaks["_source"]
-    else:
-        peak, bound, unit = FP32_ALU_TFLOPS, "alu", "TFLOP/s"
-        peak_note = "derived: 148 SMs x 128 fp32 FMA lanes x 2 x 1.965 GHz"
-    # DRAM bytes the weight-gradient kernels of one step moved under ncu (dram__bytes_read.sum +
-    # dram__bytes_write.sum summed over their launches): known for the full-size stacks on the
-    # tensor-core path only, and only while those kernels are the ones the counters were taken on.
-    traffic = None
-    if path == B.PATH_TENSOR_CORE and args.batch is None and args.layers is None:
-        traffic = DW_STEP_DRAM_BYTES.get(args.workload)
-    roofline = {"kernel": "weight gradient (all layers of one step)", "bound": bound,
-                "achieved": round(dw_tflops, 3), "peak": round(peak, 1), "unit": unit,
-                "frac": round(dw_tflops / peak, 4), "traffic": traffic, "peak_source": peak_note}
-
     # ---- end to end through the C ABI with host buffers --------------------------------------
     e2e = run_e2e(stack, layers, args, world, device, flops) if args.e2e else None
+    del stack
+    torch.cuda.empty_cache()
 
+    results = {head_key: head}
+    for key in others:
+        results[key], _ = run_stack(key, args, rank, world, device, peaks, path)
+    if args.workload == "all" and rank == 0:
+        # the top of the bandwidth sweep: 2^28 and 2^30 elements, three distributions, two ratios
+        # (+ the many-ties case at one ratio), 5 timed calls each
+        sizes = [28, 30]
+        cases = run_sweep_cases(args, device, peaks, sizes, ("relu_normal", "normal", "student_t2"), (0.5, 0.9), 5, 3)
+        cases += run_sweep_cases(args, device, peaks, sizes, ("ties16",), (0.9,), 5, 3)
+        results["sweep"] = sweep_summary(cases, peaks, sizes)
+        for lg in sizes[:-1]:
+            for dt in ("f32", "bf16"):
+                sub = [c["GB/s"] for c in cases if c["dtype"] == dt and c["log2_n"] == lg and c["dist"] != "ties16"]
+                results["sweep"]["%s_2^%d" % (dt, lg)] = frac_entry("hbm", float(np.median(sub)), peaks, True, None,
+                                                                   {"min_GB/s": round(min(sub), 1), "max_GB/s": round(max(sub), 1)})
+    barrier(world)
+
+    roofline = dict(head["weight_grad"])
+    roofline.pop("per_layer", None)
     out = {
-        "metric": METRIC, "value": round(value, 3), "unit": "TFLOP/s (dense-equivalent dW flops / whole-step time)",
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4),
+        "metric": METRIC, "value": head["step_TFLOP/s"], "unit": "TFLOP/s (dense-equivalent dW flops / whole-step time)",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": head["ms_per_step"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if path == B.PATH_TENSOR_CORE else "f32", "data": "synthetic",
-        "config": {"workload": desc_text, "layers": len(layers), "ratios": "GI/LAM rule, GI~LogNormal(0,1)",
-                   "path": args.path, "l2": "inputs larger than L2 (%.2f GB read per step)" % ((dense + sum(g.numel() * 4 for g in stack.g)) / 1e9),
-                   "replicas": world, "streams": stack.n_streams},
-        "parts": {
-            "prune_compact": {"ms": round(prune_ms, 4), "GB/s": round(prune_gbs, 1),
-                              "frac_hbm": round(prune_gbs / float(peaks["hbm_gbs"]), 4),
-                              "peak_GB/s": peaks["hbm_gbs"], "peak_source": peaks["_source"] + " copy bandwidth",
-                              "algorithmic_bytes": pbytes},
-            "weight_grad": {"ms": round(dw_ms, 4), "TFLOP/s": round(dw_tflops, 3), "flops": flops},
-            "store_bytes": stored, "dense_bytes": dense, "mean_ratio": float(np.mean(stack.ratios)),
-        },
-        "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+        "config": {"workload": head["workload"], "layers": head["layers"], "ratios": head["ratios"],
+                   "path": args.path, "l2": "inputs larger than L2 (%.2f GB read per step)" % head["read_GB_per_step"],
+                   "replicas": world, "streams": args.streams,
+                   "also_timed": [k for k in results if k != head_key]},
+        "roofline": roofline,
+        "roofline_prune_compact": head["prune_compact"],
+        "workloads": results,
+        "e2e": e2e, "gpu_launches": int(sum(r.get("gpu_launches", 0) for r in results.values() if isinstance(r, dict))),
+        "clocks": clocks,
     }
     if rank == 0:
         if args.cpu_baseline:
-            out["cpu_baseline"] = cpu_baseline(args, budget_s=20.0)
+            args_head = argparse.Namespace(**vars(args))
+            args_head.workload = head_key
+            out["cpu_baseline"] = cpu_baseline(args_head, budget_s=20.0)
         print(json.dumps(out))
 
 
 def run_e2e(stack, layers, args, world, device, flops):
-    """Same step with HOST inputs: per step, pinned host activations and gradients are copied in,
-    the path runs, and every dW is copied back to pinned host memory."""
+    """The same step with HOST inputs: per step every activation and output gradient is copied in
+    from pinned host memory and every dW is copied back to pinned host memory.  The copies run on
+    their own streams in layer order; a layer's kernels wait only for that layer's tensors, so
+    the transfers of later layers overlap the work on earlier ones."""
     steps = max(1, min(args.steps, args.e2e_steps))
+    n = len(layers)
     hx = [torch.empty(x.shape, dtype=x.dtype).pin_memory() for x in stack.x]
     hg = [torch.empty(g.shape, dtype=g.dtype).pin_memory() for g in stack.g]
     hdw = [torch.empty(d.shape, dtype=d.dtype).pin_memory() for d in stack.dw]
@@ -430,13 +633,28 @@ def run_e2e(stack, layers, args, world, device, flops):
     torch.cuda.synchronize()
     h2d = sum(t.numel() * t.element_size() for t in hx + hg)
     d2h = sum(t.numel() * t.element_size() for t in hdw)
+    s_in, s_out = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)
+    main = torch.cuda.current_stream(device)
 
     def one():
-        for d, h in zip(stack.x + stack.g, hx + hg):
-            d.copy_(h, non_blocking=True)
-        stack.step()
-        for h, d in zip(hdw, stack.dw):
-            h.copy_(d, non_blocking=True)
+        x_ready = [torch.cuda.Event() for _ in range(n)]
+        g_ready = [torch.cuda.Event() for _ in range(n)]
+        dw_done = [torch.cuda.Event() for _ in range(n)]
+        s_in.wait_stream(main)
+        with torch.cuda.stream(s_in):
+            for i in range(n):                       # forward order
+                stack.x[i].copy_(hx[i], non_blocking=True)
+                x_ready[i].record(s_in)
+            for i in reversed(range(n)):             # backward order
+                stack.g[i].copy_(hg[i], non_blocking=True)
+                g_ready[i].record(s_in)
+        stack.step(x_ready=x_ready, g_ready=g_ready, dw_done=dw_done)
+        with torch.cuda.stream(s_out):
+            for i in reversed(range(n)):
+                s_out.wait_event(dw_done[i])
+                hdw[i].copy_(stack.dw[i], non_blocking=True)
+        main.wait_stream(s_out)
+        main.wait_stream(s_in)
 
     one()
     torch.cuda.synchronize()
@@ -450,7 +668,8 @@ def run_e2e(stack, layers, args, world, device, flops):
     barrier(world)
     ms = max_over_ranks(b.elapsed_time(e), world, device) / steps
     return {"value": round(world * flops / (ms * 1e-3) / 1e12, 4), "unit": "TFLOP/s", "ms_per_step": round(ms, 3),
-            "steps": steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
+            "steps": steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "note": "PCIe-bound: copies of later layers overlap the kernels of earlier ones"}
 
 
 # ------------------------------------------------------------------------------------------
@@ -485,7 +704,7 @@ def oracle_sample(args, budget_s: float, grow: bool = False):
     while True:
         idx = list(range(0, len(small), stride))
         layers = [small[i] for i in idx]
-        inputs = [(W.as_numpy_bits(W.activation(small[i], args.seed, i)), W.grad_out(small[i], args.seed, i).numpy())
+        inputs = [(W.as_numpy_bits(W.activation(small[i], args.seed, i)), W.grad_out(small[i], args.seed, i, sigma=SIGMA.get(args.workload, 0.01)).numpy())
                   for i in idx]
         t0 = time.perf_counter()
         oracle_step(layers, inputs, ratios[idx])
@@ -539,11 +758,12 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="wrn28", choices=["wrn28", "tiny", "resnet50", "vit", "segformer", "sweep"])
-    ap.add_argument("--sweep-sizes", type=int, default=5, help="how many of 2^20,22,24,26,28,30 the sweep covers")
+    ap.add_argument("--workload", default="all",
+                    choices=["all", "vit", "wrn28", "resnet50", "resnet50_uniform", "tiny", "segformer", "sweep"])
+    ap.add_argument("--sweep-sizes", type=int, default=6, help="how many of 2^20,22,24,26,28,30 the sweep covers")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--layers", default=None, help="comma-separated layer names: run only these (profiling)")
     ap.add_argument("--path", default="tc", choices=["tc", "fp32"])
@@ -551,11 +771,14 @@ def main():
     ap.add_argument("--streams", type=int, default=8,
                     help="streams the independent layers are issued on (1 = the caller's stream only)")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--per-layer", action="store_true", help="time every layer's weight gradient alone as well")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--no-e2e", dest="e2e", action="store_false", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
+        if args.workload in ("all", "sweep"):
+            args.workload = HEADLINE
         rank = int(os.environ.get("RANK", "0"))
         run_reference(args, rank, int(os.environ.get("WORLD_SIZE", "1")))
         return

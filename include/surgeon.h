@@ -22,7 +22,8 @@
  *     void*; NULL = the legacy default stream).
  *   - Conditions that only the device can see (a bounded wait that ran out, an
  *     internal count that does not add up) are reported in
- *     surgeon_header::status, never by a trap.
+ *     surgeon_header::status, never by a trap.  Once one is seen, the kernels of
+ *     that call that have not run yet store nothing to the outputs.
  *   - Flat index j of an activation element = its row-major index in the tensor
  *     as given: NCHW for conv2d inputs, [T, C] for linear inputs.
  */
@@ -171,6 +172,13 @@ surgeon_status surgeon_prune_compact(const void* x, int64_t n, surgeon_dtype dt,
  * surgeon_prune_compact.  Unknown flag bits: INVALID_ARG.
  * ---------------------------------------------------------------------------------------- */
 #define SURGEON_STORE_DROP_ZEROS 1u
+/* Diagnostic without a counterpart in the paper, for testing the error path of the bounded
+ * device-side waits: the select's grid-wide barrier is given an arrival target it cannot reach
+ * and a cap of 1024 polls, so it gives up after some tens of microseconds.  Every kernel of the
+ * call then returns without storing to bitmap, values or block_offsets, and
+ * surgeon_header::status reads SURGEON_ERR_TIMEOUT; the other header fields are undefined.
+ * Nothing faults and nothing spins past the cap. */
+#define SURGEON_DEBUG_STALL_BARRIER 0x80000000u
 surgeon_status surgeon_prune_compact_flags(const void* x, int64_t n, surgeon_dtype dt, double ratio,
                                            uint32_t flags, surgeon_compressed* out, void* workspace,
                                            size_t workspace_bytes, void* cuda_stream);
@@ -189,8 +197,11 @@ surgeon_status surgeon_prune_compact_flags(const void* x, int64_t n, surgeon_dty
  *     SURGEON_ERR_UNSUPPORTED before anything is launched (use surgeon_prune_compact with your
  *     own workspace for such tensors);
  *   - the first call on each device looks up the array's device address (one host-side
- *     runtime query, with that device current).  Make that first call outside any stream
- *     capture; later calls on the device do no set-up;
+ *     runtime query, with that device current) and keeps it for the life of the process: the
+ *     one exception to "keeps no pointer after a call returns".  Make that first call outside
+ *     any stream capture; later calls on the device do no set-up.  The kept address does not
+ *     survive cudaDeviceReset (or any other teardown of the device's primary context): do not
+ *     call this entry point on a device after resetting it;
  *   - all calls on one device share the one array.  Each call clears what it needs before use,
  *     so calls that follow each other on a stream, or are otherwise ordered, are independent;
  *     two calls whose kernels can run at the same time on one GPU (different streams without an

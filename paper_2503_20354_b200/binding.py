@@ -119,6 +119,16 @@ def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
     return int(s.cuda_stream)
 
 
+def _scratch(nbytes: int, device, stream: Optional[torch.cuda.Stream]) -> torch.Tensor:
+    """A scratch tensor made here (the caller passed none).  It is dropped when the call returns,
+    while the kernels that use it are still queued on ``stream``: the allocator is told, so that
+    the block is not handed out again before they are done."""
+    t = torch.empty(max(int(nbytes), 16), dtype=torch.uint8, device=device)
+    if stream is not None:
+        t.record_stream(stream)
+    return t
+
+
 def dtype_code(t: torch.dtype) -> int:
     if t == torch.float32:
         return SURGEON_F32
@@ -173,7 +183,7 @@ def surgeon_gradient_importance(dw: torch.Tensor, out: Optional[torch.Tensor] = 
     if out is None:
         out = torch.empty(1, dtype=torch.float64, device=dw.device)
     if workspace is None:
-        workspace = torch.empty(SURGEON_GI_WORKSPACE_BYTES, dtype=torch.uint8, device=dw.device)
+        workspace = _scratch(SURGEON_GI_WORKSPACE_BYTES, dw.device, stream)
     st = lib().surgeon_gradient_importance(dw.data_ptr() if dw.numel() else None, dw.numel(),
                                            out.data_ptr(), workspace.data_ptr(),
                                            workspace.numel() * workspace.element_size(),
@@ -244,6 +254,7 @@ class CompressedActivation:
 
 
 SURGEON_STORE_DROP_ZEROS = 1
+SURGEON_DEBUG_STALL_BARRIER = 0x80000000
 
 
 def surgeon_prune_compact(x: torch.Tensor, ratio: float, out: Optional[CompressedActivation] = None,
@@ -265,7 +276,7 @@ def surgeon_prune_compact(x: torch.Tensor, ratio: float, out: Optional[Compresse
             raise ValueError("output store does not fit this tensor / ratio")
         out.ratio, out.sizes = float(ratio), sizes
     if workspace is None:
-        workspace = torch.empty(sizes.workspace_bytes, dtype=torch.uint8, device=x.device)
+        workspace = _scratch(sizes.workspace_bytes, x.device, stream)
     st = lib().surgeon_prune_compact_flags(x.data_ptr(), n, dt, float(ratio), int(flags), C.byref(out.c),
                                            workspace.data_ptr(),
                                            workspace.numel() * workspace.element_size(),
@@ -306,6 +317,8 @@ def surgeon_decompress(act: CompressedActivation, stream: Optional[torch.cuda.St
     """Dense flat tensor rebuilt from the store (test utility; Algorithm 1: Reshape step)."""
     vt = torch.float32 if act.dt == SURGEON_F32 else torch.bfloat16
     out = torch.empty(max(act.n, 1), dtype=vt, device=act.bitmap.device)
+    if stream is not None:
+        out.record_stream(stream)
     st = lib().surgeon_decompress(C.byref(act.c), out.data_ptr(), _stream_ptr(stream))
     _check(st, "surgeon_decompress")
     return out[: act.n]
@@ -339,7 +352,7 @@ def surgeon_weight_grad(act: CompressedActivation, desc: LayerDesc, grad_out: to
         dw = torch.empty(shape, dtype=torch.float32, device=grad_out.device)
     need = surgeon_weight_grad_workspace(desc)
     if workspace is None:
-        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=grad_out.device)
+        workspace = _scratch(need, grad_out.device, stream)
     st = lib().surgeon_weight_grad(C.byref(act.c), C.byref(desc), grad_out.data_ptr(), dw.data_ptr(),
                                    1 if accumulate else 0, workspace.data_ptr(),
                                    workspace.numel() * workspace.element_size(), _stream_ptr(stream))

@@ -181,7 +181,8 @@ surgeon_status surgeon_prune_compact(const void* x, int64_t n, surgeon_dtype dt,
 surgeon_status surgeon_prune_compact_flags(const void* x, int64_t n, surgeon_dtype dt, double ratio,
                                            uint32_t flags, surgeon_compressed* out, void* workspace,
                                            size_t workspace_bytes, void* cuda_stream) {
-  if (flags & ~static_cast<uint32_t>(SURGEON_STORE_DROP_ZEROS)) return SURGEON_ERR_INVALID_ARG;
+  if (flags & ~static_cast<uint32_t>(SURGEON_STORE_DROP_ZEROS | SURGEON_DEBUG_STALL_BARRIER))
+    return SURGEON_ERR_INVALID_ARG;
   if (!out || n < 0 || !(ratio >= 0.0 && ratio <= 1.0) ||
       (dt != SURGEON_F32 && dt != SURGEON_BF16))
     return SURGEON_ERR_INVALID_ARG;
@@ -199,7 +200,8 @@ surgeon_status surgeon_prune_compact_flags(const void* x, int64_t n, surgeon_dty
   out->reserved = 0;
   const cudaError_t e = launch_prune_compact(x, n, static_cast<int>(dt), k, *out, workspace,
                                              static_cast<cudaStream_t>(cuda_stream),
-                                             (flags & SURGEON_STORE_DROP_ZEROS) ? 1 : 0);
+                                             (flags & SURGEON_STORE_DROP_ZEROS) ? 1 : 0,
+                                             (flags & SURGEON_DEBUG_STALL_BARRIER) ? 1 : 0);
   return e == cudaSuccess ? SURGEON_OK : SURGEON_ERR_CUDA;
 }
 

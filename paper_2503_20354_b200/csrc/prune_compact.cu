@@ -566,21 +566,28 @@ __device__ __forceinline__ void load_tile(const typename Elem<DT>::type* __restr
 // ---- threshold (where still open), per-chunk counts, exclusive scan ------------------------------
 // Launched cooperatively (all CTAs resident), so that the steps can be separated by grid-wide
 // barriers: a counter every CTA increments and then polls, with a bounded number of polls.
-__device__ __forceinline__ void grid_barrier(SelectState* st, uint32_t& epoch) {
+// Returns false when the wait gave up (uniform over the CTA); the caller then leaves the kernel.
+// `stall` is the diagnostic of SURGEON_DEBUG_STALL_BARRIER: the arrival target is one more than
+// the CTAs that exist and the poll cap is 1024, so the wait is certain to run out, quickly.
+__device__ __forceinline__ bool grid_barrier(SelectState* st, uint32_t& epoch, bool stall = false) {
+  __shared__ uint32_t s_ok;
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
     atomicAdd(&st->barrier_count, 1u);
     ++epoch;
-    const uint32_t target = epoch * gridDim.x;
-    uint32_t spins = 0;
+    const uint32_t target = epoch * gridDim.x + (stall ? 1u : 0u);
+    const uint32_t cap = stall ? 1024u : (1u << 22);
+    uint32_t spins = 0, ok = 1;
     while (*reinterpret_cast<volatile uint32_t*>(&st->barrier_count) < target) {
-      if (++spins > (1u << 22)) { atomicMax(&st->error, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); break; }
+      if (++spins > cap) { atomicMax(&st->error, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); ok = 0; break; }
       __nanosleep(40);
     }
     __threadfence();
+    s_ok = ok;
   }
   __syncthreads();
+  return s_ok != 0u;
 }
 
 // Calls f(key) for the first `cc` keys of chunk c's slot; one thread, 16-byte loads, four in flight.
@@ -624,13 +631,14 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
              unsigned long long* __restrict__ val, unsigned long long* __restrict__ prefix,
              unsigned long long* __restrict__ partial, int tiles,
              uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
-             uint32_t* __restrict__ offsets, int drop_zeros) {
+             uint32_t* __restrict__ offsets, int drop_zeros, int stall) {
   using E = typename Elem<DT>::type;
   constexpr uint32_t kMask = Elem<DT>::kKeyMask;
   constexpr int EPV = 16 / sizeof(E);
   constexpr long long kChunkElems = static_cast<long long>(kTileVecs) * EPV;
   __shared__ uint32_t s_hist[kBinsB];          // level B / fall-back digit histogram
   __shared__ int s_bnd;                        // the chunk inside which the tie quota ends, if this CTA owns it
+  __shared__ uint32_t s_err;                   // a bounded wait of this call has given up
   __shared__ unsigned long long s_bnd_prefix;
   __shared__ uint32_t scratch[32];
   __shared__ uint32_t res[2];
@@ -644,6 +652,9 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
   const uint32_t mode = __ldcg(&st->mode);
   uint32_t tau = 0, n_greater = 0;
   if (tid == 0) s_bnd = -1;                    // read after several barriers below
+  // A barrier that gave up: the CTA reports it and leaves before it stores anything to the
+  // outputs (the CTAs still waiting for it run out of polls in turn).
+  auto leave = [&]() { if (tid == 0) atomicMax(&hdr->status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); };
 
   if (mode == 1u) {
     // ---- fall-back: exact radix select over the tensor itself, one digit per round ----
@@ -683,7 +694,7 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
       uint32_t* gh = hist_fb + round * kFbBins;
       for (int i = tid; i < kFbBins; i += kSelThreads)
         if (s_hist[i]) atomicAdd(&gh[i], s_hist[i]);
-      grid_barrier(st, epoch);
+      if (!grid_barrier(st, epoch, stall != 0)) { leave(); return; }
       for (int i = tid; i < kFbBins; i += kSelThreads) s_hist[i] = __ldcg(gh + i);
       __syncthreads();
       find_from_top<kFbBins>([&](int i) { return s_hist[i]; }, rank, scratch, res);
@@ -708,7 +719,7 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
           if ((rel >> shift) == pre) atomicAdd(&gh[(rel >> ns) & ((1u << nb) - 1u)], 1u);
         });
       }
-      grid_barrier(st, epoch);
+      if (!grid_barrier(st, epoch, stall != 0)) { leave(); return; }
       for (int i = tid; i < kFbBins; i += kSelThreads) s_hist[i] = __ldcg(gh + i);
       __syncthreads();
       find_from_top<kFbBins>([&](int i) { return s_hist[i]; }, rank, scratch, res);
@@ -797,7 +808,7 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
     for (int w = 0; w < 32; ++w) t += s_tot[w];
     partial[blockIdx.x] = t;
   }
-  grid_barrier(st, epoch);
+  if (!grid_barrier(st, epoch, stall != 0)) { leave(); return; }
 
   // ---- exclusive scan: carry from the CTAs before, then warp w scans a sub-range ----
   unsigned long long carry = 0;
@@ -840,8 +851,11 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
   }
   // The chunk inside which the tie quota ends is emitted here, with its ties ranked by index, by
   // the first two warps of the CTA that owns it; the compaction kernels skip that chunk.
+  // Nothing is stored to the outputs once a bounded wait has given up anywhere in this call (the
+  // counts the offsets come from may then be incomplete).
+  if (tid == 0) s_err = *reinterpret_cast<volatile uint32_t*>(&st->error);
   __syncthreads();
-  if (s_bnd >= 0 && warp < kTileWarps) {
+  if (s_err == 0u && s_bnd >= 0 && warp < kTileWarps) {
     const unsigned long long pb = s_bnd_prefix;
     uint4 q[kRows];
     load_tile<DT>(x, n, s_bnd, q);
@@ -862,7 +876,12 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
       const long long gt_all = static_cast<long long>(total >> 31);
       const long long eq_all = static_cast<long long>(total & 0x7FFFFFFFull);
       const long long ng = (mode == 2u) ? hdr->n_greater : static_cast<long long>(n_greater);
-      if (gt_all != ng || eq_all < static_cast<long long>(k) - gt_all)
+      const long long want = nz ? ng : static_cast<long long>(k);
+      const long long kept = gt_all + (eq_all < quota ? eq_all : quota);
+      // every mode and every barrier of this kernel is behind us: whatever gave up shows now
+      const uint32_t err = *reinterpret_cast<volatile uint32_t*>(&st->error);
+      if (err) atomicMax(&hdr->status, err);
+      else if (gt_all != ng || kept != want)
         atomicMax(&hdr->status, static_cast<uint32_t>(SURGEON_ERR_INTERNAL));
     }
   }
@@ -1058,18 +1077,30 @@ __device__ __forceinline__ void load_tile(const typename Elem<DT>::type* __restr
   }
 }
 
+// True when a bounded wait of the select gave up or a self-check failed (uniform over the CTA); the
+// status reaches the header, and the caller stores nothing: offsets taken from incomplete counts
+// could point past the end of `values`.
+__device__ __forceinline__ bool gave_up(surgeon_header* __restrict__ hdr, const uint32_t* __restrict__ err) {
+  const uint32_t e = __ldcg(err);
+  const uint32_t s = *reinterpret_cast<volatile uint32_t*>(&hdr->status);
+  if (e && threadIdx.x == 0) atomicMax(&hdr->status, e);
+  return (e | s) != 0u;
+}
+
 // One small CTA per tile: used for tensors too small for the streaming kernel.  The one tile
 // inside which the tie quota ends (if any) is left to the count kernel.
 template <int DT>
 __global__ void __launch_bounds__(kCompactThreads)
 compact_small_kernel(const void* __restrict__ xv, long long n, surgeon_header* __restrict__ hdr,
                uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
-               uint32_t* __restrict__ offsets, const unsigned long long* __restrict__ prefix) {
+               uint32_t* __restrict__ offsets, const unsigned long long* __restrict__ prefix,
+               const uint32_t* __restrict__ err) {
   using E = typename Elem<DT>::type;
   const E* __restrict__ x = reinterpret_cast<const E*>(xv);
   const int tile = blockIdx.x;
   uint4 q[kRows];
   load_tile<DT>(x, n, tile, q);     // in flight while the header and the scan entries arrive
+  if (gave_up(hdr, err)) return;    // the scan may be incomplete: store nothing
   const uint32_t tau = hdr->threshold_key;
   const long long quota = hdr->tie_quota;
   const unsigned long long pb = prefix[tile], pe = prefix[tile + 1];
@@ -1091,7 +1122,7 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
                       long long n, long long n_rows_full, surgeon_header* __restrict__ hdr,
                       uint32_t* __restrict__ bitmap, void* __restrict__ values_v,
                       uint32_t* __restrict__ offsets, const unsigned long long* __restrict__ prefix,
-                      int n_chunks, int n_stage_tiles) {
+                      const uint32_t* __restrict__ err, int n_chunks, int n_stage_tiles) {
   using E = typename Elem<DT>::type;
   constexpr uint32_t kMask = Elem<DT>::kKeyMask;
   constexpr int EPR = 128 / sizeof(E);         // elements per row (= per lane): 32 / 64
@@ -1109,6 +1140,7 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
   const uint32_t lane = lane_id();
   const uint32_t full_bar = smem_u32(bars);
   const uint32_t empty_bar = smem_u32(bars + kCsStages);
+  if (gave_up(hdr, err)) return;   // before any load or store; the whole CTA takes the same way
   if (threadIdx.x == 0) {
     tc::tma_prefetch_desc(&xmap);
     for (int s = 0; s < kCsStages; ++s) {
@@ -1386,7 +1418,7 @@ bool make_row_map(const void* x, long long n_rows_full, CUtensorMap* map) {
 }
 
 template <int DT>
-cudaError_t run_prune_compact(const void* x, long long n, long long k, int drop_zeros,
+cudaError_t run_prune_compact(const void* x, long long n, long long k, int drop_zeros, int stall,
                               const surgeon_compressed& out, void* workspace,
                               cudaStream_t stream) {
   using E = typename Elem<DT>::type;
@@ -1479,7 +1511,7 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k, int drop_
       void* vals = out.values;
       uint32_t* offs = out.block_offsets;
       void* args[] = {&xa, &na, &ka, &st, &hdr, &hist_b, &hist_fb, &cg, &cc, &sl, &val, &prefix,
-                      &partial, &tiles, &bm, &vals, &offs, &drop_zeros};
+                      &partial, &tiles, &bm, &vals, &offs, &drop_zeros, &stall};
       e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(count_kernel<DT>), dim3(grid),
                                       dim3(kSelThreads), args, 0, stream);
       if (e != cudaSuccess) return e;
@@ -1493,10 +1525,10 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k, int drop_
     if (streamed)
       compact_stream_kernel<DT><<<stream_grid, kCsThreads, kCsSmem, stream>>>(
           map, x, n, n_rows_full, out.header, out.bitmap, out.values, out.block_offsets, prefix,
-          n_chunks, n_stage_tiles);
+          &st->error, n_chunks, n_stage_tiles);
     else
       compact_small_kernel<DT><<<static_cast<unsigned>(L.tiles), kCompactThreads, 0, stream>>>(
-          x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix);
+          x, n, out.header, out.bitmap, out.values, out.block_offsets, prefix, &st->error);
     note_launches(1);
   }
   return cudaGetLastError();
@@ -1506,9 +1538,9 @@ cudaError_t run_prune_compact(const void* x, long long n, long long k, int drop_
 
 cudaError_t launch_prune_compact(const void* x, int64_t n, int dt, int64_t k,
                                  const surgeon_compressed& out, void* workspace,
-                                 cudaStream_t stream, int drop_zeros) {
-  return dt == 0 ? run_prune_compact<0>(x, n, k, drop_zeros, out, workspace, stream)
-                 : run_prune_compact<1>(x, n, k, drop_zeros, out, workspace, stream);
+                                 cudaStream_t stream, int drop_zeros, int stall) {
+  return dt == 0 ? run_prune_compact<0>(x, n, k, drop_zeros, stall, out, workspace, stream)
+                 : run_prune_compact<1>(x, n, k, drop_zeros, stall, out, workspace, stream);
 }
 
 cudaError_t launch_decompress(const surgeon_compressed& act, void* x_out, cudaStream_t stream) {

@@ -103,7 +103,7 @@ constexpr size_t prune_workspace_bytes(int64_t n, int dt) { return prune_layout(
 // Host launchers (each enqueues on `stream` and returns the last CUDA error).
 cudaError_t launch_prune_compact(const void* x, int64_t n, int dt, int64_t k,
                                  const surgeon_compressed& out, void* workspace,
-                                 cudaStream_t stream, int drop_zeros = 0);
+                                 cudaStream_t stream, int drop_zeros = 0, int stall = 0);
 cudaError_t launch_decompress(const surgeon_compressed& act, void* x_out, cudaStream_t stream);
 // Eq. 4 on device: *gi_out = sqrt(sum dw^2 / n); workspace = SURGEON_GI_WORKSPACE_BYTES of scratch.
 cudaError_t launch_gradient_importance(const float* dw, long long n, double* gi_out,

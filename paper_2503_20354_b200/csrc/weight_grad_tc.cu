@@ -900,6 +900,8 @@ size_t weight_grad_tc_workspace(const surgeon_layer_desc& d) {
 cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_layer_desc& d,
                                   const float* grad_out, float* dw, int accumulate,
                                   void* workspace, cudaStream_t stream) {
+  // No geometry plan fits: say so before anything touches the workspace (its size query gave 0).
+  if (weight_grad_tc_workspace(d) == 0 || workspace == nullptr) return cudaErrorNotSupported;
   uint32_t* status = static_cast<uint32_t*>(workspace);
   float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes);
   cudaError_t e = cudaMemsetAsync(status, 0, kStatusBytes, stream);

@@ -38,6 +38,11 @@ def test_own_arm_line():
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0
     assert d["gpu_launches"] > 0 and d["value"] > 0 and d["ms_per_step"] > 0
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+    # every timed workload carries a roofline entry for each of the two parts of the metric
+    w = d["workloads"]["tiny"]
+    assert w["prune_compact"]["bound"] == "hbm" and w["prune_compact"]["unit"] == "GB/s"
+    assert w["weight_grad"]["bound"] == "tensor" and w["weight_grad"]["frac"] > 0
+    assert d["roofline_prune_compact"]["frac"] > 0 and "frac_nominal" in d["roofline"]
 
 
 def test_reference_arm_line():

@@ -38,9 +38,12 @@ def _keys(x):
     return (x.view(torch.int16) & 0x7FFF).to(torch.int32)
 
 
-@pytest.mark.parametrize("bf16,ratio", [(False, 0.5), (False, 0.1), (True, 0.9)])
-def test_store_properties_at_sweep_size(bf16, ratio):
-    n = 1 << 28
+@pytest.mark.parametrize("lg,bf16,ratio", [(28, False, 0.5), (28, False, 0.1), (28, True, 0.9),
+                                            (30, False, 0.9), (30, True, 0.5)])
+def test_store_properties_at_sweep_size(lg, bf16, ratio):
+    """2^28 and 2^30 elements (the largest tensor of the bandwidth sweep: 4 GiB of fp32, where
+    byte offsets need 64 bits)."""
+    n = 1 << lg
     x = W.draw("relu_normal", n, seed=3, device="cuda")
     if bf16:
         x = x.to(torch.bfloat16)
@@ -83,30 +86,81 @@ def test_store_properties_at_sweep_size(bf16, ratio):
     assert last_kept_tie < first_dropped_tie          # ties are kept by lowest flat index
 
 
+def _stratified_entries(shape, rng, k_len):
+    """Entries of a weight-gradient tensor that reach every part of the launch grid: one random
+    entry in every cell of (16 output channels) x (16 input channels) x (kernel tap) - no tile of
+    rows, column unit, tap or accumulator of any kernel is wider than such a cell - plus random
+    entries over the whole tensor, fewer for long reductions (an entry costs k_len terms)."""
+    O, C = shape[0], shape[1]
+    taps = [(r, s) for r in range(shape[2]) for s in range(shape[3])] if len(shape) == 4 else [()]
+    cells = []
+    for tap in taps:
+        for o0 in range(0, O, 16):
+            for c0 in range(0, C, 16):
+                cells.append((int(rng.integers(o0, min(o0 + 16, O))),
+                              int(rng.integers(c0, min(c0 + 16, C)))) + tap)
+    budget = int(2.5e8 // max(k_len, 1))                 # terms the CPU adds up per case
+    if len(cells) > budget:                              # thin the cells evenly, keep the strata
+        cells = [cells[i] for i in np.linspace(0, len(cells) - 1, budget).astype(int)]
+    n_rand = int(min(2000, max(64, budget - len(cells))))
+    rand = [tuple(int(rng.integers(0, d)) for d in shape) for _ in range(n_rand)]
+    return cells + rand
+
+
+_SIGMA = {"wrn": 0.01, "vit": 1e-3, "r50": 1e-3}
+
+
+@pytest.mark.parametrize("ratio", [0.0, 0.3, 0.95])
 @pytest.mark.parametrize("which,name", [
-    ("wrn", "g3b1.conv1"), ("wrn", "g1b1.conv1"), ("wrn", "g2b0.conv1"), ("vit", "blk0.qkv"),
-    ("r50", "layer3.0.conv2"), ("r50", "stem"), ("r50", "layer2.0.downsample"),
+    ("wrn", "g1b1.conv1"),            # 160 channels, 32x32: tap stacking, two row tiles of 80 rows
+    ("wrn", "g2b1.conv1"),            # 320 channels, 16x16
+    ("wrn", "g3b1.conv1"),            # 640 channels, 8x8: five row tiles, twelve column tiles
+    ("wrn", "g2b0.conv1"),            # 3x3 stride 2 (shared-memory patch kernel)
+    ("wrn", "g2b0.shortcut"),         # 1x1 stride 2
+    ("vit", "blk0.qkv"), ("vit", "blk0.fc1"), ("vit", "blk0.fc2"),
+    ("r50", "layer1.0.conv3"),        # 1x1 64 -> 256 on 56x56: bound by the gradient read
+    ("r50", "layer3.0.conv2"),        # 3x3 stride 2 on 28x28 (im2col kernel)
+    ("r50", "stem"),                  # 7x7 stride 2
+    ("r50", "layer2.0.downsample"),   # 1x1 stride 2 on 56x56
+    ("r50", "layer4.1.conv2"),        # 3x3 on 7x7 maps (rows not a multiple of 8 wide)
+    ("r50", "fc"),
 ])
-def test_weight_gradient_of_a_whole_bench_layer_on_sampled_entries(which, name):
+def test_weight_gradient_of_a_whole_bench_layer_on_sampled_entries(which, name, ratio):
+    """A whole bench layer at a ratio the rule produces (0: the layer Eq. 7 leaves dense; 0.3: the
+    dense-tile path of the producers; 0.95).  The oracle prunes the activation itself; the GPU
+    store must equal the oracle's bit for bit, and the weight gradient is compared with the
+    oracle's on a stratified sample of entries computed from the ORACLE's pruned activation."""
     stack = {"wrn": W.wrn28_10, "vit": W.vit_b16, "r50": W.resnet50}[which]()
     layer = _layer(stack, name)
-    a = W.activation(layer, seed=0, device="cuda")
-    g = W.grad_out(layer, seed=0, sigma=1e-3, device="cuda")
-    comp = B.surgeon_prune_compact(a, 0.7)
-    dw = B.surgeon_weight_grad(comp, B.layer_desc(layer, B.PATH_TENSOR_CORE), g)
-    pruned = W.as_numpy_bits(B.surgeon_decompress(comp)).reshape(layer.act_shape)
-    gh = g.cpu().numpy()
+    a = W.activation(layer, seed=0)
+    g = W.grad_out(layer, seed=0, sigma=_SIGMA[which])
+    comp, ref = assert_store_equals_oracle(a.reshape(-1), ratio)
+    pruned = oracle.decompress(ref["bitmap"], ref["values"], layer.n_act).reshape(layer.act_shape)
+    dw = B.surgeon_weight_grad(comp, B.layer_desc(layer, B.PATH_TENSOR_CORE), g.cuda())
     dwh = dw.cpu().numpy()
+    gh = g.numpy()
     rng = np.random.default_rng(5)
-    got, ref = [], []
-    for _ in range(24):
-        idx = tuple(int(rng.integers(0, d)) for d in dwh.shape)
+    got, want = [], []
+    for idx in _stratified_entries(dwh.shape, rng, layer.gemm_k):
         if layer.kind == 1:
             r = oracle.dw_conv2d_entry(pruned, gh, layer.kh, layer.kw, layer.stride, layer.pad, *idx)
         else:
             r = oracle.dw_linear_entry(pruned, gh, *idx)
-        got.append(float(dwh[idx])); ref.append(r)
-    got, ref = np.array(got), np.array(ref)
+        got.append(float(dwh[idx])); want.append(r)
+    got, want = np.array(got), np.array(want)
     # the tolerance of the tensor-core path, taken over the sample
-    assert np.linalg.norm(got - ref) <= 5e-3 * np.linalg.norm(ref)
+    assert np.linalg.norm(got - want) <= 5e-3 * np.linalg.norm(want)
+    assert np.isfinite(dwh).all()
     assert comp.read_header().status == 0
+
+
+@pytest.mark.parametrize("which,name,ratio", [
+    ("wrn", "g1b1.conv1", 0.2), ("r50", "layer1.0.conv1", 0.3), ("vit", "blk0.fc2", 0.4),
+])
+def test_store_without_kept_zeros_at_bench_size(which, name, ratio):
+    """The store variant that spends no bit on a kept zero, on whole bench layers whose data hold
+    exact zeros in the kept set (post-ReLU at a ratio below one half) or none at all (GELU)."""
+    stack = {"wrn": W.wrn28_10, "vit": W.vit_b16, "r50": W.resnet50}[which]()
+    layer = _layer(stack, name)
+    x = W.activation(layer, seed=0)
+    assert_store_equals_oracle(x.reshape(-1), ratio, drop_zeros=True)

@@ -176,3 +176,22 @@ def test_argument_errors_on_device():
     with pytest.raises(B.SurgeonError) as e:
         B.surgeon_prune_compact(x[1:], 0.5)      # 4-byte aligned only
     assert e.value.status == B.SURGEON_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_bounded_wait_that_runs_out_reports_timeout_and_stores_nothing(bf16):
+    """The select's grid barrier is given a target it cannot reach and a cap of 1024 polls
+    (SURGEON_DEBUG_STALL_BARRIER): the wait gives up, the header says so, and no kernel of the call
+    has touched bitmap, values or block offsets.  The next ordinary call is unaffected."""
+    n = 5000
+    x = _as(W.draw("normal", n, seed=8), bf16).cuda()
+    comp = B.CompressedActivation(n, B.dtype_code(x.dtype), 0.0, x.device)
+    comp.bitmap.fill_(0x5A5A5A5A); comp.block_offsets.fill_(0x1234567)
+    comp.values.view(torch.int16 if bf16 else torch.int32).fill_(0x4D4D)
+    ws = torch.empty(comp.sizes.workspace_bytes, dtype=torch.uint8, device="cuda")
+    B.surgeon_prune_compact(x, 0.5, out=comp, workspace=ws, flags=B.SURGEON_DEBUG_STALL_BARRIER)
+    torch.cuda.synchronize()
+    assert comp.read_header().status == B.SURGEON_ERR_TIMEOUT
+    assert bool((comp.bitmap == 0x5A5A5A5A).all()) and bool((comp.block_offsets == 0x1234567).all())
+    assert bool((comp.values.view(torch.int16 if bf16 else torch.int32) == 0x4D4D).all())
+    assert_store_equals_oracle(x.cpu(), 0.5, comp=B.surgeon_prune_compact(x, 0.5, out=comp, workspace=ws))

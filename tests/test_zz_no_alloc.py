@@ -10,6 +10,7 @@ what the comparison is there to catch."""
 import ctypes as C
 
 import numpy as np
+import oracle
 import pytest
 import torch
 
@@ -46,6 +47,25 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(bf16):
     torch.cuda.synchronize()
     for x, ratio, out in outs:
         _same_store(out, B.surgeon_prune_compact(x, ratio))
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_largest_size_against_the_oracle_too(bf16):
+    """n = SURGEON_STATIC_MAX_N exactly (the scratch is laid out for this size; both dtypes take
+    the streamed select here), twice in a row, against the ordinary entry point and the oracle."""
+    n = B.SURGEON_STATIC_MAX_N
+    x = W.draw("relu_normal", n, seed=12)
+    x = x.to(torch.bfloat16) if bf16 else x
+    xd = x.cuda()
+    out = B.CompressedActivation(n, B.dtype_code(xd.dtype), 0.0, xd.device)
+    for ratio in (0.8, 0.25):
+        B.surgeon_prune_compact_static(xd, ratio, out)
+        _same_store(out, B.surgeon_prune_compact(xd, ratio))
+        ref = oracle.prune_compact(W.as_numpy_bits(x).reshape(-1), ratio)
+        bitmap, vals, offs, hdr = out.to_numpy()
+        assert hdr.threshold_key == ref["tau"] and hdr.n_keep == ref["k"]
+        assert np.array_equal(bitmap, ref["bitmap"]) and np.array_equal(offs, ref["offsets"])
+        assert np.array_equal(vals.view(np.uint8), ref["values"].view(np.uint8))
 
 
 def test_same_input_twice_and_size_limit():
