@@ -883,6 +883,8 @@ static size_t direct_partial_bytes(const DirectParams& p) {
 }
 
 size_t weight_grad_tc_workspace(const surgeon_layer_desc& d) {
+  SwapParams sp;
+  if (plan_swap(d, &sp)) return kStatusBytes + swap_partial_bytes(sp) + direct_grad_bf16_bytes(sp.d);
   DirectParams dp;
   if (plan_direct(d, &dp)) return kStatusBytes + direct_partial_bytes(dp) + direct_grad_bf16_bytes(dp);
   FastParams f;
@@ -906,10 +908,22 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
   float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes);
   cudaError_t e = cudaMemsetAsync(status, 0, kStatusBytes, stream);
   if (e != cudaSuccess) return e;
+#ifdef SURGEON_DW_STATS
+  cudaMemsetAsync(reinterpret_cast<char*>(status) + 14 * 8, 0xFF, 8, stream);
+#endif
   DirectParams dp;
-  if (plan_direct(d, &dp)) {
-    void* grad_bf16 = reinterpret_cast<char*>(partial) + direct_partial_bytes(dp);
-    e = launch_direct(act, dp, grad_out, grad_bf16, partial, status, stream);
+  SwapParams sp;
+  const bool swapped = plan_swap(d, &sp);
+  if (swapped || plan_direct(d, &dp)) {
+    if (swapped) {
+      dp = sp.d;
+      dp.splits = sp.splits;
+      void* grad_bf16 = reinterpret_cast<char*>(partial) + swap_partial_bytes(sp);
+      e = launch_swap(act, sp, grad_out, grad_bf16, partial, status, stream);
+    } else {
+      void* grad_bf16 = reinterpret_cast<char*>(partial) + direct_partial_bytes(dp);
+      e = launch_direct(act, dp, grad_out, grad_bf16, partial, status, stream);
+    }
     if (e != cudaSuccess) return e;
     const long long mn = static_cast<long long>(dp.O) * dp.C;
     if (dp.taps > 1)

@@ -1,6 +1,8 @@
 // Plan and launcher of the fast stride-1 convolution kernel (weight_grad_tc_conv.cu).
 #pragma once
 
+#include <cuda.h>
+
 #include "surgeon_internal.cuh"
 
 namespace surgeon {
@@ -69,5 +71,38 @@ size_t direct_grad_bf16_bytes(const DirectParams& p);
 cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& p,
                           const float* grad_out, void* grad_bf16, float* partial,
                           uint32_t* status, cudaStream_t stream);
+// The pre-pass that writes the bf16 copy (or shifted copies) of the output gradient, and the
+// tensor map over it (conv: boxes of 64 positions x box_rows rows; linear: 64 columns x 64 rows).
+cudaError_t launch_direct_prepass(const DirectParams& p, const float* grad_out, void* grad_bf16,
+                                  cudaStream_t stream);
+cudaError_t encode_direct_grad_map(const DirectParams& p, void* grad_bf16, int box_rows, CUtensorMap* out);
+
+// ---- the same layers on CTA pairs with the operand roles exchanged (weight_grad_tc_swap.cu) -----
+struct SwapParams {
+  DirectParams d;           // layer geometry and the layout of the bf16 gradient copy
+  int nt, half;             // input channels per pair tile (MMA N, a multiple of 16) and per CTA
+  int n_acc;                // accumulators per CTA: 128 gradient rows x nt channels each
+  int lpr;                  // lanes (runs of 32 elements) per row of the activation tile: 2 or 4
+  // conv: the stacked gradient rows (tap, output channel) are cut into units of 128 TMEM lanes.
+  // Per tap a_units full units of 128 rows (one TMA box each; the last may be partly filled when
+  // rem_box is 0); the o_real - 128 * a_full rows left over, if any, go `rpu` taps to a unit in
+  // boxes of rem_box rows (a power of two below 128).
+  int a_full, a_units, rem_box, rpu;
+  int n_units;              // units in all (linear: groups of 128 gradient columns)
+  int m_tiles, n_tiles, splits, ktiles_per_split;
+  int gw, groups;           // warps per producer group, groups (one K-tile in flight per group)
+  int a_stages, g_stages;   // depth of the activation-tile and gradient-tile rings
+  int stage_bytes;          // staging area of packed values (fp32 activations), 0 if none
+  int tmem_cols, smem_bytes;
+  long long n_words;        // words of the bitmap (filled by the launcher)
+  const long long* n_keep_ptr;
+  unsigned partial_blk;     // index of the bitmap's last block if it is partial, else 0xFFFFFFFF
+};
+bool plan_swap(const surgeon_layer_desc& d, SwapParams* out);
+int swap_resident_pairs();   // CTA pairs the device holds at once
+size_t swap_partial_bytes(const SwapParams& p);
+// partial = [splits][O][C] fp32 (O counts the stacked taps), status = one zeroed word.
+cudaError_t launch_swap(const surgeon_compressed& act, const SwapParams& p, const float* grad_out,
+                        void* grad_bf16, float* partial, uint32_t* status, cudaStream_t stream);
 
 }  // namespace surgeon

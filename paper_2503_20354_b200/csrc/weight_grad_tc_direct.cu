@@ -867,15 +867,10 @@ size_t direct_grad_bf16_bytes(const DirectParams& p) {
   return (b + 255) & ~static_cast<size_t>(255);
 }
 
-cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& plan,
-                          const float* grad_out, void* grad_bf16, float* partial,
-                          uint32_t* status, cudaStream_t stream) {
-  DirectParams p = plan;
-  if (!size_rings(&p, act.dt == 0 ? kStageBytes : 0)) return cudaErrorInvalidValue;
-  p.n_words = (act.n + 31) / 32;
-  p.n_keep_ptr = reinterpret_cast<const long long*>(reinterpret_cast<const char*>(act.header) +
-                                                    offsetof(surgeon_header, n_keep));
-  p.partial_blk = (act.n % SURGEON_BLOCK) ? static_cast<unsigned>(act.n / SURGEON_BLOCK) : 0xFFFFFFFFu;
+// The bf16 copy (or shifted copies) of the output gradient that the tensor maps of the direct
+// kernels read: one streaming pre-pass.
+cudaError_t launch_direct_prepass(const DirectParams& p, const float* grad_out, void* grad_bf16,
+                                  cudaStream_t stream) {
   cudaError_t e;
   if (p.row_shift) {
     const long long chunks = static_cast<long long>(p.imgs) * p.o_real * (p.pitch >> 3);
@@ -927,10 +922,15 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
                                  grad_bf16, stream);
   else
     e = launch_grad_to_bf16(grad_out, static_cast<long long>(p.imgs) * p.O * p.T, grad_bf16, stream);
-  if (e != cudaSuccess) return e;
+  return e;
+}
+
+// Tensor map over the bf16 gradient copy.  Linear: [T rows][O columns], box 64 columns x 64 rows.
+// Conv: [images][copies * O rows][g_len positions], box 64 positions x `box_rows` rows.
+cudaError_t encode_direct_grad_map(const DirectParams& p, void* grad_bf16, int box_rows, CUtensorMap* out) {
+  CUtensorMap& map = *out;
   const EncodeFn encode = reinterpret_cast<EncodeFn>(tensor_map_encode_fn());
   if (!encode) return cudaErrorNotSupported;
-  CUtensorMap map;
   CUresult r;
   if (p.mode == 0) {
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(p.O), static_cast<cuuint64_t>(p.T)};
@@ -946,13 +946,29 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
     const cuuint64_t strides[2] = {static_cast<cuuint64_t>(p.pitch) * 2,
                                    static_cast<cuuint64_t>(p.pitch) * rows * 2};
     const cuuint32_t box[3] = {static_cast<cuuint32_t>(kTileK),
-                               static_cast<cuuint32_t>(p.pair ? p.acc_n / 2 : p.acc_n), 1};
+                               static_cast<cuuint32_t>(box_rows), 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, grad_bf16, dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   }
-  if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& plan,
+                          const float* grad_out, void* grad_bf16, float* partial,
+                          uint32_t* status, cudaStream_t stream) {
+  DirectParams p = plan;
+  if (!size_rings(&p, act.dt == 0 ? kStageBytes : 0)) return cudaErrorInvalidValue;
+  p.n_words = (act.n + 31) / 32;
+  p.n_keep_ptr = reinterpret_cast<const long long*>(reinterpret_cast<const char*>(act.header) +
+                                                    offsetof(surgeon_header, n_keep));
+  p.partial_blk = (act.n % SURGEON_BLOCK) ? static_cast<unsigned>(act.n / SURGEON_BLOCK) : 0xFFFFFFFFu;
+  cudaError_t e = launch_direct_prepass(p, grad_out, grad_bf16, stream);
+  if (e != cudaSuccess) return e;
+  CUtensorMap map;
+  e = encode_direct_grad_map(p, grad_bf16, p.pair ? p.acc_n / 2 : p.acc_n, &map);
+  if (e != cudaSuccess) return e;
   dim3 grid(p.m_tiles, p.n_tiles, p.splits);
   auto launch = [&](auto kernel) -> cudaError_t {
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
