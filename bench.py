@@ -257,20 +257,30 @@ def barrier(world: int):
 class Stack:
     """Device-resident inputs, stores, outputs and scratch of one replica of the workload."""
 
-    def __init__(self, layers, path: int, seed: int, device, n_streams=1, sigma=0.01, ratios="rule"):
+    def __init__(self, layers, path: int, seed: int, device, n_streams=1, sigma=0.01, ratios="rule", share=True):
         from paper_2503_20354_b200 import binding as B
         from paper_2503_20354_b200 import workloads as W
         self.B, self.layers, self.path, self.device = B, layers, path, device
         self.gi = W.gradient_importance(len(layers), seed)
         self.lam = np.array([l.act_bytes for l in layers], dtype=np.float64)
         self.fixed_ratios = W.uniform_ratios(len(layers), seed) if ratios == "uniform" else None
-        self.x = [W.activation(l, seed, i, device=device) for i, l in enumerate(layers)]
+        # A residual block's shortcut convolution reads the same tensor as the block's first
+        # convolution: that tensor is pruned once, at the smaller of the two layers' ratios (the
+        # one that keeps more), and both weight gradients read the one store.
+        self.shared = W.shared_inputs(layers) if share else {}
+        self.x = [None if i in self.shared else W.activation(l, seed, i, device=device) for i, l in enumerate(layers)]
+        for j, i in self.shared.items():
+            self.x[j] = self.x[i]
         self.g = [W.grad_out(l, seed, i, sigma=sigma, device=device) for i, l in enumerate(layers)]
         self.desc = [B.layer_desc(l, path) for l in layers]
         self.dw = [torch.empty(l.dw_shape, dtype=torch.float32, device=device) for l in layers]
         # stores sized for ratio 0: ratios change every batch, the buffers do not
-        self.store = [B.CompressedActivation(l.n_act, l.dt, 0.0, device) for l in layers]
+        self.store = [None if i in self.shared else B.CompressedActivation(l.n_act, l.dt, 0.0, device)
+                      for i, l in enumerate(layers)]
+        for j, i in self.shared.items():
+            self.store[j] = self.store[i]
         ws1 = max(s.sizes.workspace_bytes for s in self.store)
+        self.own = [i for i in range(len(layers)) if i not in self.shared]    # layers that prune their input
         ws2 = max(B.surgeon_weight_grad_workspace(d) for d in self.desc)
         # Layers are independent of one another (a layer's store is written once in the forward
         # pass and read once in the backward pass), so they are issued round-robin on n_streams
@@ -300,6 +310,10 @@ class Stack:
             self.ratios = self.fixed_ratios
         else:
             self.ratios = self.B.surgeon_layer_ratios(self.gi, self.lam, allow_degenerate=True)   # Eq. 5-7
+        if self.shared:
+            self.ratios = np.array(self.ratios, dtype=np.float64)
+            for j, i in self.shared.items():
+                self.ratios[i] = self.ratios[j] = min(self.ratios[i], self.ratios[j])
         return self.ratios
 
     def step(self, ev=None, x_ready=None, g_ready=None, dw_done=None):
@@ -310,8 +324,8 @@ class Stack:
         if ev: ev[0].record()
         self.compute_ratios()
         self._fork()
-        for i in range(len(self.layers)):                                                # forward
-            k = i % self.n_streams
+        for n, i in enumerate(self.own):                                                 # forward
+            k = n % self.n_streams
             st = self.stream_of(k)
             if x_ready is not None:
                 (st or torch.cuda.current_stream(self.device)).wait_event(x_ready[i])
@@ -421,9 +435,10 @@ def run_stack(key, args, rank, world, device, peaks, path, keep_stack=False, sam
         if h.status != 0:
             raise SystemExit("device status %d in a compressed store" % h.status)
     flops = sum(l.flops for l in layers)
-    pbytes = sum(prune_alg_bytes(l, s.sizes.n_keep) for l, s in zip(layers, stack.store))
-    stored = sum(s.stored_bytes for s in stack.store)
-    dense = sum(l.act_bytes for l in layers)
+    own = stack.own                      # a tensor two layers read is pruned and stored once
+    pbytes = sum(prune_alg_bytes(layers[i], stack.store[i].sizes.n_keep) for i in own)
+    stored = sum(stack.store[i].stored_bytes for i in own)
+    dense = sum(layers[i].act_bytes for i in own)
     prune_gbs = pbytes / (prune_ms * 1e-3) / 1e9
     dw_tflops = flops / (dw_ms * 1e-3) / 1e12
     full = args.batch is None and args.layers is None
@@ -451,6 +466,7 @@ def run_stack(key, args, rank, world, device, peaks, path, keep_stack=False, sam
         "prune_compact": pc_entry, "weight_grad": dw_entry,
         "store_bytes": stored, "dense_bytes": dense, "gpu_launches": int(launches),
         "read_GB_per_step": round((dense + sum(g.numel() * 4 for g in stack.g)) / 1e9, 2),
+        "shared_inputs": len(stack.shared),
     }
     if args.per_layer or key.startswith("resnet50"):
         us = stack.per_layer_dw_us()
@@ -631,7 +647,7 @@ def run_e2e(stack, layers, args, world, device, flops):
     for h, d in zip(hx + hg, stack.x + stack.g):
         h.copy_(d)
     torch.cuda.synchronize()
-    h2d = sum(t.numel() * t.element_size() for t in hx + hg)
+    h2d = sum(hx[i].numel() * hx[i].element_size() for i in stack.own) + sum(t.numel() * t.element_size() for t in hg)
     d2h = sum(t.numel() * t.element_size() for t in hdw)
     s_in, s_out = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)
     main = torch.cuda.current_stream(device)
@@ -642,7 +658,7 @@ def run_e2e(stack, layers, args, world, device, flops):
         dw_done = [torch.cuda.Event() for _ in range(n)]
         s_in.wait_stream(main)
         with torch.cuda.stream(s_in):
-            for i in range(n):                       # forward order
+            for i in stack.own:                      # forward order; a shared tensor crosses once
                 stack.x[i].copy_(hx[i], non_blocking=True)
                 x_ready[i].record(s_in)
             for i in reversed(range(n)):             # backward order

@@ -1,6 +1,8 @@
 // extern "C" entry points of libsurgeon: argument checks and host-side arithmetic; every step
 // that touches tensor data is a kernel launched from the other translation units.
 #include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
 
 #include <atomic>
 
@@ -22,6 +24,33 @@ void* tensor_map_encode_fn() {
     return p;
   }();
   return fn;
+}
+
+cudaError_t allow_dynamic_smem(const void* kernel, int bytes) {
+  struct Seen { const void* fn; int dev; std::atomic<int> bytes; };
+  static Seen seen[256];
+  static std::atomic<int> n_seen{0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) dev = 0;
+  const int n = n_seen.load(std::memory_order_acquire);
+  Seen* hit = nullptr;
+  for (int i = 0; i < n; ++i)
+    if (seen[i].fn == kernel && seen[i].dev == dev) { hit = &seen[i]; break; }
+  if (hit && hit->bytes.load(std::memory_order_relaxed) >= bytes) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  // two threads may both set the attribute (harmless: the larger value is set again by whoever
+  // needs it); the table only grows
+  if (hit) {
+    hit->bytes.store(bytes, std::memory_order_relaxed);
+  } else {
+    const int slot = n_seen.load(std::memory_order_relaxed);
+    if (slot < 256) {
+      seen[slot].fn = kernel; seen[slot].dev = dev; seen[slot].bytes.store(bytes, std::memory_order_relaxed);
+      n_seen.store(slot + 1, std::memory_order_release);
+    }
+  }
+  return cudaSuccess;
 }
 
 int sm_count() {
@@ -230,6 +259,8 @@ surgeon_status surgeon_weight_grad(const surgeon_compressed* act, const surgeon_
       d->path == 1 ? launch_weight_grad_fp32(*act, *d, grad_out, dw, accumulate ? 1 : 0, workspace, s)
                    : launch_weight_grad_tc(*act, *d, grad_out, dw, accumulate ? 1 : 0, workspace, s);
   if (e == cudaErrorNotSupported) return SURGEON_ERR_UNSUPPORTED;
+  if (e != cudaSuccess && getenv("SURGEON_VERBOSE"))
+    fprintf(stderr, "surgeon_weight_grad: %s\n", cudaGetErrorString(e));
   return e == cudaSuccess ? SURGEON_OK : SURGEON_ERR_CUDA;
 }
 

@@ -124,8 +124,35 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
 void* tensor_map_encode_fn();
 // Number of SMs of the current device (cached per device id).
 int sm_count();
+// Lets `kernel` use `bytes` of dynamic shared memory; the attribute is set when a kernel first
+// needs that much on a device, later calls only look it up.
+cudaError_t allow_dynamic_smem(const void* kernel, int bytes);
 // Adds to the process-wide kernel-launch counter behind surgeon_launch_count().
 void note_launches(int n);
+
+// Programmatic dependent launch.  A kernel launched with `dependent` set may start while the
+// kernel before it on the stream is still running (once every CTA of that kernel has called
+// pdl_trigger or has exited): its set-up then overlaps the predecessor's tail.  It must call
+// pdl_wait before it touches anything the predecessor writes; pdl_wait returns when the
+// predecessor has completed and its writes are visible.  Both calls do nothing in a kernel that
+// was launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t stream, bool dependent, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 __device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31; }
 __device__ __forceinline__ uint32_t lanemask_lt() {

@@ -681,6 +681,7 @@ __global__ void __launch_bounds__(256)
 reduce_splits_kernel(const float* __restrict__ partial, long long mn, int splits,
                      float* __restrict__ dw, int accumulate, const uint32_t* __restrict__ status,
                      surgeon_header* __restrict__ hdr) {
+  pdl_wait();                            // the partial tiles are complete
   const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i == 0 && *status != 0 && hdr) atomicMax(&hdr->status, *status);
   if (i >= mn) return;
@@ -694,6 +695,7 @@ __global__ void __launch_bounds__(256)
 reduce_splits4_kernel(const float* __restrict__ partial, long long mn, int splits,
                       float* __restrict__ dw, int accumulate, const uint32_t* __restrict__ status,
                       surgeon_header* __restrict__ hdr) {
+  pdl_wait();                            // the partial tiles are complete
   const long long i = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
   if (i == 0 && *status != 0 && hdr) atomicMax(&hdr->status, *status);
   if (i >= mn) return;
@@ -714,12 +716,14 @@ static void launch_reduce_splits(const float* partial, long long mn, int splits,
                                  int accumulate, const uint32_t* status, surgeon_header* hdr,
                                  cudaStream_t stream) {
   const bool vec = (mn & 3) == 0 && ((reinterpret_cast<uintptr_t>(partial) | reinterpret_cast<uintptr_t>(dw)) & 15) == 0;
+  // launched as a programmatic dependent of the kernel that writes the partial tiles: it is
+  // resident (or queued) when that kernel ends and starts at once
   if (vec)
-    reduce_splits4_kernel<<<static_cast<unsigned>((mn / 4 + 255) / 256), 256, 0, stream>>>(
-        partial, mn, splits, dw, accumulate, status, hdr);
+    launch_kernel(reduce_splits4_kernel, dim3(static_cast<unsigned>((mn / 4 + 255) / 256)), dim3(256), 0, stream,
+                  true, partial, mn, splits, dw, accumulate, status, hdr);
   else
-    reduce_splits_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(
-        partial, mn, splits, dw, accumulate, status, hdr);
+    launch_kernel(reduce_splits_kernel, dim3(static_cast<unsigned>((mn + 255) / 256)), dim3(256), 0, stream,
+                  true, partial, mn, splits, dw, accumulate, status, hdr);
 }
 
 // The same for a tap-stacked partial [splits][taps * O][C]: dw[o][c][tap] gets row tap * O + o.
@@ -731,6 +735,7 @@ reduce_splits_taps_kernel(const float* __restrict__ partial, int o_real, int c_i
                           int chunk, int splits, float* __restrict__ dw, int accumulate,
                           const uint32_t* __restrict__ status, surgeon_header* __restrict__ hdr) {
   extern __shared__ __align__(16) float tile[];    // [n_c][taps]
+  pdl_wait();                                      // the partial tiles are complete
   const int c0 = blockIdx.x * chunk;
   const int o = blockIdx.y;
   if (blockIdx.x == 0 && o == 0 && threadIdx.x == 0 && *status != 0 && hdr)
@@ -933,9 +938,10 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
       while (chunk > 32 && (static_cast<long long>(dp.o_real) * ((dp.C + chunk - 1) / chunk) < 4LL * sm_count() ||
                             chunk * dp.taps * 4 > 48 * 1024))
         chunk >>= 1;
-      reduce_splits_taps_kernel<<<dim3((dp.C + chunk - 1) / chunk, dp.o_real), 256,
-                                  static_cast<size_t>(chunk) * dp.taps * sizeof(float), stream>>>(
-          partial, dp.o_real, dp.C, dp.taps, chunk, dp.splits, dw, accumulate, status, act.header);
+      launch_kernel(reduce_splits_taps_kernel, dim3((dp.C + chunk - 1) / chunk, dp.o_real), dim3(256),
+                    static_cast<size_t>(chunk) * dp.taps * sizeof(float), stream, true,
+                    static_cast<const float*>(partial), dp.o_real, dp.C, dp.taps, chunk, dp.splits, dw, accumulate,
+                    static_cast<const uint32_t*>(status), act.header);
     }
 
     else
@@ -984,14 +990,12 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
     const size_t smem = im2col_smem_bytes(p);
     dim3 grid(p.m_tiles, p.n_tiles, p.splits);
     if (act.dt == 0) {
-      e = cudaFuncSetAttribute(dw_conv_im2col_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               static_cast<int>(smem));
+      e = allow_dynamic_smem(reinterpret_cast<const void*>(dw_conv_im2col_kernel<0>), static_cast<int>(smem));
       if (e != cudaSuccess) return e;
       dw_conv_im2col_kernel<0><<<grid, kGThreads, smem, stream>>>(act.bitmap, act.values, act.block_offsets,
                                                                  map, partial, status, p);
     } else {
-      e = cudaFuncSetAttribute(dw_conv_im2col_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               static_cast<int>(smem));
+      e = allow_dynamic_smem(reinterpret_cast<const void*>(dw_conv_im2col_kernel<1>), static_cast<int>(smem));
       if (e != cudaSuccess) return e;
       dw_conv_im2col_kernel<1><<<grid, kGThreads, smem, stream>>>(act.bitmap, act.values, act.block_offsets,
                                                                  map, partial, status, p);
@@ -1007,14 +1011,12 @@ cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_l
   const uint32_t* offs = act.block_offsets;
   dim3 grid(p.m_tiles, p.n_tiles, p.splits);
   if (act.dt == 0) {
-    e = cudaFuncSetAttribute(dw_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(smem));
+    e = allow_dynamic_smem(reinterpret_cast<const void*>(dw_tc_kernel<0>), static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     dw_tc_kernel<0><<<grid, kThreads, smem, stream>>>(act.bitmap, act.values, offs, grad_out,
                                                       partial, status, p);
   } else {
-    e = cudaFuncSetAttribute(dw_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(smem));
+    e = allow_dynamic_smem(reinterpret_cast<const void*>(dw_tc_kernel<1>), static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     dw_tc_kernel<1><<<grid, kThreads, smem, stream>>>(act.bitmap, act.values, offs, grad_out,
                                                       partial, status, p);

@@ -414,6 +414,7 @@ dw_conv_fast_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict_
 // fp32 -> bf16 (round to nearest even), 8 elements per thread.
 __global__ void __launch_bounds__(256)
 grad_to_bf16_kernel(const float* __restrict__ g, long long n, unsigned short* __restrict__ out) {
+  pdl_trigger();
   const long long n8 = n >> 3;
   const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
   for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n8;
@@ -434,6 +435,7 @@ grad_to_bf16_kernel(const float* __restrict__ g, long long n, unsigned short* __
 __global__ void __launch_bounds__(256)
 grad_to_bf16_rows_kernel(const float* __restrict__ g, long long rows, int len, int pitch,
                          unsigned short* __restrict__ out) {
+  pdl_trigger();
   const int per_row = pitch >> 3;
   const long long total = rows * per_row;
   const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
@@ -469,7 +471,7 @@ TensorMapEncodeFn tensor_map_encoder() {
 
 }  // namespace
 
-bool plan_conv_fast(const surgeon_layer_desc& d, FastParams* out) {
+static bool compute_plan_conv_fast(const surgeon_layer_desc& d, FastParams* out) {
   if (d.kind != 1 || (d.stride != 1 && d.stride != 2)) return false;
   int mode;
   if (d.kh == 3 && d.kw == 3 && d.pad == 1) mode = 0;
@@ -542,6 +544,11 @@ bool plan_conv_fast(const surgeon_layer_desc& d, FastParams* out) {
   return true;
 }
 
+bool plan_conv_fast(const surgeon_layer_desc& d, FastParams* out) {
+  struct Tag {};
+  return memo_plan<Tag>(d, 0, out, [&](FastParams* p) { return compute_plan_conv_fast(d, p); });
+}
+
 cudaError_t launch_grad_to_bf16(const float* g, long long n, void* out_bf16, cudaStream_t stream) {
   const long long want = (n / 8 + 255) / 256;
   const long long cap = 16LL * sm_count();
@@ -598,14 +605,12 @@ cudaError_t launch_conv_fast(const surgeon_compressed& act, const FastParams& p,
   dim3 grid(p.m_tiles, p.n_tiles, p.splits);
   cudaError_t e;
   if (act.dt == 0) {
-    e = cudaFuncSetAttribute(dw_conv_fast_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             p.smem_bytes);
+    e = allow_dynamic_smem(reinterpret_cast<const void*>(dw_conv_fast_kernel<0>), p.smem_bytes);
     if (e != cudaSuccess) return e;
     dw_conv_fast_kernel<0><<<grid, kThreads, p.smem_bytes, stream>>>(
         act.bitmap, act.values, offs, map, partial, status, p);
   } else {
-    e = cudaFuncSetAttribute(dw_conv_fast_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             p.smem_bytes);
+    e = allow_dynamic_smem(reinterpret_cast<const void*>(dw_conv_fast_kernel<1>), p.smem_bytes);
     if (e != cudaSuccess) return e;
     dw_conv_fast_kernel<1><<<grid, kThreads, p.smem_bytes, stream>>>(
         act.bitmap, act.values, offs, map, partial, status, p);

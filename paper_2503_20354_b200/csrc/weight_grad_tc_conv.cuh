@@ -5,7 +5,37 @@
 
 #include "surgeon_internal.cuh"
 
+#include <cstring>
+
 namespace surgeon {
+
+// Plans depend only on the layer geometry (and the device's SM count): a weight-gradient call
+// looks its plan up in a small per-thread table instead of searching tilings and split counts
+// again (the searches cost microseconds, as much as a kernel launch).  `Tag` separates the tables
+// of the different planners.
+template <typename Tag, typename P, typename F>
+inline bool memo_plan(const surgeon_layer_desc& d, int extra, P* out, F compute) {
+  struct Entry { surgeon_layer_desc d; int extra, dev; bool used, ok; P p; };
+  constexpr int kEntries = 64;
+  thread_local Entry table[kEntries] = {};
+  thread_local int next = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) dev = 0;
+  for (int i = 0; i < kEntries; ++i) {
+    const Entry& e = table[i];
+    if (e.used && e.extra == extra && e.dev == dev && std::memcmp(&e.d, &d, sizeof(d)) == 0) {
+      if (e.ok) *out = e.p;
+      return e.ok;
+    }
+  }
+  Entry& e = table[next];
+  next = (next + 1) % kEntries;
+  e.d = d; e.extra = extra; e.dev = dev; e.used = true;
+  e.p = P{};
+  e.ok = compute(&e.p);
+  if (e.ok) *out = e.p;
+  return e.ok;
+}
 
 struct FastParams {
   int mode;                 // 0 = 3x3 pad 1 through a shared-memory patch, 1 = 1x1 direct

@@ -144,6 +144,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   if (PAIR) cluster_sync_all();          // both CTAs' barriers exist before either is arrived on
   tc_fence_after();
   const uint32_t tmem_base = tmem_slot;
+  pdl_trigger();                         // the split reduction may be launched; it waits for this grid
 
   if (warp == 0) {
     // ================= MMA issuer (rank 0 of a pair) =================
@@ -182,6 +183,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
   } else if (warp == 1) {
     // ================= gradient tiles by TMA =================
     if (lane == 0) {
+      pdl_wait();                                      // the bf16 gradient copy is complete
       int sb = 0;
       uint32_t round = 0;
       int img = 0, kin = 0;                            // conv: image and K-tile within it
@@ -591,6 +593,7 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
 __global__ void __launch_bounds__(256)
 grad_taps_bf16_kernel(const float* __restrict__ g, unsigned short* __restrict__ out,
                       long long chunks, DirectParams p) {
+  pdl_trigger();
   const int per_row = p.pitch >> 3;
   for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < chunks;
        i += static_cast<long long>(gridDim.x) * blockDim.x) {
@@ -631,6 +634,7 @@ template <int KW>
 __global__ void __launch_bounds__(256)
 grad_taps_same_bf16_kernel(const float* __restrict__ g, unsigned short* __restrict__ out,
                            long long items, DirectParams p) {
+  pdl_trigger();
   constexpr int H = (KW - 1) / 2;
   const int per_row = p.pitch >> 3;
   for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < items;
@@ -681,6 +685,7 @@ template <int KW, bool SAME>
 __global__ void __launch_bounds__(256)
 grad_cols_bf16_kernel(const float* __restrict__ g, unsigned short* __restrict__ out,
                       long long chunks, DirectParams p) {
+  pdl_trigger();
   const int per_row = p.in_w >> 3;                     // chunks per map row
   const int per_plane = p.pitch >> 3;                  // pitch = OH * W
   for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < chunks;
@@ -750,7 +755,7 @@ static bool size_rings(DirectParams* p, int stage_bytes) {
   return true;
 }
 
-bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
+static bool compute_plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   DirectParams p{};
   if (d.kind == 0) {
     p.mode = 0;
@@ -859,6 +864,11 @@ bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
   if (!size_rings(&p, kStageBytes)) return false;   // the launcher sizes them again for the dtype
   *out = p;
   return true;
+}
+
+bool plan_direct(const surgeon_layer_desc& d, DirectParams* out) {
+  struct Tag {};
+  return memo_plan<Tag>(d, use_pairs() ? 1 : 0, out, [&](DirectParams* p) { return compute_plan_direct(d, p); });
 }
 
 size_t direct_grad_bf16_bytes(const DirectParams& p) {
@@ -971,21 +981,23 @@ cudaError_t launch_direct(const surgeon_compressed& act, const DirectParams& pla
   if (e != cudaSuccess) return e;
   dim3 grid(p.m_tiles, p.n_tiles, p.splits);
   auto launch = [&](auto kernel) -> cudaError_t {
-    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           p.smem_bytes);
+    cudaError_t err = allow_dynamic_smem(reinterpret_cast<const void*>(kernel), p.smem_bytes);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = static_cast<size_t>(p.smem_bytes);
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = p.pair ? 2 : 1;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // starts while the gradient pre-pass drains: set-up and the first activation tiles overlap it
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kernel, act.bitmap, act.values, act.block_offsets, map, partial,
                               status, p);
   };

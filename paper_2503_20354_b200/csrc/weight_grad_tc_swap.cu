@@ -415,9 +415,19 @@ dw_swap_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ val
     long long st_w = 0;
     const long long st_pb = clock64();
 #endif
+#ifdef SURGEON_DW_STATS
+    long long ph[6] = {0, 0, 0, 0, 0, 0};
+#define PH_STAMP(i) { const long long c_ = clock64(); ph[i] += c_ - ph_t; ph_t = c_; }
+#else
+#define PH_STAMP(i)
+#endif
     for (int it = wg; it < n_kt; it += p.groups) {
+#ifdef SURGEON_DW_STATS
+      long long ph_t = clock64();
+#endif
       RunMeta nxt2 = {};
       if (it + 2 * p.groups < n_kt) { nxt2 = fetch(); advance(); }
+      PH_STAMP(0)
       uint4 chunk[4];
       if (dense) {
         // The LPR lanes of a row hold consecutive runs, so a row's kept values are one contiguous
@@ -494,6 +504,7 @@ dw_swap_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ val
           }
         }
       }
+      PH_STAMP(1)
 #ifdef SURGEON_DW_STATS
       const long long cw0 = clock64();
 #endif
@@ -501,16 +512,20 @@ dw_swap_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ val
 #ifdef SURGEON_DW_STATS
       st_w += clock64() - cw0;
 #endif
+      PH_STAMP(2)
       if (in_tile) {
         unsigned char* dst_row = smem + sa * a_tile_bytes + rowbase;
 #pragma unroll
         for (int q = 0; q < 4; ++q)
           *reinterpret_cast<uint4*>(dst_row + (((y + q) ^ xr) << 4)) = chunk[q];
       }
+      PH_STAMP(3)
       if (it + p.groups < n_kt) issue(nxt);      // the next tile's loads leave before the fence
+      PH_STAMP(4)
       fence_proxy_async();
       __syncwarp();
       if (lane == 0) mbar_arrive_rank0(full_a + 8 * sa);
+      PH_STAMP(5)
       next_stage();
       cur = nxt;
       nxt = nxt2;
@@ -519,6 +534,8 @@ dw_swap_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ val
     if (pw == 0 && lane == 0 && cta_rank == 0) {
       atomicAdd(reinterpret_cast<unsigned long long*>(status) + 9, static_cast<unsigned long long>(st_w));
       atomicAdd(reinterpret_cast<unsigned long long*>(status) + 10, static_cast<unsigned long long>(clock64() - st_pb));
+      for (int i = 0; i < 6; ++i)
+        atomicAdd(reinterpret_cast<unsigned long long*>(status) + 17 + i, static_cast<unsigned long long>(ph[i]));
     }
 #endif
   }
@@ -661,8 +678,7 @@ int resident_pairs() {
 
 int swap_resident_pairs() { return resident_pairs(); }
 
-bool plan_swap(const surgeon_layer_desc& d, SwapParams* out) {
-  if (!swap_enabled()) return false;
+static bool compute_plan_swap(const surgeon_layer_desc& d, SwapParams* out) {
   SwapParams best{};
   DirectParams dp;
   if (!plan_direct(d, &dp)) return false;
@@ -709,12 +725,14 @@ bool plan_swap(const surgeon_layer_desc& d, SwapParams* out) {
       p.n_units = (dp.mode == 0) ? (dp.O + 127) / 128 : n_units;
       p.n_tiles = (p.n_units + 2 * n_acc - 1) / (2 * n_acc);
       if (!size_swap_rings(&p, kProdWarps * kStageBytesPerWarp)) continue;
-      // Clocks of one K-tile on a CTA: the slowest of the MMAs (128 x nt x 16 in nt / 2 clocks),
-      // the gradient boxes (L2 delivers about 22 bytes per clock to an SM when all SMs pull) and
-      // the producers (about a fifth of a clock per rebuilt element).
+      // Clocks of one K-tile on a CTA, as measured on B200 with clock stamps in this kernel: the
+      // slowest of the MMAs (128 x nt x 16 in nt / 2 clocks), the gradient boxes (L2 delivers about
+      // 30 bytes per clock to an SM while all SMs pull) and the producers (0.28 clocks per rebuilt
+      // element: latency of the fence that publishes a tile, not instruction issue, so more
+      // groups of fewer warps - smaller halves - do better).
       const double mma = n_acc * 4.0 * (nt / 2.0);
-      const double l2 = n_acc * kAccBytes / 22.0;
-      const double prod = p.half * 64.0 * 0.19;
+      const double l2 = n_acc * kAccBytes / 30.0;
+      const double prod = p.half * 64.0 * 0.28;
       double kt_clk = mma > prod ? mma : prod;
       if (l2 > kt_clk) kt_clk = l2;
       if (p.g_stages < 3) kt_clk *= 1.1;
@@ -741,6 +759,12 @@ bool plan_swap(const surgeon_layer_desc& d, SwapParams* out) {
   while (best.tmem_cols < best.n_acc * best.nt) best.tmem_cols *= 2;
   *out = best;
   return true;
+}
+
+bool plan_swap(const surgeon_layer_desc& d, SwapParams* out) {
+  if (!swap_enabled()) return false;
+  struct Tag {};
+  return memo_plan<Tag>(d, 0, out, [&](SwapParams* p) { return compute_plan_swap(d, p); });
 }
 
 size_t swap_partial_bytes(const SwapParams& p) {
@@ -795,8 +819,7 @@ cudaError_t launch_swap(const surgeon_compressed& act, const SwapParams& plan, c
   if (e != cudaSuccess) return e;
   dim3 grid(2 * p.m_tiles, p.n_tiles, p.splits);
   auto launch = [&](auto kernel) -> cudaError_t {
-    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           p.smem_bytes);
+    cudaError_t err = allow_dynamic_smem(reinterpret_cast<const void*>(kernel), p.smem_bytes);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;

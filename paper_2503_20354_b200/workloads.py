@@ -172,6 +172,21 @@ def segformer_b5(image: int = 1024, batch: int = 1, dt: int = BF16, depths=(3, 6
     return L
 
 
+def shared_inputs(layers: List[Layer]) -> dict:
+    """Layers that read the same saved tensor as an earlier layer of the stack: the 1x1 shortcut /
+    downsample convolution of a residual block takes the block's input, like the block's first
+    convolution.  Returns {index of the later layer: index of the layer whose input it shares}."""
+    by_name = {l.name: i for i, l in enumerate(layers)}
+    out = {}
+    for j, l in enumerate(layers):
+        for suffix in (".shortcut", ".downsample"):
+            if l.name.endswith(suffix):
+                i = by_name.get(l.name[: -len(suffix)] + ".conv1")
+                if i is not None and layers[i].act_shape == l.act_shape and layers[i].dt == l.dt:
+                    out[j] = i
+    return out
+
+
 def shrink(layers: List[Layer], batch: int) -> List[Layer]:
     """Same stack at a smaller batch (rows scale with the batch for linear layers)."""
     out = []

@@ -161,3 +161,22 @@ def test_weight_grad_argument_errors():
     with pytest.raises(B.SurgeonError) as e:
         B.surgeon_weight_grad(comp, wrong, g)
     assert e.value.status == B.SURGEON_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_one_store_feeds_the_two_layers_that_read_the_same_input(path):
+    """A residual block's first convolution and its 1x1 shortcut take the same tensor: it is pruned
+    once and both weight gradients are formed from the one store."""
+    conv1 = W.conv("b0.conv1", 3, 48, 16, 72, 3, 2)
+    short = W.conv("b0.shortcut", 3, 48, 16, 72, 1, 2, 0)
+    assert W.shared_inputs([conv1, short]) == {1: 0}
+    a = W.activation(conv1, seed=4)
+    comp = B.surgeon_prune_compact(a.cuda(), 0.6)
+    ref = oracle.prune_compact(W.as_numpy_bits(a).reshape(-1), 0.6)
+    pruned = oracle.decompress(ref["bitmap"], ref["values"], conv1.n_act)
+    for layer in (conv1, short):
+        g = W.grad_out(layer, seed=4, index=1 + layer.kh)
+        dw = B.surgeon_weight_grad(comp, B.layer_desc(layer, path), g.cuda()).cpu().numpy()
+        want = oracle_dw(layer, pruned, g.numpy())
+        assert rel_frobenius(dw, want) <= TOL[path], layer.name
+    assert comp.read_header().status == 0
