@@ -65,6 +65,9 @@ def _load():
         lib.oracle_dw_conv2d.restype = None
         lib.oracle_dw_conv2d.argtypes = [c.c_void_p, c.c_int, c.c_void_p] + [c.c_int64] * 9 + [
             c.c_void_p]
+        lib.oracle_dw_conv2d_grouped.restype = None
+        lib.oracle_dw_conv2d_grouped.argtypes = [c.c_void_p, c.c_int, c.c_void_p] + [c.c_int64] * 10 + [
+            c.c_void_p]
         lib.oracle_dw_conv2d_entry.restype = c.c_double
         lib.oracle_dw_conv2d_entry.argtypes = [c.c_void_p, c.c_int, c.c_void_p] + [c.c_int64] * 13
         lib.oracle_dw_linear_entry.restype = c.c_double
@@ -224,6 +227,23 @@ def dw_conv2d(a: np.ndarray, g: np.ndarray, kh: int, kw: int, stride: int, pad: 
     dw = np.zeros((O, C, kh, kw), dtype=np.float64)
     _load().oracle_dw_conv2d(_ptr(a), _dt_of(a), _ptr(g), B, C, H, W, O, kh, kw, stride, pad,
                              _ptr(dw))
+    return dw
+
+
+def dw_conv2d_grouped(a: np.ndarray, g: np.ndarray, kh: int, kw: int, stride: int, pad: int,
+                      groups: int) -> np.ndarray:
+    """Weight gradient of a grouped conv2d (ResNeXt's 3x3 layers, depthwise convolutions):
+    a NCHW [B,C,H,W], g [B,O,OH,OW] f32 -> dw [O,C/groups,KH,KW] float64."""
+    a = np.ascontiguousarray(a)
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    B, C, H, W = a.shape
+    O = g.shape[1]
+    assert groups >= 1 and C % groups == 0 and O % groups == 0, (C, O, groups)
+    oh, ow = conv_out_hw(H, W, kh, kw, stride, pad)
+    assert g.shape == (B, O, oh, ow), (g.shape, (B, O, oh, ow))
+    dw = np.zeros((O, C // groups, kh, kw), dtype=np.float64)
+    _load().oracle_dw_conv2d_grouped(_ptr(a), _dt_of(a), _ptr(g), B, C, H, W, O, kh, kw, stride,
+                                     pad, groups, _ptr(dw))
     return dw
 
 

@@ -307,6 +307,47 @@ double oracle_dw_conv2d_entry(const void* a, int dt, const float* g, int64_t B, 
   return acc;
 }
 
+// Weight gradient of a GROUPED 2-D cross-correlation (the layer type of ResNeXt's 3x3 convolutions
+// and of a depthwise convolution; the paper adapts ResNeXt-29 on CIFAR100-C, Section 5.1).  The
+// standard definition: input and output channels are cut into `groups` equal consecutive ranges,
+// output channel o belongs to group g = o / (O / groups) and sees only the C / groups input
+// channels of that group:
+//   dw[o, c', r, s] = sum_{b, y, x} g[b, o, y, x] * a[b, g*(C/groups) + c', y*stride + r - pad,
+//                                                      x*stride + s - pad]
+// a: NCHW [B, C, H, W] of dt; g: [B, O, OH, OW] fp32; dw: [O, C/groups, KH, KW] double.
+void oracle_dw_conv2d_grouped(const void* a, int dt, const float* g, int64_t B, int64_t C,
+                              int64_t H, int64_t W, int64_t O, int64_t KH, int64_t KW,
+                              int64_t stride, int64_t pad, int64_t groups, double* dw) {
+  const int64_t OH = (H + 2 * pad - KH) / stride + 1;
+  const int64_t OW = (W + 2 * pad - KW) / stride + 1;
+  const int64_t Cg = C / groups, Og = O / groups;
+#pragma omp parallel for schedule(static)
+  for (int64_t o = 0; o < O; ++o) {
+    const int64_t grp = o / Og;
+    for (int64_t cl = 0; cl < Cg; ++cl) {
+      const int64_t c = grp * Cg + cl;
+      for (int64_t r = 0; r < KH; ++r) {
+        for (int64_t s = 0; s < KW; ++s) {
+          double acc = 0.0;
+          for (int64_t b = 0; b < B; ++b) {
+            for (int64_t y = 0; y < OH; ++y) {
+              const int64_t iy = y * stride + r - pad;
+              if (iy < 0 || iy >= H) continue;
+              for (int64_t xo = 0; xo < OW; ++xo) {
+                const int64_t ix = xo * stride + s - pad;
+                if (ix < 0 || ix >= W) continue;
+                acc += static_cast<double>(g[((b * O + o) * OH + y) * OW + xo]) *
+                       value_of(a, ((b * C + c) * H + iy) * W + ix, dt);
+              }
+            }
+          }
+          dw[((o * Cg + cl) * KH + r) * KW + s] = acc;
+        }
+      }
+    }
+  }
+}
+
 // One entry of the linear weight gradient.
 double oracle_dw_linear_entry(const void* a, int dt, const float* g, int64_t T, int64_t C,
                               int64_t O, int64_t o, int64_t c) {

@@ -148,3 +148,64 @@ def test_ratio_ends_and_linearity_through_the_store(bf16):
     removed = removed.reshape(a.shape)
     s = oracle.dw_conv2d(kept, g, 3, 3, 1, 1) + oracle.dw_conv2d(removed, g, 3, 3, 1, 1)
     np.testing.assert_allclose(s, dense, rtol=1e-12, atol=1e-14)
+
+
+# ---- grouped convolutions (ResNeXt's 3x3 layers, depthwise convolutions) --------------------------
+
+GROUPED_CASES = [
+    # B, C, H, W, O, k, stride, pad, groups
+    (2, 8, 7, 7, 12, 3, 1, 1, 4),
+    (2, 6, 8, 6, 6, 3, 2, 1, 6),      # depthwise, stride 2
+    (1, 4, 9, 9, 8, 3, 1, 0, 2),
+    (3, 6, 5, 5, 9, 1, 1, 0, 3),
+    (1, 4, 10, 10, 4, 5, 2, 2, 4),    # depthwise 5x5
+]
+
+
+@pytest.mark.parametrize("case", GROUPED_CASES)
+def test_grouped_conv_matches_torch_autograd_fp64(case):
+    B, C, H, Wd, O, k, s, p, groups = case
+    rng = np.random.default_rng(11)
+    a32 = rng.standard_normal((B, C, H, Wd)).astype(np.float32)
+    oh, ow = oracle.conv_out_hw(H, Wd, k, k, s, p)
+    g32 = rng.standard_normal((B, O, oh, ow)).astype(np.float32)
+    a = torch.from_numpy(a32.astype(np.float64))
+    g = torch.from_numpy(g32.astype(np.float64))
+    w = torch.zeros(O, C // groups, k, k, dtype=torch.float64, requires_grad=True)
+    y = torch.nn.functional.conv2d(a, w, None, stride=s, padding=p, groups=groups)
+    (y * g).sum().backward()
+    got = oracle.dw_conv2d_grouped(a32, g32, k, k, s, p, groups)
+    assert got.shape == (O, C // groups, k, k)
+    np.testing.assert_allclose(got, w.grad.numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_one_group_is_the_ungrouped_gradient():
+    rng = np.random.default_rng(12)
+    a = rng.standard_normal((2, 5, 6, 7)).astype(np.float32)
+    g = rng.standard_normal((2, 4, 6, 7)).astype(np.float32)
+    assert np.array_equal(oracle.dw_conv2d_grouped(a, g, 3, 3, 1, 1, 1), oracle.dw_conv2d(a, g, 3, 3, 1, 1))
+
+
+def test_groups_are_independent_ungrouped_problems():
+    """Group g of a grouped layer is the ungrouped layer on its own slices of the channels."""
+    rng = np.random.default_rng(13)
+    a = rng.standard_normal((2, 6, 6, 6)).astype(np.float32)
+    g = rng.standard_normal((2, 9, 3, 3)).astype(np.float32)
+    full = oracle.dw_conv2d_grouped(a, g, 3, 3, 2, 1, 3)
+    for grp in range(3):
+        part = oracle.dw_conv2d(a[:, 2 * grp:2 * grp + 2], g[:, 3 * grp:3 * grp + 3], 3, 3, 2, 1)
+        assert np.array_equal(full[3 * grp:3 * grp + 3], part)
+
+
+def test_depthwise_2x2_worked_by_hand():
+    """One image, two channels, 2x2 maps, 1x1 kernel, groups = channels: each weight is the plain
+    correlation of its own channel's gradient and activation."""
+    a = np.array([[[[1, 2], [3, 4]], [[-1, 0], [2, 5]]]], dtype=np.float32)
+    g = np.array([[[[1, 0], [0, 2]], [[3, 1], [1, 1]]]], dtype=np.float32)
+    dw = oracle.dw_conv2d_grouped(a, g, 1, 1, 1, 0, 2)
+    # channel 0: 1*1 + 0*2 + 0*3 + 2*4 = 9;  channel 1: 3*(-1) + 1*0 + 1*2 + 1*5 = 4
+    assert dw.reshape(-1).tolist() == [9.0, 4.0]
+    # a 2x2 kernel without padding has one output position: dw = g * a window
+    g1 = np.array([[[[2.0]], [[-1.0]]]], dtype=np.float32)
+    dw2 = oracle.dw_conv2d_grouped(a, g1, 2, 2, 1, 0, 2)
+    assert np.array_equal(dw2[0, 0], 2.0 * a[0, 0]) and np.array_equal(dw2[1, 0], -1.0 * a[0, 1])
