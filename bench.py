@@ -7,7 +7,7 @@ gradient of every layer from its compressed store (its Reshape and gradient step
 JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                  [--workload all|vit|wrn28|resnet50|resnet50_uniform|tiny|segformer|sweep]
+                  [--workload all|vit|wrn28|resnet50|resnet50_uniform|resnext29|tiny|segformer|sweep]
                   [--batch B] [--path tc|fp32]
 
 The default workload `all` runs, in one process, the ViT-B/16-shaped stack (the headline: `value`,
@@ -97,13 +97,15 @@ def get_layers(workload: str, batch):
         return W.resnet50(batch or 64), "ResNet-50-shaped stack, 224x224, batch %d, bf16 activations" % (batch or 64)
     if workload == "vit":
         return W.vit_b16(batch or 64), "ViT-B/16-shaped stack, batch %d, bf16 activations" % (batch or 64)
+    if workload == "resnext29":
+        return W.resnext29(batch or 200), "ResNeXt-29 (32x4d)-shaped stack, 32x32, batch %d, fp32 activations, grouped 3x3 convolutions" % (batch or 200)
     if workload == "segformer":
         return W.segformer_b5(1024, batch or 1), "linear layers of a Segformer-B5-shaped encoder, 1024x1024, batch %d, bf16 activations" % (batch or 1)
     raise SystemExit("unknown workload %r" % workload)
 
 
 # output-gradient scale per workload (the tiny and WideResNet configs: 0.01; ResNet-50 / ViT: 1e-3)
-SIGMA = {"wrn28": 0.01, "tiny": 0.01, "segformer": 0.01, "resnet50": 1e-3, "resnet50_uniform": 1e-3, "vit": 1e-3}
+SIGMA = {"wrn28": 0.01, "tiny": 0.01, "segformer": 0.01, "resnext29": 0.01, "resnet50": 1e-3, "resnet50_uniform": 1e-3, "vit": 1e-3}
 
 
 def prune_alg_bytes(layer, n_keep: int) -> int:
@@ -778,7 +780,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="all",
-                    choices=["all", "vit", "wrn28", "resnet50", "resnet50_uniform", "tiny", "segformer", "sweep"])
+                    choices=["all", "vit", "wrn28", "resnet50", "resnet50_uniform", "resnext29", "tiny", "segformer", "sweep"])
     ap.add_argument("--sweep-sizes", type=int, default=6, help="how many of 2^20,22,24,26,28,30 the sweep covers")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--layers", default=None, help="comma-separated layer names: run only these (profiling)")

@@ -212,7 +212,7 @@ surgeon_status surgeon_prune_compact_static(const void* x, int64_t n, surgeon_dt
                                             double ratio, surgeon_compressed* out,
                                             void* cuda_stream);
 
-/* Layer geometry for the weight gradient.  dilation 1, groups 1. */
+/* Layer geometry for the weight gradient.  Dilation 1. */
 typedef struct surgeon_layer_desc {
   int32_t kind;  /* 0 = linear: activation [batch, c_in] (batch = rows T; h = w = kh = kw = 1,
                     stride = 1, pad = 0);  1 = conv2d: activation NCHW [batch, c_in, h, w]       */
@@ -220,6 +220,13 @@ typedef struct surgeon_layer_desc {
   int32_t c_out, kh, kw, stride, pad;
   int32_t path;  /* 0 = tensor-core path (bf16 x bf16 -> fp32, tcgen05/TMEM);
                     1 = fp32 CUDA-core path                                                      */
+  int32_t groups; /* conv2d: channel groups (0 or 1 = an ordinary convolution).  groups > 1 (the
+                    3x3 layers of ResNeXt, the network the paper adapts on CIFAR100-C in Section
+                    5.1; groups = c_in = c_out is a depthwise convolution): c_in and c_out must
+                    be multiples of it, output channel o reads only the c_in / groups input
+                    channels of group o / (c_out / groups), and dw is [c_out, c_in / groups, kh,
+                    kw].  A group's problem is far smaller than a tensor-core tile, so both
+                    values of `path` run the same fp32 CUDA-core kernel for such a layer.       */
 } surgeon_layer_desc;
 
 /* Device scratch (bytes) surgeon_weight_grad needs for this layer and path; 0 on a bad desc. */
@@ -231,7 +238,9 @@ size_t surgeon_weight_grad_workspace(const surgeon_layer_desc* d);
  *   linear:  dw[o, c]       = sum_t        grad_out[t, o]       * A[t, c]
  *   conv2d:  dw[o, c, r, s] = sum_{b,y,x}  grad_out[b, o, y, x] * A[b, c, y*stride + r - pad,
  *                                                                   x*stride + s - pad]
- *            (terms outside the input are zero; oh = (h + 2*pad - kh)/stride + 1, same for ow)
+ *            (terms outside the input are zero; oh = (h + 2*pad - kh)/stride + 1, same for ow;
+ *            with groups > 1, c counts inside the group of o: input channel
+ *            (o / (c_out/groups)) * (c_in/groups) + c)
  * where A is the pruned activation (zero where the bitmap bit is 0).  dw has the layout of a
  * PyTorch weight, [c_out, c_in, kh, kw], i.e. the transpose of Eq. 2's A^T * dL/dA_{i+1}.
  * act: HOST pointer to a struct of DEVICE pointers written by surgeon_prune_compact on the
@@ -239,8 +248,9 @@ size_t surgeon_weight_grad_workspace(const surgeon_layer_desc* d);
  * [batch, c_out, oh, ow] (conv2d) or [batch, c_out] (linear).  dw: device, fp32.
  * accumulate = 0 overwrites dw, 1 adds to it.  The summation order is fixed, so results are
  * bitwise reproducible from call to call.  Asynchronous on cuda_stream.
- * Errors: INVALID_ARG, BUFFER_TOO_SMALL, UNSUPPORTED (groups/dilation are not expressible;
- * sizes beyond 2^31-1 elements), CUDA.
+ * Errors: INVALID_ARG, BUFFER_TOO_SMALL, UNSUPPORTED (dilation is not expressible; sizes beyond
+ * 2^31-1 elements; a grouped layer whose group has more than 1024 blocks of
+ * (8 output channels) x (c_in/groups * kh * kw) weights), CUDA.
  * ---------------------------------------------------------------------------------------- */
 surgeon_status surgeon_weight_grad(const surgeon_compressed* act, const surgeon_layer_desc* d,
                                    const float* grad_out, float* dw, int32_t accumulate,

@@ -49,7 +49,7 @@ class Compressed(C.Structure):
 
 class LayerDesc(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("kind", "batch", "c_in", "h", "w", "c_out", "kh", "kw",
-                                         "stride", "pad", "path")]
+                                         "stride", "pad", "path", "groups")]
 
 
 _lib = None
@@ -331,7 +331,7 @@ def surgeon_decompress(act: CompressedActivation, stream: Optional[torch.cuda.St
 def layer_desc(layer, path: int) -> LayerDesc:
     """LayerDesc from any object with kind/batch/c_in/h/w/c_out/kh/kw/stride/pad attributes."""
     return LayerDesc(layer.kind, layer.batch, layer.c_in, layer.h, layer.w, layer.c_out, layer.kh,
-                     layer.kw, layer.stride, layer.pad, int(path))
+                     layer.kw, layer.stride, layer.pad, int(path), int(getattr(layer, "groups", 1)))
 
 
 def surgeon_weight_grad_workspace(desc: LayerDesc) -> int:
@@ -345,7 +345,7 @@ def surgeon_weight_grad(act: CompressedActivation, desc: LayerDesc, grad_out: to
     """dW of the layer from the compressed activation and fp32 ``grad_out``; returns ``dw``."""
     if grad_out.dtype != torch.float32 or not grad_out.is_cuda or not grad_out.is_contiguous():
         raise ValueError("grad_out must be a contiguous fp32 CUDA tensor")
-    shape = (desc.c_out, desc.c_in, desc.kh, desc.kw) if desc.kind == 1 else (desc.c_out, desc.c_in)
+    shape = (desc.c_out, desc.c_in // max(desc.groups, 1), desc.kh, desc.kw) if desc.kind == 1 else (desc.c_out, desc.c_in)
     if dw is None:
         if accumulate:
             raise ValueError("accumulate needs an existing dw")

@@ -90,6 +90,8 @@ bool desc_ok(const surgeon_layer_desc* d, surgeon_status* why) {
                        d->pad != 0))
     return false;
   if (d->h + 2 * d->pad < d->kh || d->w + 2 * d->pad < d->kw) return false;
+  if (d->groups < 0) return false;
+  if (d->groups > 1 && (d->kind != 1 || d->c_in % d->groups != 0 || d->c_out % d->groups != 0)) return false;
   *why = SURGEON_ERR_UNSUPPORTED;
   const long long oh = (d->h + 2 * d->pad - d->kh) / d->stride + 1;
   const long long ow = (d->w + 2 * d->pad - d->kw) / d->stride + 1;
@@ -237,7 +239,8 @@ surgeon_status surgeon_prune_compact_flags(const void* x, int64_t n, surgeon_dty
 size_t surgeon_weight_grad_workspace(const surgeon_layer_desc* d) {
   surgeon_status why;
   if (!desc_ok(d, &why)) return 0;
-  const size_t b = d->path == 1 ? weight_grad_fp32_workspace(*d) : weight_grad_tc_workspace(*d);
+  const size_t b = d->groups > 1 ? weight_grad_grouped_workspace(*d)
+                   : (d->path == 1 ? weight_grad_fp32_workspace(*d) : weight_grad_tc_workspace(*d));
   return (b + 255) & ~static_cast<size_t>(255);
 }
 
@@ -255,9 +258,11 @@ surgeon_status surgeon_weight_grad(const surgeon_compressed* act, const surgeon_
   const size_t need = surgeon_weight_grad_workspace(d);
   if (need > 0 && (!workspace || workspace_bytes < need)) return SURGEON_ERR_BUFFER_TOO_SMALL;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (d->groups > 1 && need == 0) return SURGEON_ERR_UNSUPPORTED;
   const cudaError_t e =
-      d->path == 1 ? launch_weight_grad_fp32(*act, *d, grad_out, dw, accumulate ? 1 : 0, workspace, s)
-                   : launch_weight_grad_tc(*act, *d, grad_out, dw, accumulate ? 1 : 0, workspace, s);
+      d->groups > 1 ? launch_weight_grad_grouped(*act, *d, grad_out, dw, accumulate ? 1 : 0, workspace, s)
+      : d->path == 1 ? launch_weight_grad_fp32(*act, *d, grad_out, dw, accumulate ? 1 : 0, workspace, s)
+                     : launch_weight_grad_tc(*act, *d, grad_out, dw, accumulate ? 1 : 0, workspace, s);
   if (e == cudaErrorNotSupported) return SURGEON_ERR_UNSUPPORTED;
   if (e != cudaSuccess && getenv("SURGEON_VERBOSE"))
     fprintf(stderr, "surgeon_weight_grad: %s\n", cudaGetErrorString(e));

@@ -114,6 +114,11 @@ cudaError_t launch_weight_grad_fp32(const surgeon_compressed& act, const surgeon
                                     const float* grad_out, float* dw, int accumulate,
                                     void* workspace, cudaStream_t stream);
 
+size_t weight_grad_grouped_workspace(const surgeon_layer_desc& d);
+cudaError_t launch_weight_grad_grouped(const surgeon_compressed& act, const surgeon_layer_desc& d,
+                                       const float* grad_out, float* dw, int accumulate,
+                                       void* workspace, cudaStream_t stream);
+
 size_t weight_grad_tc_workspace(const surgeon_layer_desc& d);
 cudaError_t launch_weight_grad_tc(const surgeon_compressed& act, const surgeon_layer_desc& d,
                                   const float* grad_out, float* dw, int accumulate,

@@ -36,6 +36,7 @@ class Layer:
     dist: str = "relu_normal"   # distribution of the saved input activation
     dt: int = F32               # dtype of the saved activation
     rows_per_sample: int = 0    # linear layers: rows T per sample (0: see shrink)
+    groups: int = 1             # conv2d: channel groups (c_in = c_out = groups: depthwise)
 
     @property
     def oh(self) -> int:
@@ -59,11 +60,11 @@ class Layer:
 
     @property
     def dw_shape(self):
-        return (self.c_out, self.c_in, self.kh, self.kw) if self.kind == 1 else (self.c_out, self.c_in)
+        return (self.c_out, self.c_in // self.groups, self.kh, self.kw) if self.kind == 1 else (self.c_out, self.c_in)
 
     @property
     def n_weight(self) -> int:
-        return self.c_out * self.c_in * self.kh * self.kw
+        return self.c_out * (self.c_in // self.groups) * self.kh * self.kw
 
     @property
     def gemm_k(self) -> int:
@@ -83,10 +84,10 @@ class Layer:
         return self.n_act * (4 if self.dt == F32 else 2)
 
 
-def conv(name, batch, c_in, hw, c_out, k, stride=1, pad=None, dist="relu_normal", dt=F32) -> Layer:
+def conv(name, batch, c_in, hw, c_out, k, stride=1, pad=None, dist="relu_normal", dt=F32, groups=1) -> Layer:
     if pad is None:
         pad = k // 2
-    return Layer(name, 1, batch, c_in, hw, hw, c_out, k, k, stride, pad, dist, dt)
+    return Layer(name, 1, batch, c_in, hw, hw, c_out, k, k, stride, pad, dist, dt, 0, groups)
 
 
 def linear(name, rows, c_in, c_out, dist="normal", dt=BF16, rows_per_sample=0) -> Layer:
@@ -133,6 +134,31 @@ def resnet50(batch: int = 64, dt: int = BF16) -> List[Layer]:
                 L.append(conv(p + ".downsample", batch, c_prev, hw, width * 4, 1, s, 0, dt=dt))
             c_prev, hw = width * 4, hw_out
     L.append(linear("fc", batch, 2048, 1000, dist="abs_normal", dt=dt))
+    return L
+
+
+def resnext29(batch: int = 200, dt: int = F32, cardinality: int = 32, base_width: int = 4) -> List[Layer]:
+    """The conv layers and the FC layer of ResNeXt-29 (32x4d) on 32x32 inputs, the network the paper
+    adapts on CIFAR100-C (Section 5.1) and times on the embedded board (Section 5.5): a 3x3 stem,
+    three stages of three bottleneck blocks (1x1 reduce, GROUPED 3x3 with `cardinality` groups,
+    1x1 expand; a 1x1 shortcut convolution in the first block of a stage), stage outputs
+    256 / 512 / 1024 channels on 32 / 16 / 8 wide maps."""
+    L = [conv("conv1", batch, 3, 32, 64, 3, dist="normal", dt=dt)]
+    c_prev, hw = 64, 32
+    for st in range(3):
+        d = cardinality * base_width * (2 ** st)          # width of the grouped convolution
+        c_out = 256 * (2 ** st)
+        for b in range(3):
+            s = 2 if (st > 0 and b == 0) else 1
+            n = f"s{st + 1}b{b}"
+            L.append(conv(n + ".conv1", batch, c_prev, hw, d, 1, 1, 0, dt=dt))
+            L.append(conv(n + ".conv2", batch, d, hw, d, 3, s, 1, dt=dt, groups=cardinality))
+            hw_out = hw // s
+            L.append(conv(n + ".conv3", batch, d, hw_out, c_out, 1, 1, 0, dt=dt))
+            if b == 0:
+                L.append(conv(n + ".shortcut", batch, c_prev, hw, c_out, 1, s, 0, dt=dt))
+            c_prev, hw = c_out, hw_out
+    L.append(linear("fc", batch, 1024, 100, dist="abs_normal", dt=dt))
     return L
 
 

@@ -36,7 +36,7 @@ def test_exports_every_declared_symbol():
 def test_struct_layouts_match_header():
     assert ctypes.sizeof(B.Header) == 32
     assert ctypes.sizeof(B.Compressed) == 48
-    assert ctypes.sizeof(B.LayerDesc) == 44
+    assert ctypes.sizeof(B.LayerDesc) == 48
 
 
 def test_ratios_match_oracle_and_fixture():
