@@ -15,7 +15,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsurgeon.so")
+# SURGEON_LIB names another build of the same library (the checked build libsurgeon_bounds.so)
+LIB_PATH = os.environ.get("SURGEON_LIB") or os.path.join(_HERE, "libsurgeon.so")
 
 SURGEON_OK = 0
 SURGEON_ERR_INVALID_ARG = 1

@@ -1017,8 +1017,10 @@ __device__ __forceinline__ void compact_tile(const typename Elem<DT>::type* __re
 #pragma unroll
       for (int i = 0; i < EPV; ++i) {
         if ((keep >> i) & 1u) {
-          *dst++ = (DT == 0) ? static_cast<E>(w[i % 4])
+          if (SURGEON_IN_BOUNDS(dst - values, hdr->n_keep, &hdr->status))
+            *dst = (DT == 0) ? static_cast<E>(w[i % 4])
                              : static_cast<E>((w[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
+          ++dst;
         }
       }
       kept_before += total;
@@ -1319,7 +1321,9 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
         const uint32_t v_end = end / EPV;          // one past the last whole vector
         if (mis) {
           const uint32_t sl = mis + lane;
-          if (sl < static_cast<uint32_t>(EPV) && sl < end) gbase[sl] = outp[swz(sl)];
+          if (sl < static_cast<uint32_t>(EPV) && sl < end &&
+              SURGEON_IN_BOUNDS(kept_before - mis + sl, hdr->n_keep, &hdr->status))
+            gbase[sl] = outp[swz(sl)];
         }
         for (uint32_t g = v_first + lane; g < v_end; g += 32) {
           // the four words of a vector share their row: one 16-byte load, words permuted by the XOR
@@ -1328,17 +1332,20 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
           uint4 u = *reinterpret_cast<const uint4*>(region + (la ^ (xr & 0x70u)));
           if (xr & 4u) { uint32_t t = u.x; u.x = u.y; u.y = t; t = u.z; u.z = u.w; u.w = t; }
           if (xr & 8u) { uint32_t t = u.x; u.x = u.z; u.z = t; t = u.y; u.y = u.w; u.w = t; }
-          *reinterpret_cast<uint4*>(gbase + g * EPV) = u;
+          if (SURGEON_IN_BOUNDS(kept_before - mis + g * EPV + EPV - 1, hdr->n_keep, &hdr->status))
+            *reinterpret_cast<uint4*>(gbase + g * EPV) = u;
         }
         const uint32_t t0 = (v_end > v_first ? v_end : v_first) * EPV;
-        if (t0 + lane < end) gbase[t0 + lane] = outp[swz(t0 + lane)];
+        if (t0 + lane < end && SURGEON_IN_BOUNDS(kept_before - mis + t0 + lane, hdr->n_keep, &hdr->status))
+          gbase[t0 + lane] = outp[swz(t0 + lane)];
       } else {
         // a full chunk with a misaligned destination: no room for the shift, element-wise vectors
         E* dst = values + kept_before;
         uint32_t head = mis ? EPV - mis : 0;
         if (head > total) head = total;
         const uint32_t n_vec = (total - head) / EPV;
-        if (lane < head) dst[lane] = outp[swz(lane)];
+        if (lane < head && SURGEON_IN_BOUNDS(kept_before + lane, hdr->n_keep, &hdr->status))
+          dst[lane] = outp[swz(lane)];
         for (uint32_t v = lane; v < n_vec; v += 32) {
           const uint32_t b = head + v * EPV;
           uint4 o;
@@ -1350,10 +1357,12 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
                            outp[swz(b + 4 % EPV)] | (static_cast<uint32_t>(outp[swz(b + 5 % EPV)]) << 16),
                            outp[swz(b + 6 % EPV)] | (static_cast<uint32_t>(outp[swz(b + 7 % EPV)]) << 16));
           }
-          *reinterpret_cast<uint4*>(dst + head + v * EPV) = o;
+          if (SURGEON_IN_BOUNDS(kept_before + head + v * EPV + EPV - 1, hdr->n_keep, &hdr->status))
+            *reinterpret_cast<uint4*>(dst + head + v * EPV) = o;
         }
         const uint32_t done = head + n_vec * EPV;
-        if (lane < total - done) dst[done + lane] = outp[swz(done + lane)];
+        if (lane < total - done && SURGEON_IN_BOUNDS(kept_before + done + lane, hdr->n_keep, &hdr->status))
+          dst[done + lane] = outp[swz(done + lane)];
       }
     }
     tc::fence_proxy_async();     // this warp's writes to the stage precede the next TMA fill

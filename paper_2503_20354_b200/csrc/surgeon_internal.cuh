@@ -159,6 +159,18 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Checked builds (-DSURGEON_BOUNDS, the library's stand-in for a memory checker): every guarded
+// global store tests its index against the size the host computed for the buffer; an index
+// outside records SURGEON_ERR_INTERNAL in `status_word` and the store is skipped.  In the
+// ordinary build the test compiles away.
+#ifdef SURGEON_BOUNDS
+#define SURGEON_IN_BOUNDS(idx, limit, status_word)                                              \
+  ((static_cast<unsigned long long>(idx) < static_cast<unsigned long long>(limit)) ||           \
+   (atomicMax((status_word), static_cast<uint32_t>(SURGEON_ERR_INTERNAL)), false))
+#else
+#define SURGEON_IN_BOUNDS(idx, limit, status_word) true
+#endif
+
 __device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31; }
 __device__ __forceinline__ uint32_t lanemask_lt() {
   uint32_t m;

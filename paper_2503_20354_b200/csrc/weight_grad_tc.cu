@@ -416,7 +416,10 @@ dw_tc_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ value
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
             const int o = o0 + col + e;
-            if (o < p.O) out[static_cast<long long>(o) * p.n_gemm + nn] = __uint_as_float(r[e]);
+            if (o < p.O && SURGEON_IN_BOUNDS(static_cast<long long>(split) * p.O * p.n_gemm +
+                                                 static_cast<long long>(o) * p.n_gemm + nn,
+                                             static_cast<long long>(p.splits) * p.O * p.n_gemm, status))
+              out[static_cast<long long>(o) * p.n_gemm + nn] = __uint_as_float(r[e]);
           }
         }
       }
@@ -662,7 +665,10 @@ dw_conv_im2col_kernel(const uint32_t* __restrict__ bitmap, const void* __restric
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
             const int o = o0 + col + e;
-            if (o < p.O) out[static_cast<long long>(o) * p.n_gemm + nn] = __uint_as_float(r[e]);
+            if (o < p.O && SURGEON_IN_BOUNDS(static_cast<long long>(split) * p.O * p.n_gemm +
+                                                 static_cast<long long>(o) * p.n_gemm + nn,
+                                             static_cast<long long>(p.splits) * p.O * p.n_gemm, status))
+              out[static_cast<long long>(o) * p.n_gemm + nn] = __uint_as_float(r[e]);
           }
         }
       }

@@ -571,7 +571,10 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         if (lane_grp * 32 + static_cast<int>(lane) < rows_here) {
 #pragma unroll
           for (int e = 0; e < 16; ++e)
-            if (e < n_ok) out[static_cast<long long>(row0 + e) * p.C + c] = __uint_as_float(r[e]);
+            if (e < n_ok && SURGEON_IN_BOUNDS(static_cast<long long>(split) * p.O * p.C +
+                                                  static_cast<long long>(row0 + e) * p.C + c,
+                                              static_cast<long long>(p.splits) * p.O * p.C, status))
+              out[static_cast<long long>(row0 + e) * p.C + c] = __uint_as_float(r[e]);
         }
       }
     } else if (!done && lane == 0) {

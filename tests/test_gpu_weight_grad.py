@@ -180,3 +180,24 @@ def test_one_store_feeds_the_two_layers_that_read_the_same_input(path):
         want = oracle_dw(layer, pruned, g.numpy())
         assert rel_frobenius(dw, want) <= TOL[path], layer.name
     assert comp.read_header().status == 0
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("layer", [SHAPES[1], SHAPES[2], SHAPES[4], SHAPES[10], SHAPES[19], SHAPES[22], SHAPES[36]],
+                         ids=lambda l: l.name)
+def test_output_and_scratch_stay_inside_their_buffers(layer, path):
+    """dw and the scratch sit at the front of larger buffers filled with a pattern: the words after
+    `dw` and after the size surgeon_weight_grad_workspace reports must come back untouched."""
+    a, g = W.activation(layer, seed=5).cuda(), W.grad_out(layer, seed=5).cuda()
+    comp = B.surgeon_prune_compact(a, 0.6)
+    desc = B.layer_desc(layer, path)
+    need = B.surgeon_weight_grad_workspace(desc)
+    n_dw = int(np.prod(layer.dw_shape))
+    big_dw = torch.full((n_dw + 256,), 777.0, device="cuda")
+    big_ws = torch.full((need + 1024,), 0x5A, dtype=torch.uint8, device="cuda")
+    dw = big_dw[:n_dw].view(layer.dw_shape)
+    B.surgeon_weight_grad(comp, desc, g, dw=dw, workspace=big_ws[:need])
+    torch.cuda.synchronize()
+    assert bool((big_dw[n_dw:] == 777.0).all()) and bool((big_ws[need:] == 0x5A).all())
+    ref = B.surgeon_weight_grad(comp, desc, g)
+    assert torch.equal(dw, ref)
