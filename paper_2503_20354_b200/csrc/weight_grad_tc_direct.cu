@@ -160,9 +160,23 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
       uint32_t pa = 0, pb = 0, accum = 0;
       int sa = 0, sb = 0;
       bool ok = true;
+#ifdef SURGEON_DW_STATS
+      // clock stamps of the issuing thread (a build with -DSURGEON_DW_STATS; read from the scratch
+      // status area by paper_2503_20354_b200/diagnostics.py): where a K-tile's time goes
+      long long st_g = 0, st_a = 0;
+      const long long st_begin = clock64();
+#endif
       for (int it = 0; it < n_kt; ++it) {
+#ifdef SURGEON_DW_STATS
+        const long long c0 = clock64();
+        ok = mbar_wait_suspend(full_b + 8 * sb, pb);
+        const long long c1 = clock64();
+        ok = ok && (PAIR ? mbar_wait_suspend_cluster(full_a + 8 * sa, pa) : mbar_wait_suspend(full_a + 8 * sa, pa));
+        st_g += c1 - c0; st_a += clock64() - c1;
+#else
         ok = mbar_wait_suspend(full_b + 8 * sb, pb) &&
              (PAIR ? mbar_wait_suspend_cluster(full_a + 8 * sa, pa) : mbar_wait_suspend(full_a + 8 * sa, pa));
+#endif
         if (!ok) break;
         tc_fence_after();
         if (n_acc_here == 1) umma_ktile<1, kStep, PAIR>(tmem_base, p.acc_n, da, db, acc_inc, idesc, accum);
@@ -176,6 +190,12 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         if (++sb == p.b_stages) { sb = 0; pb ^= 1; db = b_base; } else { db += b_inc; }
       }
       if (!ok) { fail = 1; atomicMax(status, static_cast<uint32_t>(SURGEON_ERR_TIMEOUT)); }
+#ifdef SURGEON_DW_STATS
+      atomicAdd(reinterpret_cast<unsigned long long*>(status) + 4, static_cast<unsigned long long>(st_g));
+      atomicAdd(reinterpret_cast<unsigned long long*>(status) + 5, static_cast<unsigned long long>(st_a));
+      atomicAdd(reinterpret_cast<unsigned long long*>(status) + 6, static_cast<unsigned long long>(clock64() - st_begin));
+      atomicAdd(reinterpret_cast<unsigned long long*>(status) + 7, static_cast<unsigned long long>(n_kt));
+#endif
       if (PAIR) umma_commit_pair(acc_bar);
       else umma_commit(acc_bar);
     }

@@ -42,10 +42,7 @@ namespace {
 using namespace tc;
 
 constexpr int kTileK = 64;
-#ifndef SURGEON_PROD_WARPS
-#define SURGEON_PROD_WARPS 16
-#endif
-constexpr int kProdWarps = SURGEON_PROD_WARPS;
+constexpr int kProdWarps = 16;
 constexpr int kThreads = 64 + kProdWarps * 32;   // warp 0: MMA, warp 1: TMA, warps 2..17: producers
 constexpr int kMaxAStages = 8;
 constexpr int kMaxGStages = 4;
@@ -775,11 +772,7 @@ size_t swap_partial_bytes(const SwapParams& p) {
 cudaError_t launch_swap(const surgeon_compressed& act, const SwapParams& plan, const float* grad_out,
                         void* grad_bf16, float* partial, uint32_t* status, cudaStream_t stream) {
   SwapParams p = plan;
-#ifdef SURGEON_STAGE_MIN
-  const bool staged = true;
-#else
   const bool staged = act.dt == 0;
-#endif
   if (!size_swap_rings(&p, staged ? kProdWarps * kStageBytesPerWarp : 0)) return cudaErrorInvalidValue;
   p.n_words = (act.n + 31) / 32;
   p.n_keep_ptr = reinterpret_cast<const long long*>(reinterpret_cast<const char*>(act.header) +

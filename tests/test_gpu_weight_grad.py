@@ -148,6 +148,16 @@ def test_cta_pairs():
     assert out.returncode == 0 and "PAIRS_OK" in out.stdout, out.stdout[-2000:] + out.stderr[-2000:]
 
 
+def test_exchanged_roles_on_cta_pairs():
+    """The kernel with the operand roles exchanged on CTA pairs (off by default) in a child process."""
+    import os
+    import subprocess
+    import sys
+    worker = os.path.join(os.path.dirname(os.path.abspath(__file__)), "swap_worker.py")
+    out = subprocess.run([sys.executable, worker], capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0 and "SWAP_OK" in out.stdout, out.stdout[-2000:] + out.stderr[-2000:]
+
+
 def test_weight_grad_argument_errors():
     layer = W.conv("err", 2, 4, 8, 4, 3)
     a = W.activation(layer, 1).cuda()
