@@ -228,6 +228,203 @@ dw_grouped_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ 
   }
 }
 
+// ---- 3x3, padding 1, stride 1 or 2, output rows a multiple of 8 wide (ResNeXt's grouped layers) ----
+// Register tiles instead of one column per thread: a thread owns TO output channels x TC input
+// channels x 9 taps of accumulators and walks strips of 8 consecutive output positions.  Per strip
+// and (channel, kernel row) it loads the 10 (stride 2: 17) input values the three taps need as
+// aligned 16-byte vectors and reuses them for all TO channels and all 3 column taps, so a
+// shared-memory load feeds 13-26 FMAs instead of 2.  The band's input rows are rebuilt word by
+// word: a lane takes one 32-bit bitmap word, ranks its first kept element (block offset plus the
+// popcounts of the block's words before it) and scatters the word's kept values into the zeroed
+// tile, so the work is per kept element and there is one index division per word.  Sums stay in fp32 inside a thread (at most kTermsPerThread terms, the planner cuts the
+// images into chunks accordingly), the threads' tiles are added in double in a fixed order.
+struct Grouped3Params {
+  int B, C, H, W, O, OH, OW, G, Cg, Og;
+  int band, n_bands, in_rows, Wp;
+  int units, n_cb, S;          // (output block, channel block) units; channel blocks; strip splits
+  int chunks, imgs_per_chunk, nb;
+  int a_floats, g_floats;      // per image
+  int dt;
+  long long n_words;
+  unsigned partial_blk;
+};
+constexpr int kTermsPerThread = 4096;
+// Three CTAs share an SM: rebuilding a tile is two dependent global loads per element, so what
+// hides that latency is the other CTAs' work.  That leaves a CTA 85 registers per thread (tiles of
+// at most 4 channel pairs: 36 accumulators) and about 74 KB of shared memory.
+constexpr int kG3CtasPerSm = 3;
+constexpr int kG3Smem = 74 * 1024;
+
+template <int TO, int TC, int ST>
+__global__ void __launch_bounds__(kThreads, kG3CtasPerSm)
+dw_grouped3_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ values,
+                   const uint32_t* __restrict__ offsets, const float* __restrict__ grad,
+                   double* __restrict__ partial, Grouped3Params p) {
+  constexpr int ACC = TO * TC * 9;
+  constexpr int AW = ST == 1 ? 12 : 20;              // input values loaded per (channel, kernel row)
+  extern __shared__ __align__(16) float sm[];
+  float* As = sm;                                     // [nb][Cg][in_rows][Wp], column 0 = input column -1
+  float* Gs = sm + p.nb * p.a_floats;                 // [nb][Og][band * OW]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int grp = blockIdx.x, band = blockIdx.y, chunk = blockIdx.z;
+  const int y0 = band * p.band;
+  const int rows = min(p.band, p.OH - y0);
+  const int npos = rows * p.OW;
+  const int iy0 = y0 * ST - 1;                        // input row of As row 0
+  const int iy_lo = max(iy0, 0), iy_hi = min(iy0 + (rows - 1) * ST + 3, p.H);   // valid input rows [lo, hi)
+  const int n_valid = iy_hi - iy_lo;
+  const int b_begin = chunk * p.imgs_per_chunk;
+  const int b_end = min(b_begin + p.imgs_per_chunk, p.B);
+  const int gpitch = p.band * p.OW;
+  const int spr = p.OW >> 3;                          // strips per output row
+  const int n_strips = rows * spr;
+
+  float acc[ACC];
+#pragma unroll
+  for (int i = 0; i < ACC; ++i) acc[i] = 0.0f;
+
+  // this thread's unit and strip split
+  const int unit = tid / p.S, sidx = tid - unit * p.S;
+  const bool worker = unit < p.units;
+  const int ob = unit / p.n_cb, cb = unit - ob * p.n_cb;
+
+  // rebuilding: a lane takes one bitmap word of a channel plane's valid rows and scatters its kept
+  // values (the tiles are zeroed every round, so pruned elements cost nothing)
+  const int plane_len = n_valid * p.W;
+  const int wpp = (plane_len + 31) / 32 + 1;          // words a plane's range can touch
+  const uint32_t rcpW = p.W < 32 ? (65536u + p.W - 1) / p.W : 0u;   // exact c / W for c < 2048
+
+  for (int b0 = b_begin; b0 < b_end; b0 += p.nb) {
+    const int nb_here = min(p.nb, b_end - b0);
+    __syncthreads();                                  // the previous round's tiles are no longer read
+    for (int i = tid; i < (nb_here * p.a_floats) >> 2; i += kThreads)
+      reinterpret_cast<float4*>(As)[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    // ---- gradient planes of the group, rows of the band: 16-byte copies, a warp per plane ----
+    {
+      const int q4 = npos >> 2;                       // vectors per plane
+      for (int pl = warp; pl < nb_here * p.Og; pl += kThreads / 32) {
+        const int bi = pl / p.Og, o = pl - bi * p.Og;
+        const float4* src = reinterpret_cast<const float4*>(
+            grad + (static_cast<long long>(b0 + bi) * p.O + grp * p.Og + o) * (p.OH * p.OW) + y0 * p.OW);
+        float4* dst = reinterpret_cast<float4*>(Gs + bi * p.g_floats + o * gpitch);
+#pragma unroll 4
+        for (int v = lane; v < q4; v += 32) dst[v] = __ldg(src + v);
+      }
+    }
+    __syncthreads();                                  // the zeros are in place before values land on them
+    // ---- the band's input rows of the group's channels from the store ----
+    {
+      const int total = nb_here * p.Cg * wpp;
+      for (int item = tid; item < total; item += kThreads) {
+        const int plane = item / wpp, k = item - plane * wpp;
+        const int bi = plane / p.Cg, cl = plane - bi * p.Cg;
+        const long long e_lo = (static_cast<long long>(b0 + bi) * p.C + grp * p.Cg + cl) * (p.H * p.W) + iy_lo * p.W;
+        const long long e_hi = e_lo + plane_len;
+        const long long w = (e_lo >> 5) + k;          // this lane's word
+        const long long j0 = w << 5;
+        if (j0 >= e_hi) continue;
+        const uint32_t full = __ldg(bitmap + w);
+        const int lo = j0 < e_lo ? static_cast<int>(e_lo - j0) : 0;           // first bit inside the range
+        uint32_t bits = full & (0xFFFFFFFFu << lo);
+        if (e_hi - j0 < 32) bits &= (1u << static_cast<int>(e_hi - j0)) - 1u;
+        if (!bits) continue;
+        // place of the first kept value in the packed vector
+        const long long blk = w >> 2;
+        uint32_t kfirst = __ldg(offsets + blk) + __popc(full & ~(0xFFFFFFFFu << lo));
+        for (int q = 0; q < static_cast<int>(w & 3); ++q) kfirst += __popc(__ldg(bitmap + blk * 4 + q));
+        // row and column of bit `lo` inside the plane's valid rows
+        const int rel = static_cast<int>(j0 + lo - e_lo);
+        const int row0 = rel / p.W, col0 = rel - row0 * p.W;
+        float* tile = As + bi * p.a_floats + (cl * p.in_rows + (iy_lo - iy0)) * p.Wp + 1;
+        const int cnt = __popc(bits);
+        for (int i = 0; i < cnt; i += 4) {
+          float v[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            v[q] = 0.0f;
+            if (i + q < cnt) {
+              const long long kk = static_cast<long long>(kfirst) + i + q;
+              v[q] = p.dt == 0 ? __ldg(reinterpret_cast<const float*>(values) + kk)
+                               : __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(values) + kk)) << 16);
+            }
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            if (i + q < cnt) {
+              const int e = __ffs(bits) - 1;
+              bits &= bits - 1;
+              int c = col0 + (e - lo), r = row0;
+              if (p.W >= 32) { if (c >= p.W) { c -= p.W; ++r; } }
+              else { const int qd = static_cast<int>((static_cast<uint32_t>(c) * rcpW) >> 16); c -= qd * p.W; r += qd; }
+              tile[r * p.Wp + c] = v[q];
+            }
+          }
+        }
+      }
+    }
+    __syncthreads();
+    // ---- products ----
+    if (worker) {
+      const int total = nb_here * n_strips;
+      for (int fs = sidx; fs < total; fs += p.S) {
+        const int bi = fs / n_strips, st = fs - bi * n_strips;
+        const int yl = st / spr, x0 = (st - yl * spr) << 3;
+        const float* gp = Gs + bi * p.g_floats + (ob * TO) * gpitch + yl * p.OW + x0;
+        float g[TO][8];
+#pragma unroll
+        for (int o = 0; o < TO; ++o) {
+          const float4 lo = *reinterpret_cast<const float4*>(gp + o * gpitch);
+          const float4 hi = *reinterpret_cast<const float4*>(gp + o * gpitch + 4);
+          g[o][0] = lo.x; g[o][1] = lo.y; g[o][2] = lo.z; g[o][3] = lo.w;
+          g[o][4] = hi.x; g[o][5] = hi.y; g[o][6] = hi.z; g[o][7] = hi.w;
+        }
+        const float* abase = As + bi * p.a_floats + ((cb * TC) * p.in_rows + ST * yl) * p.Wp + ST * x0;
+#pragma unroll
+        for (int c = 0; c < TC; ++c) {
+#pragma unroll
+          for (int r = 0; r < 3; ++r) {
+            const float* ap = abase + (c * p.in_rows + r) * p.Wp;
+            float a[AW];
+#pragma unroll
+            for (int v = 0; v < AW / 4; ++v) {
+              const float4 t = *reinterpret_cast<const float4*>(ap + 4 * v);
+              a[4 * v] = t.x; a[4 * v + 1] = t.y; a[4 * v + 2] = t.z; a[4 * v + 3] = t.w;
+            }
+#pragma unroll
+            for (int o = 0; o < TO; ++o)
+#pragma unroll
+              for (int s = 0; s < 3; ++s) {
+                float f = acc[(o * TC + c) * 9 + r * 3 + s];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) f = fmaf(g[o][i], a[ST * i + s], f);
+                acc[(o * TC + c) * 9 + r * 3 + s] = f;
+              }
+          }
+        }
+      }
+    }
+  }
+  // ---- add the strip splits of every unit in a fixed order, write this CTA's partial tile ----
+  __syncthreads();
+  float* red = sm;                                    // [thread][ACC]
+  if (worker) {
+#pragma unroll
+    for (int i = 0; i < ACC; ++i) red[tid * ACC + i] = acc[i];
+  }
+  __syncthreads();
+  const int ncol = p.Cg * 9;
+  double* out = partial + static_cast<long long>(chunk * p.n_bands + band) * p.O * ncol;
+  for (int i = tid; i < p.units * ACC; i += kThreads) {
+    const int u = i / ACC, a = i - u * ACC;
+    double s = 0.0;
+    for (int sp = 0; sp < p.S; ++sp) s += static_cast<double>(red[(u * p.S + sp) * ACC + a]);
+    const int uo = u / p.n_cb, uc = u - uo * p.n_cb;
+    const int o = a / (TC * 9), rem = a - o * (TC * 9);
+    const int c = rem / 9, rs = rem - c * 9;
+    out[static_cast<long long>(grp * p.Og + uo * TO + o) * ncol + (uc * TC + c) * 9 + rs] = s;
+  }
+}
+
 // dw[i] (= [o][c'][r][s] flattened, the layout of the partial tiles) = sum of the partial tiles in
 // index order, in double.
 __global__ void __launch_bounds__(256)
@@ -286,6 +483,65 @@ bool plan_grouped(const surgeon_layer_desc& d, GroupedParams* out) {
   return true;
 }
 
+// The register-tiled kernel's launch: 3x3, padding 1, stride 1 or 2, even maps under stride 2, output
+// rows a multiple of 8 wide.  TO / TC = the largest of 4, 2, 1 that divide the group's output /
+// input channels with TO * TC <= 4.
+struct Grouped3Tile { int to, tc; };
+bool plan_grouped3(const surgeon_layer_desc& d, Grouped3Params* out, Grouped3Tile* tile) {
+  if (d.kind != 1 || d.groups <= 1 || d.c_in % d.groups || d.c_out % d.groups) return false;
+  if (d.kh != 3 || d.kw != 3 || d.pad != 1 || (d.stride != 1 && d.stride != 2)) return false;
+  if (d.stride == 2 && ((d.h | d.w) & 1)) return false;
+  Grouped3Params p{};
+  p.B = d.batch; p.C = d.c_in; p.H = d.h; p.W = d.w; p.O = d.c_out;
+  p.OH = (d.h + 2 - 3) / d.stride + 1;
+  p.OW = (d.w + 2 - 3) / d.stride + 1;
+  if (p.OW % 8 || p.OW < 8) return false;
+  p.G = d.groups; p.Cg = d.c_in / d.groups; p.Og = d.c_out / d.groups;
+  int to = p.Og % 4 == 0 ? 4 : (p.Og % 2 == 0 ? 2 : 1);
+  int tc = p.Cg % 4 == 0 ? 4 : (p.Cg % 2 == 0 ? 2 : 1);
+  while (to * tc > 4) { if (tc >= to) tc >>= 1; else to >>= 1; }   // 2x2 where both allow it
+  p.n_cb = p.Cg / tc;
+  p.units = (p.Og / to) * p.n_cb;
+  if (p.units > kThreads) return false;
+  p.S = kThreads / p.units;
+  p.Wp = p.W + 4;                                   // column 0 = input column -1; 16-byte aligned rows
+  const long long red_bytes = static_cast<long long>(kThreads) * to * tc * 9 * 4;
+  int band = p.OH;
+  for (;; --band) {
+    if (band < 1) return false;
+    const long long in_rows = static_cast<long long>(band - 1) * d.stride + 3;
+    const long long a = static_cast<long long>(p.Cg) * in_rows * p.Wp;
+    const long long g = static_cast<long long>(p.Og) * band * p.OW;
+    if ((a + g) * 4 <= kG3Smem) { p.in_rows = static_cast<int>(in_rows); p.a_floats = static_cast<int>(a); p.g_floats = static_cast<int>(g); break; }
+  }
+  if (red_bytes > kG3Smem) return false;
+  p.band = band;
+  p.n_bands = (p.OH + band - 1) / band;
+  p.nb = static_cast<int>(kG3Smem / (static_cast<long long>(p.a_floats + p.g_floats) * 4));
+  if (p.nb > 8) p.nb = 8;
+  // image chunks: one resident wave of CTAs, and no thread adds more than kTermsPerThread terms in fp32
+  const long long per_chunk0 = static_cast<long long>(p.G) * p.n_bands;
+  long long chunks = (static_cast<long long>(kG3CtasPerSm) * sm_count()) / per_chunk0;
+  const long long strips = static_cast<long long>(band) * (p.OW / 8);
+  const long long max_imgs = (static_cast<long long>(kTermsPerThread) / 8) * p.S / strips;   // strips per thread = imgs * strips / S
+  if (max_imgs < 1) return false;
+  if (chunks < (p.B + max_imgs - 1) / max_imgs) chunks = (p.B + max_imgs - 1) / max_imgs;
+  if (chunks > p.B) chunks = p.B;
+  if (chunks < 1) chunks = 1;
+  if (chunks > 65535 || p.n_bands > 65535) return false;
+  p.imgs_per_chunk = static_cast<int>((p.B + chunks - 1) / chunks);
+  p.chunks = (p.B + p.imgs_per_chunk - 1) / p.imgs_per_chunk;
+  if (p.nb > p.imgs_per_chunk) p.nb = p.imgs_per_chunk;
+  *out = p;
+  tile->to = to; tile->tc = tc;
+  return true;
+}
+size_t grouped3_smem(const Grouped3Params& p, const Grouped3Tile& t) {
+  const size_t tiles = static_cast<size_t>(p.nb) * (p.a_floats + p.g_floats) * 4;
+  const size_t red = static_cast<size_t>(kThreads) * t.to * t.tc * 9 * 4;
+  return (tiles > red ? tiles : red) + 16;
+}
+
 size_t grouped_smem(const GroupedParams& p) {
   const size_t tiles = static_cast<size_t>(p.nb) * (p.a_floats + p.g_floats) * 4;
   const size_t red = static_cast<size_t>(p.S) * p.n_units * kRO * 8;
@@ -295,6 +551,10 @@ size_t grouped_smem(const GroupedParams& p) {
 }  // namespace
 
 size_t weight_grad_grouped_workspace(const surgeon_layer_desc& d) {
+  Grouped3Params p3;
+  Grouped3Tile t3;
+  if (plan_grouped3(d, &p3, &t3))
+    return static_cast<size_t>(p3.chunks) * p3.n_bands * p3.O * p3.Cg * 9 * sizeof(double);
   GroupedParams p;
   if (!plan_grouped(d, &p)) return 0;
   return static_cast<size_t>(p.chunks) * p.n_bands * p.O * p.ncol * sizeof(double);
@@ -303,9 +563,44 @@ size_t weight_grad_grouped_workspace(const surgeon_layer_desc& d) {
 cudaError_t launch_weight_grad_grouped(const surgeon_compressed& act, const surgeon_layer_desc& d,
                                        const float* grad_out, float* dw, int accumulate,
                                        void* workspace, cudaStream_t stream) {
+  double* partial = static_cast<double*>(workspace);
+  Grouped3Params p3;
+  Grouped3Tile t3;
+  if (plan_grouped3(d, &p3, &t3)) {
+    p3.dt = act.dt;
+    p3.n_words = (act.n + 31) / 32;
+    p3.partial_blk = (act.n % SURGEON_BLOCK) ? static_cast<unsigned>(act.n / SURGEON_BLOCK) : 0xFFFFFFFFu;
+    const size_t smem = grouped3_smem(p3, t3);
+    const dim3 grid(p3.G, p3.n_bands, p3.chunks);
+    cudaError_t e = cudaSuccess;
+    auto launch = [&](auto kernel) {
+      e = allow_dynamic_smem(reinterpret_cast<const void*>(kernel), static_cast<int>(smem));
+      if (e == cudaSuccess)
+        kernel<<<grid, kThreads, smem, stream>>>(act.bitmap, act.values, act.block_offsets, grad_out, partial, p3);
+    };
+    auto by_stride = [&](auto to, auto tc) {
+      constexpr int TO = decltype(to)::value, TC = decltype(tc)::value;
+      if (d.stride == 1) launch(dw_grouped3_kernel<TO, TC, 1>);
+      else launch(dw_grouped3_kernel<TO, TC, 2>);
+    };
+    using I1 = std::integral_constant<int, 1>;
+    using I2 = std::integral_constant<int, 2>;
+    using I4 = std::integral_constant<int, 4>;
+    if (t3.to == 4) by_stride(I4{}, I1{});
+    else if (t3.to == 2 && t3.tc == 2) by_stride(I2{}, I2{});
+    else if (t3.to == 2) by_stride(I2{}, I1{});
+    else if (t3.tc == 4) by_stride(I1{}, I4{});
+    else if (t3.tc == 2) by_stride(I1{}, I2{});
+    else by_stride(I1{}, I1{});
+    if (e != cudaSuccess) return e;
+    const long long mn = static_cast<long long>(p3.O) * p3.Cg * 9;
+    grouped_reduce_kernel<<<static_cast<unsigned>((mn + 255) / 256), 256, 0, stream>>>(partial, mn, p3.chunks * p3.n_bands,
+                                                                                   dw, accumulate);
+    note_launches(2);
+    return cudaGetLastError();
+  }
   GroupedParams p;
   if (!plan_grouped(d, &p)) return cudaErrorNotSupported;
-  double* partial = static_cast<double*>(workspace);
   p.n_words = (act.n + 31) / 32;
   p.partial_blk = (act.n % SURGEON_BLOCK) ? static_cast<unsigned>(act.n / SURGEON_BLOCK) : 0xFFFFFFFFu;
   const size_t smem = grouped_smem(p);

@@ -24,6 +24,18 @@ SHAPES = [
     W.conv("g3_1x1", 4, 18, 7, 12, 1, 1, 0, groups=3),
     W.conv("depthwise5x5_w40", 1, 6, 40, 6, 5, 1, 2, groups=6),
     W.conv("tall_map_bands", 1, 4, 200, 4, 3, groups=2),            # a map too tall for one band of shared memory
+    # the register-tiled 3x3 kernel (output rows a multiple of 8 wide): every tile shape, both strides,
+    # batches that do not divide into rounds, rows of 8, 16, 32, 40 and 64
+    W.conv("t22_w32", 5, 16, 32, 16, 3, groups=4),                  # 4 -> 4 per group: 2 x 2 tiles
+    W.conv("t41_w16", 3, 6, 16, 24, 3, groups=6),                   # 1 -> 4 per group
+    W.conv("t14_w8", 7, 16, 8, 4, 3, groups=4),                     # 4 -> 1 per group
+    W.conv("t21_t12_w40", 2, 6, 40, 6, 3, groups=3),                # 2 -> 2: 2 x 2; rows wider than a warp
+    W.conv("t12_w24", 2, 4, 24, 6, 3, groups=2),                    # 2 -> 3 per group: 1 x 2 tiles
+    W.conv("t21_w8_s2", 3, 9, 16, 6, 3, 2, groups=3),               # 3 -> 2 per group, stride 2: 2 x 1 tiles
+    W.conv("depthwise_w64_s2", 2, 5, 128, 5, 3, 2, groups=5),       # 1 x 1 tiles, two column chunks per row
+    W.conv("depthwise_w16", 9, 12, 16, 12, 3, groups=12),
+    W.conv("t22_s2_w16", 3, 32, 32, 32, 3, 2, groups=4),            # 8 -> 8 per group, stride 2
+    replace(W.conv("t22_tall_bands", 1, 8, 64, 8, 3, groups=2), h=240),   # several bands of output rows
 ]
 
 
