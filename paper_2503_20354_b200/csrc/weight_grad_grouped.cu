@@ -251,8 +251,12 @@ constexpr int kTermsPerThread = 4096;
 // n / d by one multiplication: rcp = floor((2^32 - 1) / d) + 1, exact while n * d < 2^32 (d = 1: rcp
 // wraps to 0 and the quotient is n itself).
 __host__ __device__ __forceinline__ uint32_t div_magic(int d) { return 0xFFFFFFFFu / static_cast<uint32_t>(d) + 1u; }
-__device__ __forceinline__ void prefetch_l2(const void* p) {
-  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
+               "l"(gsrc));
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
 }
 __device__ __forceinline__ int fast_div(int n, uint32_t rcp) {
   return rcp ? static_cast<int>(__umulhi(static_cast<uint32_t>(n), rcp)) : n;
@@ -304,67 +308,15 @@ dw_grouped3_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__
   const int wpp = (plane_len + 31) / 32 + 1;          // words a plane's range can touch
   const uint32_t rcp_wpp_k = div_magic(wpp);
 
-  // Rebuilding a tile is a chain of dependent loads (bitmap word -> block offset -> values), each a
-  // trip to DRAM when cold.  The rounds therefore run a prefetch pipeline into L2: the bitmap and
-  // offset lines of a round are requested two rounds ahead, and one round ahead a thread per plane
-  // reads the (by then L2-resident) offsets at the ends of the plane's range and requests the lines
-  // of packed values between them; the gradient planes of the next round are requested as well.
-  const int esize = p.dt == 0 ? 4 : 2;
   auto plane_range = [&](int b, int cl, long long& e_lo, long long& e_hi) {
     e_lo = (static_cast<long long>(b) * p.C + grp * p.Cg + cl) * (p.H * p.W) + iy_lo * p.W;
     e_hi = e_lo + plane_len;
   };
-  auto prefetch_meta = [&](int bfirst) {              // bitmap words and block offsets of a round's planes
-    const int nbr = min(p.nb, b_end - bfirst);
-    for (int t = tid; t < nbr * p.Cg; t += kThreads) {
-      const int bi = fast_div(t, p.rcp_cg), cl = t - bi * p.Cg;
-      long long e_lo, e_hi;
-      plane_range(bfirst + bi, cl, e_lo, e_hi);
-      const char* w0 = reinterpret_cast<const char*>(bitmap + (e_lo >> 5));
-      const char* w1 = reinterpret_cast<const char*>(bitmap + ((e_hi - 1) >> 5));
-      for (const char* a = w0; a <= w1; a += 128) prefetch_l2(a);
-      prefetch_l2(w1);
-      const char* o0 = reinterpret_cast<const char*>(offsets + (e_lo >> kBlockShift));
-      const char* o1 = reinterpret_cast<const char*>(offsets + ((e_hi - 1) >> kBlockShift) + 1);
-      for (const char* a = o0; a <= o1; a += 128) prefetch_l2(a);
-      prefetch_l2(o1);
-    }
-  };
-  auto prefetch_data = [&](int bfirst) {              // packed values and gradient planes of a round
-    const int nbr = min(p.nb, b_end - bfirst);
-    const int lines_per_plane = (npos * 4 + 127) >> 7;
-    for (int t = tid; t < nbr * p.Og * lines_per_plane; t += kThreads) {
-      const int pl = t / lines_per_plane, ln = t - pl * lines_per_plane;
-      const int bi = pl / p.Og, o = pl - bi * p.Og;
-      prefetch_l2(reinterpret_cast<const char*>(
-                      grad + (static_cast<long long>(bfirst + bi) * p.O + grp * p.Og + o) * (p.OH * p.OW) + y0 * p.OW) +
-                  128 * ln);
-    }
-    for (int t = tid; t < nbr * p.Cg; t += kThreads) {
-      const int bi = fast_div(t, p.rcp_cg), cl = t - bi * p.Cg;
-      long long e_lo, e_hi;
-      plane_range(bfirst + bi, cl, e_lo, e_hi);
-      const uint32_t k0 = __ldg(offsets + (e_lo >> kBlockShift));
-      const uint32_t k1 = __ldg(offsets + ((e_hi - 1) >> kBlockShift) + 1);     // the table ends with a sentinel entry
-      const char* v = reinterpret_cast<const char*>(values);
-      for (long long a = static_cast<long long>(k0) * esize; a < static_cast<long long>(k1) * esize; a += 128) prefetch_l2(v + a);
-    }
-  };
-  if (n_valid > 0) {
-    prefetch_meta(b_begin);
-    if (b_begin + p.nb < b_end) prefetch_meta(b_begin + p.nb);
-  }
-
   for (int b0 = b_begin; b0 < b_end; b0 += p.nb) {
     const int nb_here = min(p.nb, b_end - b0);
     __syncthreads();                                  // the previous round's tiles are no longer read
-    if (n_valid > 0) {
-      if (b0 + 2 * p.nb < b_end) prefetch_meta(b0 + 2 * p.nb);
-      if (b0 + p.nb < b_end) prefetch_data(b0 + p.nb);
-    }
-    for (int i = tid; i < (nb_here * p.a_floats) >> 2; i += kThreads)
-      reinterpret_cast<float4*>(As)[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-    // ---- gradient planes of the group, rows of the band: 16-byte copies, a warp per plane ----
+    // ---- gradient planes of the group, rows of the band: asynchronous 16-byte copies, a warp per
+    // plane; all of a thread's copies are in flight together and are waited for once ----
     {
       const int q4 = npos >> 2;                       // vectors per plane
       for (int pl = warp; pl < nb_here * p.Og; pl += kThreads / 32) {
@@ -372,64 +324,87 @@ dw_grouped3_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__
         const float4* src = reinterpret_cast<const float4*>(
             grad + (static_cast<long long>(b0 + bi) * p.O + grp * p.Og + o) * (p.OH * p.OW) + y0 * p.OW);
         float4* dst = reinterpret_cast<float4*>(Gs + bi * p.g_floats + o * gpitch);
-#pragma unroll 4
-        for (int v = lane; v < q4; v += 32) dst[v] = __ldg(src + v);
+        for (int v = lane; v < q4; v += 32) cp_async16(dst + v, src + v);
       }
     }
-    __syncthreads();                                  // the zeros are in place before values land on them
+    for (int i = tid; i < (nb_here * p.a_floats) >> 2; i += kThreads)
+      reinterpret_cast<float4*>(As)[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
     // ---- the band's input rows of the group's channels from the store ----
-    // A lane takes one bitmap word: it ranks the word's first kept element (block offset plus the
-    // popcounts of the block's words before it) and scatters the word's kept values into the zeroed
-    // tile, four loads in flight at a time.  The work is per kept element; a warp that walks 32
-    // words with one lane per bit (coalesced loads, no dependent rounds) measured 1.6x slower,
-    // because it spends instructions on every element, kept or not.
+    // A lane takes one bitmap word at a time (two per pass): it fetches the word's block (bitmap
+    // words and offset, independent loads), ranks the word's first kept element and scatters the
+    // word's kept values into the zeroed tile, eight loads in flight at a time.  The metadata of the
+    // first pass is requested before the barrier that ends the zeroing, so its latency and that of
+    // the gradient copies overlap.  The work is per kept element; a warp that walks 32 words with
+    // one lane per bit (coalesced loads, no dependent rounds) measured 1.6x slower, because it
+    // spends instructions on every element, kept or not.
     {
+      struct WordRef { uint32_t bits, kfirst; int lo, col0, pos; };   // pos: tile index of bit `lo`
       const int total = nb_here * p.Cg * wpp;
-      for (int wi = tid; wi < total; wi += kThreads) {
+      auto fetch = [&](int wi) {
+        WordRef r{0u, 0u, 0, 0, 0};
+        if (wi >= total) return r;
         const int plane = fast_div(wi, rcp_wpp_k), k = wi - plane * wpp;
         const int bi = fast_div(plane, p.rcp_cg), cl = plane - bi * p.Cg;
         long long e_lo, e_hi;
         plane_range(b0 + bi, cl, e_lo, e_hi);
         const long long w = (e_lo >> 5) + k;          // this lane's word
         const long long j0 = w << 5;
-        if (j0 >= e_hi) continue;
-        const uint32_t full = __ldg(bitmap + w);
+        if (j0 >= e_hi) return r;
+        const ActRef m = act_meta(bitmap, offsets, j0, p.n_words, p.partial_blk);
+        const uint32_t wq = static_cast<uint32_t>(w) & 3u;
+        const uint32_t full = wq == 0 ? m.words.x : (wq == 1 ? m.words.y : (wq == 2 ? m.words.z : m.words.w));
         int lo = j0 < e_lo ? static_cast<int>(e_lo - j0) : 0;                 // first bit inside the range
         uint32_t bits = full & (0xFFFFFFFFu << lo);
         if (e_hi - j0 < 32) bits &= (1u << static_cast<int>(e_hi - j0)) - 1u;
-        if (!bits) continue;
+        if (!bits) return r;
         lo = __ffs(bits) - 1;                         // the word's first kept bit inside the range
-        // place of that bit's value in the packed vector
-        const long long blk = w >> 2;
-        uint32_t kfirst = __ldg(offsets + blk) + __popc(full & ~(0xFFFFFFFFu << lo));
-        for (int q = 0; q < static_cast<int>(w & 3); ++q) kfirst += __popc(__ldg(bitmap + blk * 4 + q));
-        // row and column of bit `lo` inside the plane's valid rows
+        uint32_t kfirst = m.base + __popc(full & ~(0xFFFFFFFFu << lo));
+        kfirst += wq > 0 ? __popc(m.words.x) : 0u;
+        kfirst += wq > 1 ? __popc(m.words.y) : 0u;
+        kfirst += wq > 2 ? __popc(m.words.z) : 0u;
         const int rel = static_cast<int>(j0 + lo - e_lo);
-        const int row0 = fast_div(rel, p.rcp_w), col0 = rel - row0 * p.W;
-        float* tile = As + bi * p.a_floats + (cl * p.in_rows + (iy_lo - iy0)) * p.Wp + 1;
+        const int row0 = fast_div(rel, p.rcp_w);
+        r.bits = bits; r.kfirst = kfirst; r.lo = lo; r.col0 = rel - row0 * p.W;
+        r.pos = bi * p.a_floats + (cl * p.in_rows + (iy_lo - iy0) + row0) * p.Wp + 1 + r.col0;
+        return r;
+      };
+      auto emit = [&](const WordRef& r) {
+        uint32_t bits = r.bits;
         const int cnt = __popc(bits);
-        for (int i = 0; i < cnt; i += 4) {
-          float v[4];
+        for (int i = 0; i < cnt; i += 8) {
+          float v[8];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
+          for (int q = 0; q < 8; ++q) {
             v[q] = 0.0f;
             if (i + q < cnt) {
-              const long long kk = static_cast<long long>(kfirst) + i + q;
+              const long long kk = static_cast<long long>(r.kfirst) + i + q;
               v[q] = p.dt == 0 ? __ldg(reinterpret_cast<const float*>(values) + kk)
                                : __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(values) + kk)) << 16);
             }
           }
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
+          for (int q = 0; q < 8; ++q) {
             if (i + q < cnt) {
               const int e = __ffs(bits) - 1;
               bits &= bits - 1;
-              const int c = col0 + (e - lo);          // < W + 32
-              const int qd = fast_div(c, p.rcp_w);
-              tile[(row0 + qd) * p.Wp + c - qd * p.W] = v[q];
+              // the tile's rows are 4 places longer than the input's: every wrap past the end of an
+              // input row skips those
+              const int d = e - r.lo;
+              As[r.pos + d + 4 * fast_div(r.col0 + d, p.rcp_w)] = v[q];
             }
           }
         }
+      };
+      bool first = true;
+      for (int base = 0; base < total || first; base += 2 * kThreads) {
+        const WordRef r0 = fetch(base + tid), r1 = fetch(base + kThreads + tid);
+        if (first) {
+          cp_async_wait_all();
+          __syncthreads();                            // zeros in place, gradient planes landed
+          first = false;
+        }
+        emit(r0);
+        emit(r1);
       }
     }
     __syncthreads();
