@@ -244,7 +244,7 @@ struct Grouped3Params {
   int a_floats, g_floats;      // per image
   int dt;
   uint32_t rcp_cg, rcp_spr, rcp_w;    // 2^32 / d rounded up: __umulhi(n, rcp) = n / d while n * d < 2^32
-  long long n_words;
+  long long n_words, n, n_blocks;
   unsigned partial_blk;
 };
 constexpr int kTermsPerThread = 4096;
@@ -297,6 +297,9 @@ dw_grouped3_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__
 #pragma unroll
   for (int i = 0; i < ACC; ++i) acc[i] = 0.0f;
 
+  // more than 55 % of the tensor kept (the last block offset is the kept count): the rebuild walks
+  // the bitmap words with a lane per bit instead of a lane per word
+  const bool dense = static_cast<double>(__ldg(offsets + p.n_blocks)) > 0.55 * static_cast<double>(p.n);
   // this thread's unit and strip split
   const int unit = tid / p.S, sidx = tid - unit * p.S;
   const bool worker = unit < p.units;
@@ -334,9 +337,10 @@ dw_grouped3_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__
     // words and offset, independent loads), ranks the word's first kept element and scatters the
     // word's kept values into the zeroed tile, eight loads in flight at a time.  The metadata of the
     // first pass is requested before the barrier that ends the zeroing, so its latency and that of
-    // the gradient copies overlap.  The work is per kept element; a warp that walks 32 words with
-    // one lane per bit (coalesced loads, no dependent rounds) measured 1.6x slower, because it
-    // spends instructions on every element, kept or not.
+    // the gradient copies overlap.  The work is per kept element, which is what wins on sparse
+    // stores (ResNeXt stage 1 at the rule's ratios: 108 us against 158 us for the lane-per-bit walk
+    // below); on mostly kept stores it loses (a lane's loads each touch their own cache line: 149
+    // against 128 us on a stage-2 layer), hence the two paths.
     {
       struct WordRef { uint32_t bits, kfirst; int lo, col0, pos; };   // pos: tile index of bit `lo`
       const int total = nb_here * p.Cg * wpp;
@@ -396,15 +400,54 @@ dw_grouped3_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__
         }
       };
       bool first = true;
-      for (int base = 0; base < total || first; base += 2 * kThreads) {
-        const WordRef r0 = fetch(base + tid), r1 = fetch(base + kThreads + tid);
-        if (first) {
-          cp_async_wait_all();
-          __syncthreads();                            // zeros in place, gradient planes landed
-          first = false;
+      if (!dense) {
+        for (int base = 0; base < total || first; base += 2 * kThreads) {
+          const WordRef r0 = fetch(base + tid), r1 = fetch(base + kThreads + tid);
+          if (first) {
+            cp_async_wait_all();
+            __syncthreads();                          // zeros in place, gradient planes landed
+            first = false;
+          }
+          emit(r0);
+          emit(r1);
         }
-        emit(r0);
-        emit(r1);
+      } else {
+        // Mostly kept words: a lane's 20-32 loads would each touch their own cache line.  Here lane j
+        // fetches the metadata of word base + j and the warp then walks those 32 words with lane l
+        // on bit l: one coalesced load per word, the words' loads independent of one another.
+        const uint32_t lt = (1u << lane) - 1u;
+        for (int base = warp * 32; base < total || first; base += kThreads) {
+          const WordRef r = fetch(base + lane);
+          if (first) {
+            cp_async_wait_all();
+            __syncthreads();
+            first = false;
+          }
+          for (int i0 = 0; i0 < 32; i0 += 8) {        // eight words' loads in flight before the first store
+            float v[8];
+            int dst[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const uint32_t b = __shfl_sync(0xFFFFFFFFu, r.bits, i0 + q);
+              const uint32_t k0 = __shfl_sync(0xFFFFFFFFu, r.kfirst, i0 + q);
+              const int lo = __shfl_sync(0xFFFFFFFFu, r.lo, i0 + q);
+              const int c0 = __shfl_sync(0xFFFFFFFFu, r.col0, i0 + q);
+              const int ps = __shfl_sync(0xFFFFFFFFu, r.pos, i0 + q);
+              dst[q] = -1;
+              v[q] = 0.0f;
+              if ((b >> lane) & 1u) {
+                const long long kk = static_cast<long long>(k0) + __popc(b & lt);   // b starts at bit `lo`, whose rank is k0
+                v[q] = p.dt == 0 ? __ldg(reinterpret_cast<const float*>(values) + kk)
+                                 : __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(values) + kk)) << 16);
+                const int d = static_cast<int>(lane) - lo;
+                dst[q] = ps + d + 4 * fast_div(c0 + d, p.rcp_w);
+              }
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              if (dst[q] >= 0) As[dst[q]] = v[q];
+          }
+        }
       }
     }
     __syncthreads();
@@ -617,6 +660,8 @@ cudaError_t launch_weight_grad_grouped(const surgeon_compressed& act, const surg
   if (plan_grouped3(d, &p3, &t3)) {
     p3.dt = act.dt;
     p3.n_words = (act.n + 31) / 32;
+    p3.n = act.n;
+    p3.n_blocks = (act.n + SURGEON_BLOCK - 1) / SURGEON_BLOCK;
     p3.partial_blk = (act.n % SURGEON_BLOCK) ? static_cast<unsigned>(act.n / SURGEON_BLOCK) : 0xFFFFFFFFu;
     const size_t smem = grouped3_smem(p3, t3);
     const dim3 grid(p3.G, p3.n_bands, p3.chunks);
