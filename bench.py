@@ -265,7 +265,10 @@ class Stack:
         self.B, self.layers, self.path, self.device = B, layers, path, device
         self.gi = W.gradient_importance(len(layers), seed)
         self.lam = np.array([l.act_bytes for l in layers], dtype=np.float64)
-        self.fixed_ratios = W.uniform_ratios(len(layers), seed) if ratios == "uniform" else None
+        if isinstance(ratios, str):
+            self.fixed_ratios = W.uniform_ratios(len(layers), seed) if ratios == "uniform" else None
+        else:                       # given per layer (a profiling subset keeps the whole stack's ratios)
+            self.fixed_ratios = np.asarray(ratios, dtype=np.float64)
         # A residual block's shortcut convolution reads the same tensor as the block's first
         # convolution: that tensor is pruned once, at the smaller of the two layers' ratios (the
         # one that keeps more), and both weight gradients read the one store.
@@ -398,15 +401,28 @@ def run_stack(key, args, rank, world, device, peaks, path, keep_stack=False, sam
     during the timed region."""
     from paper_2503_20354_b200 import binding as B
     layers, desc_text = get_layers(key, args.batch)
-    if args.layers:      # profiling aid: keep only the named layers of the stack
-        keep = set(args.layers.split(","))
-        layers = [l for l in layers if l.name in keep]
-        desc_text += " (layers %s only)" % args.layers
-        if len(layers) < 2:
-            raise SystemExit("--layers must name at least two layers of the stack (the ratio rule needs two)")
     uniform = key == "resnet50_uniform"
+    recipe = "uniform" if uniform else "rule"
+    if args.layers:      # profiling aid: keep only the named layers of the stack, at the ratios they have in the whole stack
+        from paper_2503_20354_b200 import binding as B
+        from paper_2503_20354_b200 import workloads as W
+        keep = set(args.layers.split(","))
+        idx = [i for i, l in enumerate(layers) if l.name in keep]
+        if not idx:
+            raise SystemExit("--layers names no layer of the stack")
+        if uniform:
+            full = np.asarray(W.uniform_ratios(len(layers), args.seed + rank), dtype=np.float64)
+        else:
+            full = np.asarray(B.surgeon_layer_ratios(W.gradient_importance(len(layers), args.seed + rank),
+                                                     np.array([l.act_bytes for l in layers], dtype=np.float64),
+                                                     allow_degenerate=True), dtype=np.float64)
+        for j, i in W.shared_inputs(layers).items():
+            full[i] = full[j] = min(full[i], full[j])
+        recipe = full[idx]
+        layers = [layers[i] for i in idx]
+        desc_text += " (layers %s only)" % args.layers
     stack = Stack(layers, path, args.seed + rank, device, n_streams=args.streams, sigma=SIGMA[key],
-                  ratios="uniform" if uniform else "rule")
+                  ratios=recipe)
     torch.cuda.synchronize()
     for _ in range(args.warmup):
         stack.step()
@@ -474,8 +490,8 @@ def run_stack(key, args, rank, world, device, peaks, path, keep_stack=False, sam
         us = stack.per_layer_dw_us()
         res["weight_grad"]["per_layer"] = {
             "note": "each layer's call alone on one stream; roofline_us = max(flops / tensor peak, least bytes / HBM peak)",
-            "name": [l.name for l in layers], "us": [round(u, 1) for u in us],
-            "roofline_us": [round(r, 1) for r in roof_us],
+            "name": [l.name for l in layers], "ratio": [round(float(r), 3) for r in stack.ratios],
+            "us": [round(u, 1) for u in us], "roofline_us": [round(r, 1) for r in roof_us],
             "sum_us": round(sum(us), 1), "sum_roofline_us": round(sum(roof_us), 1),
             "frac": round(sum(roof_us) / sum(us), 4)}
     if sampler is not None:

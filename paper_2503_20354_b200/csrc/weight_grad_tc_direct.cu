@@ -467,8 +467,28 @@ dw_direct_kernel(const uint32_t* __restrict__ bitmap, const void* __restrict__ v
         // through the staging copy; for sparser ones the copy's fixed cost outweighs the
         // scattered loads it saves, and bf16 values (half as many cache lines per load) never
         // gain from it, so bf16 launches reserve no staging area.
-        const bool dense = DT == 0 && __reduce_add_sync(0xFFFFFFFFu, cnt) > 560u;
-        if (dense) {
+        // Every run of the warp fully kept and its values 16-byte aligned: the layer that Eq. 7 gives
+        // ratio 0 (there is one in every batch: the layer with the largest importance), or an
+        // unpruned tensor.  The run is then 64 (128) consecutive bytes of the packed vector.
+        const bool whole = __all_sync(0xFFFFFFFFu, bits == 0xFFFFFFFFu && (rank & static_cast<uint32_t>(V - 1)) == 0u);
+        const bool dense = !whole && DT == 0 && __reduce_add_sync(0xFFFFFFFFu, cnt) > 560u;
+        if (whole) {
+          if (DT == 0) {
+            const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(values) + rank);
+            float4 f[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) f[q] = __ldg(src + q);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              chunk[q].x = pack_bf16x2(f[2 * q].x, f[2 * q].y); chunk[q].y = pack_bf16x2(f[2 * q].z, f[2 * q].w);
+              chunk[q].z = pack_bf16x2(f[2 * q + 1].x, f[2 * q + 1].y); chunk[q].w = pack_bf16x2(f[2 * q + 1].z, f[2 * q + 1].w);
+            }
+          } else {
+            const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned short*>(values) + rank);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) chunk[q] = __ldg(src + q);
+          }
+        } else if (dense) {
         uint32_t seg_len = cnt + __shfl_xor_sync(0xFFFFFFFFu, cnt, 1);
         if (MODE == 0) seg_len += __shfl_xor_sync(0xFFFFFFFFu, seg_len, 2);
         const uint32_t seg_start = __shfl_sync(0xFFFFFFFFu, rank, lane & ~(LPR - 1));
