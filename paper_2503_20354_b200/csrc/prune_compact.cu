@@ -359,6 +359,7 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
   } else {
     // ---- consumers ----
     uint32_t w_above = 0, w_cand = 0;
+    uint32_t w_kmax = 0, w_kinv = 0;     // largest key inside the bracket seen by this lane, and largest ~key
     for (int it = 0; it < n_it; ++it) {
       const int s = it % kCsStages;
       const int chunk = (first + it * static_cast<int>(gridDim.x)) * kCsWarps + warp;
@@ -419,30 +420,65 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
         if (lane == 0) { cnt_gt[chunk] = a_tot; cand_cnt[chunk] = c_tot; }
         w_above += a_tot;
         w_cand += c_tot;
+        const bool ragged = grow >= n_rows_full;
+        const unsigned char* row = region + lane * 128;
+        auto key_at = [&](int e) -> uint32_t {        // key of element e of this lane's row
+          if (ragged) return static_cast<uint32_t>(x[grow * EPR + e]) & kMask;
+          const int byte = e * static_cast<int>(sizeof(E));
+          return static_cast<uint32_t>(*reinterpret_cast<const E*>(
+                     row + (((byte >> 4) ^ (lane & 7)) << 4) + (byte & 15))) & kMask;
+        };
         if (c_tot > static_cast<uint32_t>(kSlot)) {
           if (lane == 0) st->list_overflow = 1u;
+          // Too many keys inside the bracket for the slot: massive ties.  If they all are one and the
+          // same key - here and in every other chunk - that key is the threshold and the counts
+          // above are all the count kernel needs; the last CTA checks that through the extremes.
+          const int src = __ffs(__ballot_sync(kFull, cc != 0u)) - 1;
+          uint32_t k0 = 0;
+          if (static_cast<int>(lane) == src) {
+#pragma unroll
+            for (int w = WPL - 1; w >= 0; --w)
+              if (cw[w]) k0 = key_at(32 * w + __ffs(cw[w]) - 1);
+          }
+          k0 = __shfl_sync(kFull, k0, src);
+          uint32_t eq = 0;
+          if (DT == 0) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              eq += ((q[j].x & kMask) == k0 ? 1u : 0u) + ((q[j].y & kMask) == k0 ? 1u : 0u) +
+                    ((q[j].z & kMask) == k0 ? 1u : 0u) + ((q[j].w & kMask) == k0 ? 1u : 0u);
+            }
+          } else {
+            const uint32_t c_ge = ge_const(k0), c_gt = ge_const(k0 + 1u);   // k0 <= 0x7FFF
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint32_t c[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const uint32_t keys2 = c[i] & 0x7FFF7FFFu;
+                eq += __popc(((keys2 + c_ge) & ~(keys2 + c_gt)) & 0x80008000u);
+              }
+            }
+          }
+          // (a ragged row's fill is key 0, never a candidate)
+          const bool one_key = __reduce_add_sync(kFull, eq) == c_tot;
+          w_kmax = one_key ? max(w_kmax, k0) : 0xFFFFFFFFu;
+          w_kinv = one_key ? max(w_kinv, ~k0) : 0xFFFFFFFFu;
         } else if (c_tot) {
           // keys inside the bracket -> the chunk's slot (order does not matter)
           uint32_t pos = warp_excl_scan(cc);
           E* slot = slots + static_cast<long long>(chunk) * kSlot;
-          const bool ragged = grow >= n_rows_full;
-          const unsigned char* row = region + lane * 128;
 #pragma unroll
           for (int w = 0; w < WPL; ++w) {
             uint32_t m = cw[w];
             while (m) {
               const int e = 32 * w + __ffs(m) - 1;
               m &= m - 1;
-              uint32_t key;
-              if (ragged) {
-                key = static_cast<uint32_t>(x[grow * EPR + e]) & kMask;
-              } else {
-                const int byte = e * static_cast<int>(sizeof(E));
-                key = static_cast<uint32_t>(*reinterpret_cast<const E*>(
-                          row + (((byte >> 4) ^ (lane & 7)) << 4) + (byte & 15))) & kMask;
-              }
+              const uint32_t key = key_at(e);
               slot[pos++] = static_cast<E>(key);
               atomicAdd(&s_hist[(key - lo_key) >> shiftA], 1u);
+              w_kmax = max(w_kmax, key);
+              w_kinv = max(w_kinv, ~key);
             }
           }
         }
@@ -450,9 +486,13 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(empty_bar + 8 * s);
     }
+    w_kmax = __reduce_max_sync(kFull, w_kmax);
+    w_kinv = __reduce_max_sync(kFull, w_kinv);
     if (lane == 0) {
       if (w_above) atomicAdd(&s_tot[0], w_above);
       if (w_cand) atomicAdd(&s_tot[1], w_cand);
+      if (w_kmax) atomicMax(&st->cand_key_max, w_kmax);
+      if (w_kinv) atomicMax(&st->cand_keyinv_max, w_kinv);
     }
   }
   __syncthreads();
@@ -476,7 +516,13 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
   const long long r = static_cast<long long>(k) - above_total;     // rank among the rest
   const long long zeros = (lo_key == 1u) ? n - above_total - n_cand : 0;
   uint32_t mode, tau = 0, n_greater = 0;
-  if (overflow || r < 1) {
+  if (overflow && r >= 1 && r <= n_cand &&
+      __ldcg(&st->cand_key_max) == ~__ldcg(&st->cand_keyinv_max)) {
+    // every key inside the bracket is the same one: it is the threshold, all candidates are ties
+    mode = 4;
+    tau = __ldcg(&st->cand_key_max);
+    n_greater = above_total;
+  } else if (overflow || r < 1) {
     mode = 1;
   } else if (r <= n_cand) {
     // level A from the top: lane L owns bins [kBinsA - 16(L+1), kBinsA - 16L)
@@ -518,7 +564,7 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
     mode = 1;
   }
   if (lane == 0) {
-    if (mode == 2) {
+    if (mode == 2 || mode == 4) {
       // store variant without kept zeros: a threshold of key 0 keeps the non-zero elements only
       const bool nz = drop_zeros && tau == 0u;
       hdr->threshold_key = tau;
@@ -735,7 +781,8 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
     tau = hdr->threshold_key;
   }
   const bool nz = drop_zeros && tau == 0u;       // store variant without kept zeros (see classify_kernel)
-  if (mode != 2u && blockIdx.x == 0 && tid == 0) {
+  const bool hdr_final = mode == 2u || mode == 4u;   // the classify pass has written the header
+  if (!hdr_final && blockIdx.x == 0 && tid == 0) {
     hdr->threshold_key = tau;
     hdr->status = __ldcg(&st->error);
     hdr->n_keep = nz ? static_cast<long long>(n_greater) : static_cast<long long>(k);
@@ -743,7 +790,7 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
     hdr->tie_quota = nz ? 0 : static_cast<long long>(k) - n_greater;
   }
 
-  const long long quota = (mode == 2u) ? hdr->tie_quota : (nz ? 0 : static_cast<long long>(k) - n_greater);
+  const long long quota = hdr_final ? hdr->tie_quota : (nz ? 0 : static_cast<long long>(k) - n_greater);
 
   // ---- per-chunk values; CTA b owns the chunks [b*per, (b+1)*per) ----
   const int per = (tiles + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
@@ -755,10 +802,14 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
     for (int c = c_begin + tid; c < c_end; c += kSelThreads) {
       const uint32_t cc = __ldg(cand_cnt + c), cg = __ldg(cnt_gt + c);
       uint32_t g = cg, q = 0;
-      for_slot_keys<DT>(slots, c, cc, [&](uint32_t key) {
-        g += key > tau ? 1u : 0u;
-        q += key == tau ? 1u : 0u;
-      });
+      if (mode == 4u) {       // every key inside the bracket equals the threshold (the slots may have overflowed)
+        q = cc;
+      } else {
+        for_slot_keys<DT>(slots, c, cc, [&](uint32_t key) {
+          g += key > tau ? 1u : 0u;
+          q += key == tau ? 1u : 0u;
+        });
+      }
       if (tau == 0) {         // lo_key == 1: whatever is neither above nor inside the bracket is 0
         const long long left = n - static_cast<long long>(c) * kChunkElems;
         q += static_cast<uint32_t>(left < kChunkElems ? left : kChunkElems) - cg - cc;
@@ -869,13 +920,13 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
     if (tid == 0) {
       // the sentinel entry of the block offsets = the number of stored values
       offsets[(n + SURGEON_BLOCK - 1) >> kBlockShift] =
-          nz ? static_cast<uint32_t>((mode == 2u) ? hdr->n_greater : n_greater) : k;
+          nz ? static_cast<uint32_t>(hdr_final ? hdr->n_greater : n_greater) : k;
       unsigned long long total = 0;
       for (int b = 0; b <= static_cast<int>(blockIdx.x); ++b) total += __ldcg(partial + b);
       prefix[tiles] = total;
       const long long gt_all = static_cast<long long>(total >> 31);
       const long long eq_all = static_cast<long long>(total & 0x7FFFFFFFull);
-      const long long ng = (mode == 2u) ? hdr->n_greater : static_cast<long long>(n_greater);
+      const long long ng = hdr_final ? hdr->n_greater : static_cast<long long>(n_greater);
       const long long want = nz ? ng : static_cast<long long>(k);
       const long long kept = gt_all + (eq_all < quota ? eq_all : quota);
       // every mode and every barrier of this kernel is behind us: whatever gave up shows now

@@ -53,14 +53,16 @@ struct SelectState {
   uint32_t lo_key, hi_key;       // the same bracket as an inclusive key range (lo_key >= 1)
   uint32_t mode;                 // 0 = threshold among the candidates, level B pending (fp32);
                                  // 1 = bracket unusable, fall back to a radix select over x;
-                                 // 2 = threshold already final in the header
+                                 // 2 = threshold already final in the header;
+                                 // 4 = likewise, and every key inside the bracket equals it
   uint32_t list_overflow;
   uint32_t above_total, cand_total;   // keys above hi_key / inside [lo_key, hi_key]
   uint32_t shiftA;               // level A bin of a key = (key - lo_key) >> shiftA
   uint32_t binA, rankA, aboveA;  // level A: bin of the threshold, its rank inside, candidates above
   uint32_t fb_prefix, fb_rank, fb_above;   // fall-back select: key bits fixed so far, rank, count above
   uint32_t reserved0;            // (unused)
-  uint32_t pad[12];
+  uint32_t cand_key_max, cand_keyinv_max;   // extremes of the keys inside the bracket: max key, max ~key
+  uint32_t pad[10];
 };
 static_assert(sizeof(SelectState) == 128, "SelectState layout");
 constexpr size_t kWsStateBytes = 256;
