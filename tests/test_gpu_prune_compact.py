@@ -115,6 +115,30 @@ def test_all_equal_and_two_level(bf16):
 
 
 @pytest.mark.parametrize("bf16", [False, True])
+def test_massive_ties_on_the_sampled_path(bf16):
+    """Tensors large enough for the sampled select in which one magnitude holds far more elements
+    than a chunk's candidate slot: every key inside the bracket is then one key, which the select
+    takes as the threshold without a fall-back pass.  The tie quota ends in the middle of the
+    tensor, at its very start and at its very end; a second magnitude close by (the next key up)
+    makes the bracket hold two keys, which must take the fall-back and still agree."""
+    n = (1 << 22) + 77
+    g = torch.Generator().manual_seed(11)
+    u = torch.rand(n, generator=g)
+    sign = torch.where(torch.rand(n, generator=g) < 0.5, -1.0, 1.0)
+    x = torch.where(u < 0.6, 1.0, 2.0) * sign                 # 60 % at |1|, 40 % at |2|
+    for ratio in (0.3, 0.6, 0.7, 0.95, 1.0 - 1.0 / n, 1.0 / n):
+        assert_store_equals_oracle(_as(x, bf16), ratio)
+    x = torch.full((n,), -0.75)                                # every key equal
+    for ratio in (0.5, 0.001):
+        comp, ref = assert_store_equals_oracle(_as(x, bf16), ratio)
+        assert ref["c_gt"] == 0 and ref["q"] == ref["k"]
+    up = torch.tensor(1.0).view(torch.int32) + 1 if not bf16 else None
+    y = torch.where(u < 0.5, 1.0, 1.0078125 if bf16 else float(up.view(torch.float32)))   # two adjacent keys
+    for ratio in (0.25, 0.5, 0.75):
+        assert_store_equals_oracle(_as(y, bf16), ratio)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
 @pytest.mark.parametrize("odd", [1, 3, 5, 7])
 def test_fully_kept_chunks_behind_a_misaligned_kept_count(odd, bf16):
     # A head of small magnitudes of which an odd number is kept, then large magnitudes that are all
