@@ -285,6 +285,58 @@ __device__ __forceinline__ uint32_t valid_mask(int nv, int w) {
   return left >= 32 ? 0xFFFFFFFFu : (left <= 0 ? 0u : ((1u << left) - 1u));
 }
 
+// The chunk's keys inside the bracket (flagged in cw0 / cw1, `c_tot` of them in the warp) if they
+// all are one key, else 0 (no candidate key is 0).  Called for chunks whose slot overflows only,
+// and kept out of line so that the classify kernel's registers are those of its common path; it
+// reads the lane's row again, a piece at a time.
+template <int DT>
+__device__ __noinline__ uint32_t one_key_of_chunk(const unsigned char* region,
+                                                  const typename Elem<DT>::type* x, long long n,
+                                                  long long n_rows_full, long long grow,
+                                                  uint32_t cw0, uint32_t cw1, uint32_t c_tot) {
+  using E = typename Elem<DT>::type;
+  constexpr uint32_t kMask = Elem<DT>::kKeyMask;
+  constexpr int EPR = 128 / sizeof(E);
+  const uint32_t lane = lane_id();
+  const bool ragged = grow >= n_rows_full;
+  const unsigned char* row = region + lane * 128;
+  const int src = __ffs(__ballot_sync(kFull, (cw0 | cw1) != 0u)) - 1;
+  uint32_t k0 = 0;
+  if (static_cast<int>(lane) == src) {
+    const int e = cw0 ? __ffs(cw0) - 1 : 32 + __ffs(cw1) - 1;      // (fp32: cw1 is cw0)
+    if (ragged) {
+      k0 = static_cast<uint32_t>(x[grow * EPR + e]) & kMask;
+    } else {
+      const int byte = e * static_cast<int>(sizeof(E));
+      k0 = static_cast<uint32_t>(*reinterpret_cast<const E*>(row + (((byte >> 4) ^ (lane & 7)) << 4) + (byte & 15))) & kMask;
+    }
+  }
+  k0 = __shfl_sync(kFull, k0, src);
+  uint32_t eq = 0;
+  if (ragged) {                                  // the tensor's last, partial row: element by element
+    for (int e = 0; e < EPR; ++e)
+      if (grow * EPR + e < n) eq += (static_cast<uint32_t>(x[grow * EPR + e]) & kMask) == k0 ? 1u : 0u;
+  } else {
+    const uint32_t c_ge = ge_const(k0 & 0x7FFFu), c_gt = ge_const((k0 & 0x7FFFu) + 1u);   // bf16: k0 <= 0x7FFF
+#pragma unroll 1
+    for (int j = 0; j < 8; ++j) {                // one 16-byte piece at a time: few registers
+      const uint4 v = *reinterpret_cast<const uint4*>(row + ((j ^ (lane & 7)) << 4));
+      const uint32_t c[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (DT == 0) {
+          eq += (c[i] & kMask) == k0 ? 1u : 0u;
+        } else {
+          const uint32_t keys2 = c[i] & 0x7FFF7FFFu;
+          eq += __popc(((keys2 + c_ge) & ~(keys2 + c_gt)) & 0x80008000u);
+        }
+      }
+    }
+  }
+  // (a ragged row's fill is key 0, never a candidate)
+  return __reduce_add_sync(kFull, eq) == c_tot ? k0 : 0u;
+}
+
 // ---- the select's read of the tensor ---------------------------------------------------------
 // Per chunk: how many keys lie above the bracket, how many inside; the keys inside go to the
 // chunk's slot.  A level-A histogram of the keys inside (relative to lo_key) is kept per CTA.
@@ -308,7 +360,7 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
       (reinterpret_cast<uintptr_t>(cs_smem_raw) + kCsAlign - 1) & ~(kCsAlign - 1));
   __shared__ __align__(8) unsigned long long bars[2 * kCsStages];
   __shared__ uint32_t s_hist[kBinsA];
-  __shared__ uint32_t s_tot[2];
+  __shared__ uint32_t s_tot[4];        // keys above / inside the bracket, largest key inside, largest ~key inside
   __shared__ bool s_last;
   const E* __restrict__ x = reinterpret_cast<const E*>(xv);
   E* __restrict__ slots = reinterpret_cast<E*>(slots_v);   // fp32: 32-bit keys, bf16: 16-bit keys
@@ -335,6 +387,8 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
     tc::fence_barrier_init();
     s_tot[0] = 0;
     s_tot[1] = 0;
+    s_tot[2] = 0;
+    s_tot[3] = 0;
   }
   for (int i = tid; i < kBinsA; i += kCsThreads) s_hist[i] = 0;
   __syncthreads();
@@ -433,37 +487,9 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
           // Too many keys inside the bracket for the slot: massive ties.  If they all are one and the
           // same key - here and in every other chunk - that key is the threshold and the counts
           // above are all the count kernel needs; the last CTA checks that through the extremes.
-          const int src = __ffs(__ballot_sync(kFull, cc != 0u)) - 1;
-          uint32_t k0 = 0;
-          if (static_cast<int>(lane) == src) {
-#pragma unroll
-            for (int w = WPL - 1; w >= 0; --w)
-              if (cw[w]) k0 = key_at(32 * w + __ffs(cw[w]) - 1);
-          }
-          k0 = __shfl_sync(kFull, k0, src);
-          uint32_t eq = 0;
-          if (DT == 0) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              eq += ((q[j].x & kMask) == k0 ? 1u : 0u) + ((q[j].y & kMask) == k0 ? 1u : 0u) +
-                    ((q[j].z & kMask) == k0 ? 1u : 0u) + ((q[j].w & kMask) == k0 ? 1u : 0u);
-            }
-          } else {
-            const uint32_t c_ge = ge_const(k0), c_gt = ge_const(k0 + 1u);   // k0 <= 0x7FFF
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const uint32_t c[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const uint32_t keys2 = c[i] & 0x7FFF7FFFu;
-                eq += __popc(((keys2 + c_ge) & ~(keys2 + c_gt)) & 0x80008000u);
-              }
-            }
-          }
-          // (a ragged row's fill is key 0, never a candidate)
-          const bool one_key = __reduce_add_sync(kFull, eq) == c_tot;
-          w_kmax = one_key ? max(w_kmax, k0) : 0xFFFFFFFFu;
-          w_kinv = one_key ? max(w_kinv, ~k0) : 0xFFFFFFFFu;
+          const uint32_t k1 = one_key_of_chunk<DT>(region, x, n, n_rows_full, grow, cw[0], cw[WPL - 1], c_tot);
+          w_kmax = k1 ? max(w_kmax, k1) : 0xFFFFFFFFu;
+          w_kinv = k1 ? max(w_kinv, ~k1) : 0xFFFFFFFFu;
         } else if (c_tot) {
           // keys inside the bracket -> the chunk's slot (order does not matter)
           uint32_t pos = warp_excl_scan(cc);
@@ -491,8 +517,8 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
     if (lane == 0) {
       if (w_above) atomicAdd(&s_tot[0], w_above);
       if (w_cand) atomicAdd(&s_tot[1], w_cand);
-      if (w_kmax) atomicMax(&st->cand_key_max, w_kmax);
-      if (w_kinv) atomicMax(&st->cand_keyinv_max, w_kinv);
+      if (w_kmax) atomicMax(&s_tot[2], w_kmax);
+      if (w_kinv) atomicMax(&s_tot[3], w_kinv);
     }
   }
   __syncthreads();
@@ -501,6 +527,8 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
   if (tid == 0) {
     if (s_tot[0]) atomicAdd(&st->above_total, s_tot[0]);
     if (s_tot[1]) atomicAdd(&st->cand_total, s_tot[1]);
+    if (s_tot[2]) atomicMax(&st->cand_key_max, s_tot[2]);
+    if (s_tot[3]) atomicMax(&st->cand_keyinv_max, s_tot[3]);
   }
   __threadfence();
   __syncthreads();
