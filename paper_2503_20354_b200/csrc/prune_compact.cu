@@ -825,19 +825,23 @@ count_kernel(const void* __restrict__ xv, long long n, uint32_t k, SelectState* 
   const int c_begin = blockIdx.x * per < tiles ? blockIdx.x * per : tiles;
   const int c_end = c_begin + per < tiles ? c_begin + per : tiles;
   unsigned long long acc = 0;
-  if (mode != 1u) {
+  if (mode == 4u) {
+    // every key inside the bracket equals the threshold (the slots may have overflowed): the
+    // classify pass's counts are the answer
+    for (int c = c_begin + tid; c < c_end; c += kSelThreads) {
+      const unsigned long long v = (static_cast<unsigned long long>(__ldg(cnt_gt + c)) << 31) | __ldg(cand_cnt + c);
+      val[c] = v;
+      acc += v;
+    }
+  } else if (mode != 1u) {
     // one thread per chunk: the listed keys above / equal to the threshold complete the counts
     for (int c = c_begin + tid; c < c_end; c += kSelThreads) {
       const uint32_t cc = __ldg(cand_cnt + c), cg = __ldg(cnt_gt + c);
       uint32_t g = cg, q = 0;
-      if (mode == 4u) {       // every key inside the bracket equals the threshold (the slots may have overflowed)
-        q = cc;
-      } else {
-        for_slot_keys<DT>(slots, c, cc, [&](uint32_t key) {
-          g += key > tau ? 1u : 0u;
-          q += key == tau ? 1u : 0u;
-        });
-      }
+      for_slot_keys<DT>(slots, c, cc, [&](uint32_t key) {
+        g += key > tau ? 1u : 0u;
+        q += key == tau ? 1u : 0u;
+      });
       if (tau == 0) {         // lo_key == 1: whatever is neither above nor inside the bracket is 0
         const long long left = n - static_cast<long long>(c) * kChunkElems;
         q += static_cast<uint32_t>(left < kChunkElems ? left : kChunkElems) - cg - cc;
