@@ -154,6 +154,37 @@ def test_weight_gradient_of_a_whole_bench_layer_on_sampled_entries(which, name, 
     assert comp.read_header().status == 0
 
 
+@pytest.mark.parametrize("ratio", [0.0, 0.3, 0.95])
+@pytest.mark.parametrize("name", ["s1b1.conv2",      # 32 groups of 4 channels, 32x32
+                                  "s2b0.conv2",      # 8 channels per group, stride 2, 32x32 -> 16x16
+                                  "s3b1.conv2"])     # 16 channels per group, 8x8
+def test_grouped_weight_gradient_of_a_whole_resnext_layer_on_sampled_entries(name, ratio):
+    """The grouped 3x3 layers of the ResNeXt-29-shaped stack at batch 200, from the oracle's own store
+    (asserted equal to the GPU's bit for bit), at a ratio that takes the mostly-kept rebuild path
+    (0, 0.3) and one that takes the sparse path (0.95).  An entry (o, c', r, s) of a grouped layer
+    is the ungrouped entry (o, group(o) * C/G + c', r, s), so the entry-wise oracle serves; the
+    sample has one entry in every 16 x 16 x tap cell plus random ones.  fp32 kernel: 1e-5."""
+    layer = _layer(W.resnext29(), name)
+    assert layer.groups == 32
+    a = W.activation(layer, seed=0)
+    g = W.grad_out(layer, seed=0, sigma=0.01)
+    comp, ref = assert_store_equals_oracle(a.reshape(-1), ratio)
+    pruned = oracle.decompress(ref["bitmap"], ref["values"], layer.n_act).reshape(layer.act_shape)
+    dwh = B.surgeon_weight_grad(comp, B.layer_desc(layer, B.PATH_TENSOR_CORE), g.cuda()).cpu().numpy()
+    assert dwh.shape == layer.dw_shape
+    gh = g.numpy()
+    cg, og = layer.c_in // layer.groups, layer.c_out // layer.groups
+    rng = np.random.default_rng(6)
+    got, want = [], []
+    for (o, cl, r, s_) in _stratified_entries(dwh.shape, rng, layer.gemm_k):
+        c = (o // og) * cg + cl
+        want.append(oracle.dw_conv2d_entry(pruned, gh, layer.kh, layer.kw, layer.stride, layer.pad, o, c, r, s_))
+        got.append(float(dwh[o, cl, r, s_]))
+    got, want = np.array(got), np.array(want)
+    assert np.linalg.norm(got - want) <= 1e-5 * np.linalg.norm(want)
+    assert np.isfinite(dwh).all()
+
+
 @pytest.mark.parametrize("which,name,ratio", [
     ("wrn", "g1b1.conv1", 0.2), ("r50", "layer1.0.conv1", 0.3), ("vit", "blk0.fc2", 0.4),
 ])
