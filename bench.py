@@ -100,7 +100,7 @@ def get_layers(workload: str, batch):
     if workload == "resnext29":
         return W.resnext29(batch or 200), "ResNeXt-29 (32x4d)-shaped stack, 32x32, batch %d, fp32 activations, grouped 3x3 convolutions" % (batch or 200)
     if workload == "segformer":
-        return W.segformer_b5(1024, batch or 1), "linear layers of a Segformer-B5-shaped encoder, 1024x1024, batch %d, bf16 activations" % (batch or 1)
+        return W.segformer_b5(1024, batch or 1), "blocks of a Segformer-B5-shaped encoder (linear layers, reduction and depthwise convolutions), 1024x1024, batch %d, bf16 activations" % (batch or 1)
     raise SystemExit("unknown workload %r" % workload)
 
 
@@ -716,7 +716,9 @@ def oracle_step(layers, inputs, ratios):
     for l, (a, g), p in zip(layers, inputs, ratios):
         r = oracle.prune_compact(a.reshape(-1), float(p))
         pruned = oracle.decompress(r["bitmap"], r["values"], a.size).reshape(l.act_shape)
-        if l.kind == 1:
+        if l.kind == 1 and l.groups > 1:
+            oracle.dw_conv2d_grouped(pruned, g, l.kh, l.kw, l.stride, l.pad, l.groups)
+        elif l.kind == 1:
             oracle.dw_conv2d(pruned, g, l.kh, l.kw, l.stride, l.pad)
         else:
             oracle.dw_linear(pruned, g)

@@ -174,13 +174,15 @@ def vit_b16(batch: int = 64, dt: int = BF16, blocks: int = 12) -> List[Layer]:
     return L
 
 
-def segformer_b5(image: int = 1024, batch: int = 1, dt: int = BF16, depths=(3, 6, 40, 3)) -> List[Layer]:
-    """The linear layers of a Segformer-B5-shaped encoder (Section 5.1: semantic segmentation at
+def segformer_b5(image: int = 1024, batch: int = 1, dt: int = BF16, depths=(3, 6, 40, 3),
+                 convs: bool = True) -> List[Layer]:
+    """The layers of a Segformer-B5-shaped encoder's blocks (Section 5.1: semantic segmentation at
     batch 1) on an image x image input: four stages of widths 64 / 128 / 320 / 512 on token grids
     of 1/4, 1/8, 1/16 and 1/32 of the image side, attention with keys and values on a grid reduced
-    8 / 4 / 2 / 1 times per side, MLP ratio 4.  Per block: q, kv, proj, fc1, fc2.  The strided
-    reduction convolutions and the depthwise 3x3 convolution of the MLP (a grouped layer) are not
-    part of this stack."""
+    8 / 4 / 2 / 1 times per side, MLP ratio 4.  Per block the linear layers q, kv, proj, fc1, fc2
+    and, with `convs`, the two convolutions: the spatial reduction before kv (kernel = stride =
+    the reduction, stages 1-3) and the depthwise 3x3 between fc1 and fc2 (groups = channels).  The
+    overlapping patch embeddings between the stages are not part of this stack."""
     widths, reductions = (64, 128, 320, 512), (8, 4, 2, 1)
     L = []
     for s in range(4):
@@ -191,9 +193,13 @@ def segformer_b5(image: int = 1024, batch: int = 1, dt: int = BF16, depths=(3, 6
         for b in range(depths[s]):
             n = f"s{s}b{b}"
             L.append(linear(n + ".q", batch * t_q, c, c, "normal", dt, t_q))
+            if convs and reductions[s] > 1:
+                L.append(conv(n + ".sr", batch, c, side, c, reductions[s], reductions[s], 0, "normal", dt))
             L.append(linear(n + ".kv", batch * t_kv, c, 2 * c, "normal", dt, t_kv))
             L.append(linear(n + ".proj", batch * t_q, c, c, "normal", dt, t_q))
             L.append(linear(n + ".fc1", batch * t_q, c, 4 * c, "normal", dt, t_q))
+            if convs:
+                L.append(conv(n + ".dwconv", batch, 4 * c, side, 4 * c, 3, 1, 1, "normal", dt, groups=4 * c))
             L.append(linear(n + ".fc2", batch * t_q, 4 * c, c, "gelu_normal", dt, t_q))
     return L
 

@@ -1,7 +1,9 @@
-"""GPU parity on Segformer-B5-shaped linear layers (Section 5.1: the segmentation model, batch 1):
-widths 64 / 128 / 320 / 512, MLP ratio 4, keys and values on a reduced token grid.  One block per
-stage on a 256x256 image (4096 / 1024 / 256 / 64 tokens), ratios from Eq. 5-7 over the stack:
-stores bit for bit, weight gradients within the path's tolerance of the fp64 oracle."""
+"""GPU parity on the layers of Segformer-B5-shaped blocks (Section 5.1: the segmentation model, batch
+1): widths 64 / 128 / 320 / 512, MLP ratio 4, keys and values on a token grid reduced by a strided
+convolution, a depthwise 3x3 convolution inside the MLP.  One block per stage on a 256x256 image
+(4096 / 1024 / 256 / 64 tokens), ratios from Eq. 5-7 over the stack: stores bit for bit, weight
+gradients within the path's tolerance of the fp64 oracle (the depthwise layers run the fp32
+grouped kernel on both paths)."""
 import numpy as np
 import pytest
 import torch
@@ -24,11 +26,16 @@ def _ratios():
 
 
 def test_stack_shape():
+    lin = W.segformer_b5(convs=False)
+    assert len(lin) == 5 * (3 + 6 + 40 + 3)
+    assert [l.batch for l in lin[:5]] == [65536, 1024, 65536, 65536, 65536]
+    assert (lin[-1].c_in, lin[-1].c_out, lin[-1].batch) == (2048, 512, 1024)
     full = W.segformer_b5()
-    assert len(full) == 5 * (3 + 6 + 40 + 3)
-    assert [l.batch for l in full[:5]] == [65536, 1024, 65536, 65536, 65536]
-    assert (full[-1].c_in, full[-1].c_out, full[-1].batch) == (2048, 512, 1024)
-    assert len(LAYERS) == 20 and LAYERS[1].batch == 64      # a 64 x 64 token grid reduced 8 times per side
+    assert len(full) == len(lin) + (3 + 6 + 40) + (3 + 6 + 40 + 3)      # reductions in stages 1-3, a depthwise conv per block
+    sr, dwc = full[1], full[5]
+    assert (sr.name, sr.kh, sr.stride, sr.pad, sr.h, sr.c_in, sr.c_out) == ("s0b0.sr", 8, 8, 0, 256, 64, 64)
+    assert (dwc.name, dwc.groups, dwc.c_in, dwc.kh, dwc.h) == ("s0b0.dwconv", 256, 256, 3, 256)
+    assert len(LAYERS) == 20 + 3 + 4 and LAYERS[2].batch == 64      # a 64 x 64 token grid reduced 8 times per side
 
 
 @pytest.mark.parametrize("path", [B.PATH_TENSOR_CORE, B.PATH_FP32])
@@ -42,9 +49,14 @@ def test_layer_store_and_weight_gradient(li, path):
     dw = B.surgeon_weight_grad(comp, B.layer_desc(layer, path), g.cuda())
     torch.cuda.synchronize()
     pruned = oracle.decompress(ref["bitmap"], ref["values"], layer.n_act)
-    want = oracle_dw(layer, pruned, g.numpy())
-    assert dw.shape == (layer.c_out, layer.c_in)
+    if layer.groups > 1:
+        want = oracle.dw_conv2d_grouped(pruned.reshape(layer.act_shape), g.numpy(), layer.kh, layer.kw,
+                                        layer.stride, layer.pad, layer.groups)
+    else:
+        want = oracle_dw(layer, pruned, g.numpy())
+    assert tuple(dw.shape) == tuple(layer.dw_shape)
+    tol = 1e-5 if layer.groups > 1 else TOL[path]
     if not want.any():
         assert not dw.cpu().numpy().any()
     else:
-        assert rel_frobenius(dw.cpu().numpy(), want) <= TOL[path]
+        assert rel_frobenius(dw.cpu().numpy(), want) <= tol
