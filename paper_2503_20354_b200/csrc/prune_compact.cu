@@ -369,9 +369,6 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
   const uint32_t lane = lane_id();
   if (st->mode == 1u) return;          // the sample found no usable bracket
   const uint32_t lo_key = st->lo_key, hi_key = st->hi_key;
-  // keys inside the bracket: key - cand_lo <= range (nothing when the bracket holds only key 0)
-  const uint32_t cand_lo = hi_key >= lo_key ? lo_key : 0xFFFFFFFFu;
-  const uint32_t range = hi_key >= lo_key ? hi_key - lo_key : 0u;
   const uint32_t shiftA = st->shiftA;
   // bf16: the two comparisons as additions on packed pairs of keys (hi_key <= 0x7FFF there)
   const uint32_t c_above = ge_const(hi_key >= 0x7FFFu ? 0x8000u : hi_key + 1u);
@@ -429,21 +426,26 @@ classify_kernel(const __grid_constant__ CUtensorMap xmap, const void* __restrict
         uint32_t cw[WPL];
         uint32_t ac = 0, cc = 0;
         if (DT == 0) {
-          uint32_t aw = 0;
-          cw[0] = 0;
+          // Keys are below 2^31, so the sign bit of (hi_key - key) says key > hi_key and that of
+          // (key - lo) says key < lo; a funnel shift collects it: two instructions per element
+          // and comparison.  Element e ends up in bit 31 - e, one bit reversal per word puts it back.
+          uint32_t aw = 0, lw = 0;
+          const uint32_t lo_cmp = hi_key >= lo_key ? lo_key : 0x7FFFFFFFu;   // bracket {0}: nothing is a candidate
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const uint32_t c[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const uint32_t key = c[i] & kMask;
-              aw |= (key > hi_key ? 1u : 0u) << (4 * j + i);
-              cw[0] |= (key - cand_lo <= range ? 1u : 0u) << (4 * j + i);
+              aw = __funnelshift_l(hi_key - key, aw, 1);
+              lw = __funnelshift_l(key - lo_cmp, lw, 1);
             }
           }
           const uint32_t vm = valid_mask(nv, 0);
-          cw[0] &= vm;
-          ac = __popc(aw & vm);
+          aw = __brev(aw) & vm;
+          cw[0] = ~__brev(lw) & ~aw & vm;
+          if (hi_key < lo_key) cw[0] = 0u;
+          ac = __popc(aw);
         } else {
           // above: key >= hi_key + 1; inside the bracket: key >= lo_key and not above
           uint32_t ga[WPL], gl[WPL];
@@ -1316,7 +1318,9 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           if (DT == 0) {
-            word[0] |= ((c[i] & kMask) >= thr ? 1u : 0u) << (4 * j + i);
+            // key < thr is the sign bit of key - thr (key < 2^31, thr <= 2^31); collected by a funnel
+            // shift with element e in bit 31 - e, put back in order below
+            word[0] = __funnelshift_l((c[i] & kMask) - thr, word[0], 1);
           } else {
             const int pw = 4 * j + i;             // packed word of the row: elements 2pw, 2pw + 1
             word[(pw >> 4) % WPL] |= pair_flags(c[i] & 0x7FFF7FFFu, c_thr, pw & 15);
@@ -1326,6 +1330,8 @@ compact_stream_kernel(const __grid_constant__ CUtensorMap xmap, const void* __re
       if (DT != 0) {
 #pragma unroll
         for (int w = 0; w < WPL; ++w) word[w] = pairs_to_element_order(word[w]);
+      } else {
+        word[0] = ~__brev(word[0]);
       }
 #pragma unroll
       for (int w = 0; w < WPL; ++w) {
